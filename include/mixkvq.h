@@ -1,0 +1,149 @@
+/*
+ * mixkvq.h — C ABI of the MixKVQ decode hot path for NVIDIA B200 (sm_100a).
+ *
+ * MixKVQ (arxiv 2512.19206) keeps the KV cache of a decoder in three stores per (layer, batch element,
+ * KV head) "stream" (Appendix D, "Storage Layout"): bit-packed low-precision codes, the critical key
+ * channels in BF16, and a full-precision residual window of the newest <= R tokens.  This library
+ * implements the three data-parallel steps of one decode step on that cache:
+ *
+ *   mixkvq_select_channels   query-aware key-channel scoring and three-tier assignment (Section 4.2)
+ *   mixkvq_quantize_append   append to the residual window and, every R tokens, quantize and pack
+ *                            (Section 4.2 workflow, Eq. 2; Appendix D.1 lazy update, D.2 accumulator)
+ *   mixkvq_decode_attention  softmax(q K~^T * scale) V~ over the mixed-precision cache (Eq. 1, Eq. 3)
+ *
+ * Conventions
+ *   - Every pointer named *_dev is DEVICE memory, owned by the caller, 16-byte aligned.  The library
+ *     allocates no device memory and frees none.  `mixkvq_cache*` is a small HOST object.
+ *   - bf16 tensors are passed as `const void*` (raw 16-bit bfloat16, row-major, innermost dim = head_dim).
+ *   - `stream` is a `cudaStream_t` passed as `void*` (NULL = default stream).  All work is enqueued on
+ *     it; only mixkvq_query_status synchronizes.
+ *   - Every function returns MIXKVQ_OK (0) or a negative MIXKVQ_E_* code.  Nothing aborts, traps or
+ *     throws.  Conditions discovered on the device (extras arena full, a staged copy that never arrived)
+ *     set a sticky device status word that mixkvq_query_status returns.
+ *   - All sequences of the batch have the same length (the library tracks it per layer on the host).
+ *   - head_dim must be 128.
+ */
+#ifndef MIXKVQ_H_
+#define MIXKVQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  MIXKVQ_OK = 0,
+  MIXKVQ_E_INVALID_ARG = -1,          /* null pointer, bad dimension, layer out of range            */
+  MIXKVQ_E_UNSUPPORTED = -2,          /* head_dim != 128, v_bits != 2, unsupported R or G            */
+  MIXKVQ_E_ALIGNMENT = -3,            /* a device pointer is not 16-byte aligned                     */
+  MIXKVQ_E_BUFFER_TOO_SMALL = -4,     /* cache memory or attention workspace smaller than required   */
+  MIXKVQ_E_CAPACITY = -5,             /* append would exceed max_tokens                              */
+  MIXKVQ_E_CUDA = -6,                 /* a CUDA runtime call or kernel launch reported an error      */
+  MIXKVQ_E_EMPTY = -7                 /* attention or selection requested on a layer with no tokens  */
+};
+
+/* bits of the sticky device status word */
+enum {
+  MIXKVQ_DEV_EXTRAS_FULL = 1,         /* a block's promoted channels did not fit the extras arena: that
+                                         block was not written and the layer's cache is invalid      */
+  MIXKVQ_DEV_COPY_TIMEOUT = 2         /* a bounded wait for a staged bulk copy gave up               */
+};
+
+typedef struct mixkvq_config {
+  int32_t n_layers;
+  int32_t batch;                      /* B                                                           */
+  int32_t n_q_heads;                  /* Hq, a multiple of n_kv_heads, Hq/Hkv <= 8                   */
+  int32_t n_kv_heads;                 /* Hkv                                                         */
+  int32_t head_dim;                   /* D, must be 128                                              */
+  int32_t max_tokens;                 /* capacity per sequence                                       */
+  int32_t residual_len;               /* R (Section 5.1: 128): multiple of 32, <= 256, multiple of G */
+  int32_t group_size;                 /* G (Section 5.1: 32): 32, 64 or 128                          */
+  int32_t v_bits;                     /* value bit-width, must be 2 (Section 4.2)                    */
+  int32_t score_bits;                 /* B of the sensitivity score S_d (Section 4.2), 2 or 4        */
+  float tau_bf16;                     /* A_d >  tau_bf16            -> BF16                          */
+  float tau_u4;                       /* tau_u4 < A_d <= tau_bf16   -> UINT4, else UINT2             */
+  int32_t importance_mode;            /* 0: |q| accumulated within the current window (Section 4.2);
+                                         1: cumulative over the whole history (Appendix D.2)         */
+  int32_t reserved;
+  uint64_t extras_budget_bytes;       /* per stream, for promoted channels; 0 = library default
+                                         (1/8 of the bf16 size of max_tokens keys)                   */
+} mixkvq_config;
+
+typedef struct mixkvq_cache mixkvq_cache;
+
+/* Byte offsets (from the start of the cache memory) and strides of one layer's arrays, for tools
+ * and tests that inspect the cache.  The element formats are part of the library's documentation. */
+typedef struct mixkvq_layout_desc {
+  uint64_t state_off, state_stride;       /* per stream: acc fp64[128], cnt u32, extras_used16 u32   */
+  uint64_t table_off, table_stride;       /* per stream: max_blocks entries of 8 bytes               */
+  uint64_t resk_off, resk_stride;         /* per stream: [R][128] bf16                               */
+  uint64_t resv_off, resv_stride;         /* per stream: [128][R] bf16                               */
+  uint64_t base_off, base_stride;         /* per stream: max_blocks blocks of base_bytes             */
+  uint64_t extras_off, extras_stride;     /* per stream: extras arena                                */
+  uint64_t base_bytes;                    /* size of one block's fixed part                          */
+  uint32_t max_blocks, n_streams;
+  uint32_t n_blocks, residual_tokens;     /* current fill of this layer (same for all streams)       */
+} mixkvq_layout_desc;
+
+/* Sizes the caller must provide: the cache memory for all layers and the workspace of one
+ * mixkvq_decode_attention call (split partials).  Host-only, no CUDA call. */
+int mixkvq_cache_bytes(const mixkvq_config* cfg, size_t* cache_bytes, size_t* attn_workspace_bytes);
+
+/* Creates the host handle over caller-owned device memory and enqueues the zeroing of the per-stream
+ * state on `stream`.  cache_dev must hold at least the size reported by mixkvq_cache_bytes. */
+int mixkvq_cache_init(const mixkvq_config* cfg, void* cache_dev, size_t bytes, void* stream, mixkvq_cache** out);
+
+/* Frees the host handle only. */
+int mixkvq_cache_destroy(mixkvq_cache* cache);
+
+/* Empties one layer (layer >= 0) or all layers (layer < 0): lengths to zero, state re-zeroed on `stream`. */
+int mixkvq_cache_reset(mixkvq_cache* cache, int layer, void* stream);
+
+/* (1) Section 4.2: I_d (mean |q| over the window and the GQA group), S_d (key range over the window
+ * divided by 2^score_bits - 1), A_d = I_d * S_d, and the tier of every key channel for the CURRENT
+ * residual window of `layer`; a pure function of the cache state.
+ *   tiers_dev    [B, Hkv, 128] uint8: 0 = UINT2, 1 = UINT4, 2 = BF16
+ *   salience_dev [B, Hkv, 128] double A_d, or NULL */
+int mixkvq_select_channels(mixkvq_cache* cache, int layer, uint8_t* tiers_dev, double* salience_dev, void* stream);
+
+/* Stateless form of (1) on explicit windows: q_dev [B, Hq, Lq, 128] bf16, k_dev [B, Hkv, Lk, 128] bf16. */
+int mixkvq_select_channels_raw(const void* q_dev, const void* k_dev, int batch, int n_q_heads, int n_kv_heads,
+                               int lq, int lk, int score_bits, float tau_bf16, float tau_u4,
+                               uint8_t* tiers_dev, double* salience_dev, void* stream);
+
+/* (2) Appends n_tokens (1 = decode step, > 1 = prefill / bulk) post-RoPE tokens to `layer`, in token order:
+ * for each token, if the residual window already holds R tokens it is first scored, quantized (keys per
+ * channel at the tier's bit-width, values per token at 2 bits, groups of G, Eq. 2) and packed; then the
+ * token is stored in the window and |q| is added to the importance accumulator.
+ *   k_dev, v_dev [B, Hkv, n_tokens, 128] bf16;  q_dev [B, Hq, n_tokens, 128] bf16 */
+int mixkvq_quantize_append(mixkvq_cache* cache, int layer, const void* k_dev, const void* v_dev, const void* q_dev,
+                           int n_tokens, void* stream);
+
+/* (3) Eq. 1 for one decode step of `layer` over [packed blocks, residual window], keys and values
+ * dequantized on the fly (Eq. 3).
+ *   q_dev [B, Hq, 128] bf16  ->  out_dev [B, Hq, 128] float
+ *   workspace_dev: at least attn_workspace_bytes (mixkvq_cache_bytes); contents are scratch */
+int mixkvq_decode_attention(mixkvq_cache* cache, int layer, const void* q_dev, float* out_dev, float softmax_scale,
+                            void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/* Selects the decode-attention kernel: 0 = tensor-core kernel (default), 1 = plain-ALU kernel
+ * (kept for comparison; same results within tolerance, much slower). */
+int mixkvq_set_attention_kernel(mixkvq_cache* cache, int kind);
+
+/* Synchronizes `stream`, then returns the sticky device status word (MIXKVQ_DEV_* bits). */
+int mixkvq_query_status(mixkvq_cache* cache, int* device_status, void* stream);
+
+/* Where one layer's arrays live inside the cache memory, and how full the layer is. */
+int mixkvq_cache_describe(const mixkvq_cache* cache, int layer, mixkvq_layout_desc* out);
+
+/* Number of kernels launched by this handle since it was created (diagnostic). */
+uint64_t mixkvq_launch_count(const mixkvq_cache* cache);
+
+const char* mixkvq_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MIXKVQ_H_ */

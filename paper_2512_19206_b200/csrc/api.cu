@@ -1,0 +1,289 @@
+// Host side of the C ABI: argument checking, the cache memory map, per-layer length tracking and the
+// scheduling of the kernels.  No device allocation happens here.
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+using namespace mixkvq;
+
+struct mixkvq_cache {
+  mixkvq_config cfg;
+  char* mem;
+  size_t bytes;
+  int S, g, R, G, U, NG, VG, max_blocks;
+  uint32_t base_bytes, unit_bytes;
+  uint64_t extras_budget;
+  // byte offsets inside one layer and per-stream strides
+  uint64_t state_off, table_off, resk_off, resv_off, base_off, extras_off, layer_stride;
+  uint64_t state_stride, table_stride, resk_stride, resv_stride, base_stride, extras_stride;
+  std::vector<int> n_blocks, r;
+  int n_sms;
+  int attn_kind;
+  uint64_t launches;
+};
+
+namespace {
+
+constexpr uint64_t kHeaderBytes = 256;   // device status word lives at offset 0
+
+uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+
+int check_config(const mixkvq_config* c) {
+  if (!c) return MIXKVQ_E_INVALID_ARG;
+  if (c->n_layers < 1 || c->batch < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1 || c->max_tokens < 1)
+    return MIXKVQ_E_INVALID_ARG;
+  if (c->n_q_heads % c->n_kv_heads != 0) return MIXKVQ_E_INVALID_ARG;
+  if (c->head_dim != kD || c->v_bits != 2) return MIXKVQ_E_UNSUPPORTED;
+  if (c->n_q_heads / c->n_kv_heads > 8) return MIXKVQ_E_UNSUPPORTED;
+  if (c->group_size != 32 && c->group_size != 64 && c->group_size != 128) return MIXKVQ_E_UNSUPPORTED;
+  if (c->residual_len < 32 || c->residual_len > 256 || c->residual_len % 32 != 0 ||
+      c->residual_len % c->group_size != 0)
+    return MIXKVQ_E_UNSUPPORTED;
+  if (c->score_bits != 2 && c->score_bits != 4) return MIXKVQ_E_UNSUPPORTED;
+  if (c->importance_mode != 0 && c->importance_mode != 1) return MIXKVQ_E_INVALID_ARG;
+  return MIXKVQ_OK;
+}
+
+// Fills the geometry and the memory map; returns total bytes.
+uint64_t plan(const mixkvq_config* c, mixkvq_cache* h) {
+  h->cfg = *c;
+  h->S = c->batch * c->n_kv_heads;
+  h->g = c->n_q_heads / c->n_kv_heads;
+  h->R = c->residual_len;
+  h->G = c->group_size;
+  h->U = h->R / 32;
+  h->NG = h->R / h->G;
+  h->VG = kD / h->G;
+  h->max_blocks = (c->max_tokens + h->R - 1) / h->R;
+  h->unit_bytes = 2048u + 128u * h->VG;
+  h->base_bytes = (uint32_t)h->NG * 512u + (uint32_t)h->U * h->unit_bytes;
+  h->extras_budget = c->extras_budget_bytes ? align_up(c->extras_budget_bytes, 16)
+                                            : align_up((uint64_t)h->max_blocks * h->R * 32, 256);
+  h->state_stride = kStateBytes;
+  h->table_stride = align_up((uint64_t)h->max_blocks * 8, 256);
+  h->resk_stride = (uint64_t)h->R * 256;
+  h->resv_stride = (uint64_t)h->R * 256;
+  h->base_stride = (uint64_t)h->max_blocks * h->base_bytes;
+  h->extras_stride = align_up(h->extras_budget, 256);
+  uint64_t off = 0;
+  h->state_off = off;  off = align_up(off + h->state_stride * h->S, 256);
+  h->table_off = off;  off = align_up(off + h->table_stride * h->S, 256);
+  h->resk_off = off;   off = align_up(off + h->resk_stride * h->S, 256);
+  h->resv_off = off;   off = align_up(off + h->resv_stride * h->S, 256);
+  h->base_off = off;   off = align_up(off + h->base_stride * h->S, 256);
+  h->extras_off = off; off = align_up(off + h->extras_stride * h->S, 256);
+  h->layer_stride = off;
+  return kHeaderBytes + h->layer_stride * (uint64_t)c->n_layers;
+}
+
+size_t workspace_bytes(int S) { return (size_t)(kMaxCtas + S) * kPartialFloats * sizeof(float); }
+
+LayerView view(const mixkvq_cache* h, int layer) {
+  LayerView v{};
+  v.B = h->cfg.batch; v.Hq = h->cfg.n_q_heads; v.Hkv = h->cfg.n_kv_heads; v.g = h->g;
+  v.R = h->R; v.G = h->G; v.U = h->U; v.NG = h->NG; v.VG = h->VG;
+  v.max_blocks = h->max_blocks;
+  v.n_blocks = h->n_blocks[layer]; v.r = h->r[layer];
+  v.base_bytes = h->base_bytes; v.unit_bytes = h->unit_bytes;
+  v.extras_budget = h->extras_budget;
+  v.score_bits = h->cfg.score_bits; v.importance_mode = h->cfg.importance_mode;
+  v.tau_bf16 = h->cfg.tau_bf16; v.tau_u4 = h->cfg.tau_u4;
+  char* L = h->mem + kHeaderBytes + h->layer_stride * (uint64_t)layer;
+  v.state = L + h->state_off;   v.state_stride = h->state_stride;
+  v.table = L + h->table_off;   v.table_stride = h->table_stride;
+  v.resk = L + h->resk_off;     v.resk_stride = h->resk_stride;
+  v.resv = L + h->resv_off;     v.resv_stride = h->resv_stride;
+  v.base = L + h->base_off;     v.base_stride = h->base_stride;
+  v.extras = L + h->extras_off; v.extras_stride = h->extras_stride;
+  v.status = reinterpret_cast<uint32_t*>(h->mem);
+  return v;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int zero_layer_state(mixkvq_cache* h, int layer, cudaStream_t st) {
+  char* L = h->mem + kHeaderBytes + h->layer_stride * (uint64_t)layer;
+  if (cudaMemsetAsync(L + h->state_off, 0, h->state_stride * h->S, st) != cudaSuccess) return MIXKVQ_E_CUDA;
+  h->n_blocks[layer] = 0;
+  h->r[layer] = 0;
+  return MIXKVQ_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int mixkvq_cache_bytes(const mixkvq_config* cfg, size_t* cache_bytes, size_t* attn_workspace_bytes) {
+  int rc = check_config(cfg);
+  if (rc != MIXKVQ_OK) return rc;
+  mixkvq_cache tmp{};
+  uint64_t total = plan(cfg, &tmp);
+  if (cache_bytes) *cache_bytes = (size_t)total;
+  if (attn_workspace_bytes) *attn_workspace_bytes = workspace_bytes(tmp.S);
+  return MIXKVQ_OK;
+}
+
+int mixkvq_cache_init(const mixkvq_config* cfg, void* cache_dev, size_t bytes, void* stream, mixkvq_cache** out) {
+  int rc = check_config(cfg);
+  if (rc != MIXKVQ_OK) return rc;
+  if (!cache_dev || !out) return MIXKVQ_E_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(cache_dev) & 255u) return MIXKVQ_E_ALIGNMENT;
+  mixkvq_cache* h = new (std::nothrow) mixkvq_cache();
+  if (!h) return MIXKVQ_E_INVALID_ARG;
+  uint64_t total = plan(cfg, h);
+  if (bytes < total) { delete h; return MIXKVQ_E_BUFFER_TOO_SMALL; }
+  h->mem = static_cast<char*>(cache_dev);
+  h->bytes = bytes;
+  h->n_blocks.assign(cfg->n_layers, 0);
+  h->r.assign(cfg->n_layers, 0);
+  h->attn_kind = 0;
+  h->launches = 0;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&h->n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+    delete h;
+    return MIXKVQ_E_CUDA;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(h->mem, 0, kHeaderBytes, st) != cudaSuccess) { delete h; return MIXKVQ_E_CUDA; }
+  for (int l = 0; l < cfg->n_layers; ++l)
+    if (zero_layer_state(h, l, st) != MIXKVQ_OK) { delete h; return MIXKVQ_E_CUDA; }
+  if (attention_mma_setup() != cudaSuccess) { delete h; return MIXKVQ_E_CUDA; }
+  *out = h;
+  return MIXKVQ_OK;
+}
+
+int mixkvq_cache_destroy(mixkvq_cache* cache) {
+  delete cache;
+  return MIXKVQ_OK;
+}
+
+int mixkvq_cache_reset(mixkvq_cache* cache, int layer, void* stream) {
+  if (!cache || layer >= cache->cfg.n_layers) return MIXKVQ_E_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (layer >= 0) return zero_layer_state(cache, layer, st);
+  if (cudaMemsetAsync(cache->mem, 0, kHeaderBytes, st) != cudaSuccess) return MIXKVQ_E_CUDA;
+  for (int l = 0; l < cache->cfg.n_layers; ++l)
+    if (zero_layer_state(cache, l, st) != MIXKVQ_OK) return MIXKVQ_E_CUDA;
+  return MIXKVQ_OK;
+}
+
+int mixkvq_select_channels(mixkvq_cache* cache, int layer, uint8_t* tiers_dev, double* salience_dev, void* stream) {
+  if (!cache || !tiers_dev || layer < 0 || layer >= cache->cfg.n_layers) return MIXKVQ_E_INVALID_ARG;
+  if (cache->r[layer] == 0) return MIXKVQ_E_EMPTY;
+  LayerView lv = view(cache, layer);
+  cache->launches += 1;
+  return launch_select_window(lv, tiers_dev, salience_dev, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? MIXKVQ_OK : MIXKVQ_E_CUDA;
+}
+
+int mixkvq_select_channels_raw(const void* q_dev, const void* k_dev, int batch, int n_q_heads, int n_kv_heads,
+                               int lq, int lk, int score_bits, float tau_bf16, float tau_u4,
+                               uint8_t* tiers_dev, double* salience_dev, void* stream) {
+  if (!q_dev || !k_dev || !tiers_dev || batch < 1 || n_q_heads < 1 || n_kv_heads < 1 || lq < 1 || lk < 1 ||
+      n_q_heads % n_kv_heads != 0)
+    return MIXKVQ_E_INVALID_ARG;
+  if (score_bits != 2 && score_bits != 4) return MIXKVQ_E_UNSUPPORTED;
+  return launch_select_raw(q_dev, k_dev, batch, n_q_heads, n_kv_heads, lq, lk, score_bits, tau_bf16, tau_u4,
+                           tiers_dev, salience_dev, static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? MIXKVQ_OK : MIXKVQ_E_CUDA;
+}
+
+int mixkvq_quantize_append(mixkvq_cache* cache, int layer, const void* k_dev, const void* v_dev, const void* q_dev,
+                           int n_tokens, void* stream) {
+  if (!cache || !k_dev || !v_dev || !q_dev || layer < 0 || layer >= cache->cfg.n_layers || n_tokens < 1)
+    return MIXKVQ_E_INVALID_ARG;
+  if (!aligned16(k_dev) || !aligned16(v_dev) || !aligned16(q_dev)) return MIXKVQ_E_ALIGNMENT;
+  const long long have = (long long)cache->n_blocks[layer] * cache->R + cache->r[layer];
+  if (have + n_tokens > cache->cfg.max_tokens) return MIXKVQ_E_CAPACITY;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int t = 0;
+  while (t < n_tokens) {
+    if (cache->r[layer] == cache->R) {
+      LayerView lv = view(cache, layer);
+      if (launch_flush(lv, st) != cudaSuccess) return MIXKVQ_E_CUDA;
+      cache->launches += 1;
+      cache->n_blocks[layer] += 1;
+      cache->r[layer] = 0;
+    }
+    const int m = (n_tokens - t < cache->R - cache->r[layer]) ? n_tokens - t : cache->R - cache->r[layer];
+    LayerView lv = view(cache, layer);
+    if (launch_append(lv, k_dev, v_dev, q_dev, n_tokens, t, m, st) != cudaSuccess) return MIXKVQ_E_CUDA;
+    cache->launches += 1;
+    cache->r[layer] += m;
+    t += m;
+  }
+  return MIXKVQ_OK;
+}
+
+int mixkvq_decode_attention(mixkvq_cache* cache, int layer, const void* q_dev, float* out_dev, float softmax_scale,
+                            void* workspace_dev, size_t workspace_bytes_given, void* stream) {
+  if (!cache || !q_dev || !out_dev || !workspace_dev || layer < 0 || layer >= cache->cfg.n_layers)
+    return MIXKVQ_E_INVALID_ARG;
+  if (!aligned16(q_dev) || !aligned16(out_dev) || !aligned16(workspace_dev)) return MIXKVQ_E_ALIGNMENT;
+  if (workspace_bytes_given < workspace_bytes(cache->S)) return MIXKVQ_E_BUFFER_TOO_SMALL;
+  if (cache->n_blocks[layer] == 0 && cache->r[layer] == 0) return MIXKVQ_E_EMPTY;
+  LayerView lv = view(cache, layer);
+  int launches = 0;
+  cudaError_t e;
+  if (cache->attn_kind == 1)
+    e = launch_attention_simt(lv, q_dev, out_dev, softmax_scale, static_cast<float*>(workspace_dev), cache->n_sms,
+                              static_cast<cudaStream_t>(stream), &launches);
+  else
+    e = launch_attention_mma(lv, q_dev, out_dev, softmax_scale, static_cast<float*>(workspace_dev), cache->n_sms,
+                             static_cast<cudaStream_t>(stream), &launches);
+  cache->launches += launches;
+  return e == cudaSuccess ? MIXKVQ_OK : MIXKVQ_E_CUDA;
+}
+
+int mixkvq_set_attention_kernel(mixkvq_cache* cache, int kind) {
+  if (!cache || (kind != 0 && kind != 1)) return MIXKVQ_E_INVALID_ARG;
+  cache->attn_kind = kind;
+  return MIXKVQ_OK;
+}
+
+int mixkvq_query_status(mixkvq_cache* cache, int* device_status, void* stream) {
+  if (!cache || !device_status) return MIXKVQ_E_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  uint32_t w = 0;
+  if (cudaMemcpyAsync(&w, cache->mem, sizeof(w), cudaMemcpyDeviceToHost, st) != cudaSuccess) return MIXKVQ_E_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return MIXKVQ_E_CUDA;
+  *device_status = (int)w;
+  return MIXKVQ_OK;
+}
+
+int mixkvq_cache_describe(const mixkvq_cache* cache, int layer, mixkvq_layout_desc* out) {
+  if (!cache || !out || layer < 0 || layer >= cache->cfg.n_layers) return MIXKVQ_E_INVALID_ARG;
+  const uint64_t L = kHeaderBytes + cache->layer_stride * (uint64_t)layer;
+  out->state_off = L + cache->state_off;   out->state_stride = cache->state_stride;
+  out->table_off = L + cache->table_off;   out->table_stride = cache->table_stride;
+  out->resk_off = L + cache->resk_off;     out->resk_stride = cache->resk_stride;
+  out->resv_off = L + cache->resv_off;     out->resv_stride = cache->resv_stride;
+  out->base_off = L + cache->base_off;     out->base_stride = cache->base_stride;
+  out->extras_off = L + cache->extras_off; out->extras_stride = cache->extras_stride;
+  out->base_bytes = cache->base_bytes;
+  out->max_blocks = (uint32_t)cache->max_blocks;
+  out->n_streams = (uint32_t)cache->S;
+  out->n_blocks = (uint32_t)cache->n_blocks[layer];
+  out->residual_tokens = (uint32_t)cache->r[layer];
+  return MIXKVQ_OK;
+}
+
+uint64_t mixkvq_launch_count(const mixkvq_cache* cache) { return cache ? cache->launches : 0; }
+
+const char* mixkvq_status_string(int status) {
+  switch (status) {
+    case MIXKVQ_OK: return "ok";
+    case MIXKVQ_E_INVALID_ARG: return "invalid argument";
+    case MIXKVQ_E_UNSUPPORTED: return "unsupported configuration";
+    case MIXKVQ_E_ALIGNMENT: return "device pointer not 16-byte aligned";
+    case MIXKVQ_E_BUFFER_TOO_SMALL: return "cache memory or workspace too small";
+    case MIXKVQ_E_CAPACITY: return "append exceeds max_tokens";
+    case MIXKVQ_E_CUDA: return "CUDA error";
+    case MIXKVQ_E_EMPTY: return "layer holds no tokens";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

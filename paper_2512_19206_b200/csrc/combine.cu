@@ -1,0 +1,46 @@
+// Log-sum-exp merge of the split partials of decode attention.
+#include "common.cuh"
+
+namespace mixkvq {
+
+// Partials live at ws[slot * kPartialFloats + h * 130 + {0: m (log2 domain), 1: l, 2..129: o}].
+// mode 0: stream s owns slots [s*n, s*n + n).  mode 1: the attention grid of `n` CTAs split the
+// S*units_per_stream work units evenly; CTA c wrote its part of stream s to slot c + s.
+__global__ void __launch_bounds__(128)
+combine_kernel(const float* __restrict__ ws, float* __restrict__ out, int g, int Hkv, int Hq, int mode, int n,
+               long long units_per_stream, int S) {
+  const int s = blockIdx.x, c = threadIdx.x;
+  int first, count;
+  if (mode == 0) {
+    first = s * n;
+    count = n;
+  } else {
+    const long long total = units_per_stream * S;
+    const long long x0 = units_per_stream * s, x1 = units_per_stream * (s + 1) - 1;
+    const int c0 = (int)(((x0 + 1) * n - 1) / total), c1 = (int)(((x1 + 1) * n - 1) / total);
+    first = c0 + s;
+    count = c1 - c0 + 1;
+  }
+  const int b = s / Hkv, hk = s % Hkv;
+  for (int h = 0; h < g; ++h) {
+    float M = -INFINITY;
+    for (int i = 0; i < count; ++i) M = fmaxf(M, ws[(size_t)(first + i) * kPartialFloats + h * 130]);
+    float l = 0.f, o = 0.f;
+    for (int i = 0; i < count; ++i) {
+      const float* p = ws + (size_t)(first + i) * kPartialFloats + h * 130;
+      const float m = p[0];
+      const float f = (m == -INFINITY) ? 0.f : exp2f(m - M);
+      l += f * p[1];
+      o += f * p[2 + c];
+    }
+    out[((size_t)b * Hq + hk * g + h) * kD + c] = o / l;
+  }
+}
+
+cudaError_t launch_combine(const float* ws, float* out, int g, int Hkv, int Hq, int mode, int n,
+                           long long units_per_stream, int S, cudaStream_t stream) {
+  combine_kernel<<<S, 128, 0, stream>>>(ws, out, g, Hkv, Hq, mode, n, units_per_stream, S);
+  return cudaGetLastError();
+}
+
+}  // namespace mixkvq

@@ -1,0 +1,128 @@
+// Internal definitions shared by the kernels: per-layer views of the caller-owned cache memory,
+// the byte layout constants, and the small numeric helpers whose results must be bit-exact.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/mixkvq.h"
+
+namespace mixkvq {
+
+constexpr int kD = 128;                 // head dimension
+constexpr int kStateBytes = 1152;       // acc fp64[128] | cnt u32 | extras_used16 u32 | zeros
+constexpr int kPartialFloats = 8 * 130; // per (CTA, stream) split partial: 8 heads x {m, l, o[128]}
+constexpr int kMaxCtas = 148 * 8;       // upper bound on the attention grid (sizes the workspace)
+
+enum Tier : uint8_t { kU2 = 0, kU4 = 1, kBF16 = 2 };
+
+// Geometry + pointers of one layer, passed by value to every kernel.
+struct LayerView {
+  // geometry
+  int B, Hq, Hkv, g;          // batch, query heads, KV heads, GQA group size
+  int R, G, U, NG, VG;        // residual length, group size, units/block, key groups/block, value groups/token
+  int max_blocks;
+  int n_blocks, r;            // current fill (same for all streams)
+  uint32_t base_bytes, unit_bytes;
+  uint64_t extras_budget;     // bytes per stream
+  // method parameters
+  int score_bits, importance_mode;
+  float tau_bf16, tau_u4;
+  // per-stream arrays (base pointer + stride in bytes)
+  char* state;  uint64_t state_stride;
+  char* table;  uint64_t table_stride;
+  char* resk;   uint64_t resk_stride;
+  char* resv;   uint64_t resv_stride;
+  char* base;   uint64_t base_stride;
+  char* extras; uint64_t extras_stride;
+  uint32_t* status;           // sticky device status word
+};
+
+__host__ __device__ inline uint32_t extras_header_bytes(int n16, int n4) {
+  int n16p = (n16 + 1) >> 1, n4p = ((n4 + 1) >> 1) << 1;
+  return 16u * ((2 * n16p + n4p + 15) >> 4);
+}
+__host__ __device__ inline uint32_t extras_unit_bytes(int n16, int n4) {
+  int n16p = (n16 + 1) >> 1, n4p = ((n4 + 1) >> 1) << 1;
+  return 128u * n16p + 8u * n4p;
+}
+
+// ---- bf16 bit helpers (no rounding involved)
+__device__ inline float bf16_bits_to_float(uint32_t u16) { return __uint_as_float(u16 << 16); }
+__device__ inline uint32_t float_to_bf16_bits_exact(float f) { return __float_as_uint(f) >> 16; }
+
+// Scale of Eq. 2 as stored: fp32 (max - min) / levels, rounded up to bf16 (returned as float).
+__device__ inline float stored_scale(float mx, float mn, float levels) {
+  float q = __fdiv_rn(__fsub_rn(mx, mn), levels);
+  uint32_t b = __float_as_uint(q);
+  if (b & 0xFFFFu) b = (b + 0x10000u) & 0xFFFF0000u;
+  return __uint_as_float(b);
+}
+
+// Code of Eq. 2: round-half-even of the IEEE fp32 quotient (x - z) / s, clamped; 0 when s == 0.
+__device__ inline int quant_code(float x, float z, float s, int max_code) {
+  if (s == 0.0f) return 0;
+  float y = __fdiv_rn(__fsub_rn(x, z), s);
+  int c = __float2int_rn(y);
+  return min(max(c, 0), max_code);
+}
+
+// Section 4.2: A_d = (acc / cnt) * (range / (2^B - 1)) in fp64; tier by the two thresholds.
+__device__ inline uint8_t salience_tier(double acc, uint32_t cnt, float mx, float mn, int score_bits,
+                                        float tau_bf16, float tau_u4, double* a_out) {
+  double range = (double)mx - (double)mn;
+  double S = __ddiv_rn(range, (double)((1 << score_bits) - 1));
+  double I = __ddiv_rn(acc, (double)cnt);
+  double A = __dmul_rn(I, S);
+  if (a_out) *a_out = A;
+  if (A > (double)tau_bf16) return kBF16;
+  if (A > (double)tau_u4) return kU4;
+  return kU2;
+}
+
+// ---- layout: positions inside a unit (see the layout description in the repository's design notes)
+// K low-plane code of (token jj in unit, channel d): 32-bit word index inside the unit's K codes, bit offset.
+__host__ __device__ inline void k_code_pos(int jj, int d, int* word, int* bit) {
+  int mt = jj >> 4, row = jj & 15, r = row & 7, rh = row >> 3;
+  int kt = d >> 4, col = d & 15, ch = col >> 3, t = (col & 7) >> 1, e = col & 1;
+  *word = mt * 128 + (4 * r + t) * 4 + (2 * ch + rh);
+  *bit = 16 * e + 2 * kt;
+}
+// V code of (token jj in unit, channel c).
+__host__ __device__ inline void v_code_pos(int jj, int c, int* word, int* bit) {
+  int ct = c >> 4, row = c & 15, r = row & 7, rh = row >> 3;
+  int ks = jj >> 4, col = jj & 15, ch = col >> 3, t = (col & 7) >> 1, e = col & 1;
+  *word = (ct >> 2) * 128 + (4 * r + t) * 4 + (ct & 3);
+  *bit = 16 * e + 2 * (4 * rh + 2 * ks + ch);
+}
+// UINT4 high-plane code of (token jj, half e) inside a channel pair's four words.
+__host__ __device__ inline void hi_plane_pos(int jj, int e, int* word, int* bit) {
+  int mt = jj >> 4, row = jj & 15, r = row & 7, rh = row >> 3;
+  *word = r & 3;
+  *bit = 16 * e + 8 * (r >> 2) + 2 * (2 * mt + rh);
+}
+
+// Even split of `total` work units over `parts`: [begin(i), begin(i+1)).
+__host__ __device__ inline long long split_begin(long long total, int parts, int i) {
+  return (total * (long long)i) / parts;
+}
+
+}  // namespace mixkvq
+
+// launchers implemented in the .cu files (host side, all asynchronous on `stream`)
+namespace mixkvq {
+cudaError_t launch_append(const LayerView& lv, const void* k, const void* v, const void* q, int n_tokens, int t0,
+                          int m, cudaStream_t stream);
+cudaError_t launch_flush(const LayerView& lv, cudaStream_t stream);
+cudaError_t launch_select_window(const LayerView& lv, uint8_t* tiers, double* salience, cudaStream_t stream);
+cudaError_t launch_select_raw(const void* q, const void* k, int B, int Hq, int Hkv, int lq, int lk, int score_bits,
+                              float tau_bf16, float tau_u4, uint8_t* tiers, double* salience, cudaStream_t stream);
+// decode attention: writes split partials to `ws`, then the combine kernel writes `out`; returns launches made
+cudaError_t launch_attention_simt(const LayerView& lv, const void* q, float* out, float scale, float* ws,
+                                  int n_sms, cudaStream_t stream, int* launches);
+cudaError_t launch_attention_mma(const LayerView& lv, const void* q, float* out, float scale, float* ws,
+                                 int n_sms, cudaStream_t stream, int* launches);
+cudaError_t attention_mma_setup();
+}  // namespace mixkvq

@@ -1,0 +1,221 @@
+"""GPU parity: the CUDA path through the C ABI against the CPU oracle on the same seeded inputs.
+
+Codes, packed bytes, selected channels and accumulator state must be bit-exact; attention outputs
+within 2e-3 max-abs (the stated tolerance for fp32 outputs on bf16 inputs)."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+import gpu_util as U
+from oracle import mixkvq_oracle as O
+from paper_2512_19206_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+ATTN_TOL = 2e-3
+
+
+@pytest.fixture(scope="module")
+def binding():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2512_19206_b200 import build
+    build.build()
+    from paper_2512_19206_b200 import binding as b
+    b.lib()
+    return b
+
+
+def small(name="qwen7b", **kw):
+    base = dict(n_layers=1, batch=2, tokens=300)
+    base.update(kw)
+    return W.small(W.CONFIGS[name], **base)
+
+
+# ------------------------------------------------------------------------------------------ selection
+@pytest.mark.parametrize("bits,preset", [(2, W.P27), (4, W.P4BASE)])
+def test_select_channels_raw_bit_exact(binding, bits, preset):
+    w = small(tokens=128, **{k: v for k, v in preset.items()})
+    k, v, q = W.tokens(w, 0, 0, 128)
+    tiers, sal = binding.select_channels_raw(q.cuda(), k.cuda(), bits, w.tau_bf16, w.tau_u4)
+    for b in range(w.batch):
+        for hk in range(w.n_kv_heads):
+            acc, cnt = O.importance_from_queries(U.f32(q[b, hk * w.g:(hk + 1) * w.g]))
+            _, _, A = O.salience(acc, cnt, U.f32(k[b, hk]), bits)
+            assert np.array_equal(sal[b, hk].cpu().numpy(), A)                       # fp64, bit for bit
+            assert np.array_equal(tiers[b, hk].cpu().numpy(), O.assign_tiers(A, w.tau_bf16, w.tau_u4))
+    assert int((tiers == 2).sum()) >= 4 * w.batch * w.n_kv_heads - 4
+
+
+def test_select_channels_of_current_window(binding):
+    w = small(tokens=128 + 57, **W.P27)
+    k, v, q = W.tokens(w, 0, 0, w.tokens)
+    cache = U.make_cache(binding, w)
+    cache.quantize_append(0, k.cuda(), v.cuda(), q.cuda())
+    tiers, sal = cache.select_channels(0)
+    orc = U.oracle_streams(w, 0, k, v, q)
+    for (b, hk), st in orc.items():
+        t, A = st.current_tiers()
+        assert st.r == 57
+        assert np.array_equal(tiers[b, hk].cpu().numpy(), t)
+        assert np.array_equal(sal[b, hk].cpu().numpy(), A)
+
+
+# --------------------------------------------------------------------------------- quantize + pack bytes
+GEOMS = [(128, 32), (128, 128), (128, 64), (64, 32), (96, 32), (256, 64), (32, 32)]
+
+
+@pytest.mark.parametrize("R,G", GEOMS)
+@pytest.mark.parametrize("preset", ["P24", "P27", "P4BASE"])
+def test_packed_cache_is_byte_exact(binding, R, G, preset):
+    w = small(tokens=2 * R + 41, residual_len=R, group_size=G, **getattr(W, preset))
+    k, v, q = W.tokens(w, 0, 0, w.tokens)
+    cache = U.make_cache(binding, w)
+    cache.quantize_append(0, k.cuda(), v.cuda(), q.cuda())
+    assert cache.status() == 0
+    orc = U.oracle_streams(w, 0, k, v, q)
+    U.compare_regions(cache, 0, w, orc)
+    d = cache.describe(0)
+    assert (d.n_blocks, d.residual_tokens) == (2, 41)
+    if preset == "P27":
+        assert any((b.tiers == O.TIER_U4).any() for st in orc.values() for b in st.blocks)
+    if preset == "P4BASE":
+        assert all(not (b.tiers == O.TIER_U2).any() for st in orc.values() for b in st.blocks)
+
+
+def test_tiny_config_full_parity(binding):
+    # configuration 1: 1 layer, batch 1, 1 KV head, 1 query head, 1024 cached tokens, then one decode step
+    w = W.CONFIGS["tiny"]
+    w = dataclasses.replace(w, **W.P27)
+    k, v, q = W.tokens(w, 0, 0, 1025)
+    cache = U.make_cache(binding, w)
+    cache.quantize_append(0, k[:, :, :1024].cuda(), v[:, :, :1024].cuda(), q[:, :, :1024].cuda())
+    orc = U.oracle_streams(w, 0, k[:, :, :1024], v[:, :, :1024], q[:, :, :1024])
+    U.compare_regions(cache, 0, w, orc)
+    assert cache.describe(0).n_blocks == 7 and cache.describe(0).residual_tokens == 128
+    # the decode step: append (triggers the flush of block 8), then attention
+    cache.quantize_append(0, k[:, :, 1024:].cuda().contiguous(), v[:, :, 1024:].cuda().contiguous(),
+                          q[:, :, 1024:].cuda().contiguous())
+    st = orc[(0, 0)]
+    st.append(U.f32(k[0, 0, 1024]), U.f32(v[0, 0, 1024]), U.f32(q[0, :, 1024]))
+    U.compare_regions(cache, 0, w, orc)
+    qd = q[:, :, 1024].contiguous()
+    ref = U.oracle_attention(w, orc, qd)
+    for kind in (0, 1):
+        cache.set_attention_kernel(kind)
+        out = cache.decode_attention(0, qd.cuda(), W.softmax_scale())
+        assert U.max_abs_err(w, out, ref) <= ATTN_TOL, kind
+    assert cache.status() == 0
+
+
+def test_streamed_appends_equal_bulk(binding):
+    w = small(batch=1, tokens=128 + 70, **W.P27)
+    k, v, q = W.tokens(w, 0, 0, w.tokens)
+    kc, vc, qc = k.cuda(), v.cuda(), q.cuda()
+    bulk = U.make_cache(binding, w)
+    bulk.quantize_append(0, kc, vc, qc)
+    one = U.make_cache(binding, w)
+    for t in range(w.tokens):
+        one.quantize_append(0, kc[:, :, t:t + 1].contiguous(), vc[:, :, t:t + 1].contiguous(),
+                            qc[:, :, t:t + 1].contiguous())
+    # in two ragged pieces as well
+    two = U.make_cache(binding, w)
+    two.quantize_append(0, kc[:, :, :93].contiguous(), vc[:, :, :93].contiguous(), qc[:, :, :93].contiguous())
+    two.quantize_append(0, kc[:, :, 93:].contiguous(), vc[:, :, 93:].contiguous(), qc[:, :, 93:].contiguous())
+    for s in range(w.n_kv_heads):
+        a, b, c = bulk.stream_regions(0, s), one.stream_regions(0, s), two.stream_regions(0, s)
+        r = bulk.describe(0).residual_tokens
+        for key in ("table", "base", "extras", "state", "resK"):
+            assert a[key] == b[key] == c[key], key
+        av = np.frombuffer(a["resV_full"], "<u2").reshape(128, -1)[:, :r]
+        assert np.array_equal(av, np.frombuffer(b["resV_full"], "<u2").reshape(128, -1)[:, :r])
+    U.compare_regions(bulk, 0, w, U.oracle_streams(w, 0, k, v, q))
+
+
+def test_cumulative_importance_mode(binding):
+    w = small(batch=1, tokens=2 * 128 + 9, **W.P27)
+    k, v, q = W.tokens(w, 0, 0, w.tokens)
+    cache = U.make_cache(binding, w, importance_mode=1)
+    cache.quantize_append(0, k.cuda(), v.cuda(), q.cuda())
+    U.compare_regions(cache, 0, w, U.oracle_streams(w, 0, k, v, q, importance_mode=1))
+
+
+# ------------------------------------------------------------------------------------------- attention
+@pytest.mark.parametrize("kind", [0, 1])
+@pytest.mark.parametrize("name,tokens,preset", [
+    ("qwen7b", 1, "P24"), ("qwen7b", 31, "P24"), ("qwen7b", 128, "P24"), ("qwen7b", 129, "P24"),
+    ("qwen7b", 1153, "P27"), ("llama8b", 700, "P27"), ("llama8b", 700, "P4BASE"), ("qwen32b", 1000, "P24"),
+    ("tiny", 2500, "P27"),
+])
+def test_attention_matches_oracle(binding, kind, name, tokens, preset):
+    w = small(name, batch=2 if name != "tiny" else 1, tokens=tokens, **getattr(W, preset))
+    k, v, q = W.tokens(w, 0, 0, tokens)
+    cache = U.make_cache(binding, w)
+    cache.quantize_append(0, k.cuda(), v.cuda(), q.cuda())
+    cache.set_attention_kernel(kind)
+    orc = U.oracle_streams(w, 0, k, v, q)
+    for step in range(2):
+        qd = W.decode_query(w, 0, step)
+        out = cache.decode_attention(0, qd.cuda(), W.softmax_scale())
+        err = U.max_abs_err(w, out, U.oracle_attention(w, orc, qd))
+        assert err <= ATTN_TOL, (err, step)
+    assert cache.status() == 0
+
+
+@pytest.mark.parametrize("kind", [0, 1])
+@pytest.mark.parametrize("R,G", [(128, 128), (64, 32), (256, 64), (32, 32), (96, 32)])
+def test_attention_other_geometries(binding, kind, R, G):
+    w = small("llama8b", batch=1, tokens=3 * R + 17, residual_len=R, group_size=G, **W.P27)
+    k, v, q = W.tokens(w, 0, 0, w.tokens)
+    cache = U.make_cache(binding, w)
+    cache.quantize_append(0, k.cuda(), v.cuda(), q.cuda())
+    cache.set_attention_kernel(kind)
+    orc = U.oracle_streams(w, 0, k, v, q)
+    qd = W.decode_query(w, 0, 0)
+    out = cache.decode_attention(0, qd.cuda(), W.softmax_scale())
+    assert U.max_abs_err(w, out, U.oracle_attention(w, orc, qd)) <= ATTN_TOL
+
+
+def test_layers_are_independent(binding):
+    w = small(n_layers=3, batch=1, tokens=200, **W.P27)
+    cache = U.make_cache(binding, w)
+    data = [W.tokens(w, l, 0, 150 + 20 * l) for l in range(3)]
+    for l in (2, 0, 1):
+        k, v, q = data[l]
+        cache.quantize_append(l, k.cuda(), v.cuda(), q.cuda())
+    for l in range(3):
+        k, v, q = data[l]
+        orc = U.oracle_streams(w, l, k, v, q)
+        U.compare_regions(cache, l, w, orc)
+        qd = W.decode_query(w, l, 0)
+        out = cache.decode_attention(l, qd.cuda(), W.softmax_scale())
+        assert U.max_abs_err(w, out, U.oracle_attention(w, orc, qd)) <= ATTN_TOL
+
+
+# ------------------------------------------------------------------------------------- errors and status
+def test_capacity_and_empty_errors(binding):
+    w = small(batch=1, tokens=100)
+    cache = U.make_cache(binding, w, max_tokens=128)
+    qd = W.decode_query(w, 0, 0).cuda()
+    with pytest.raises(binding.MixKVQError) as e:
+        cache.decode_attention(0, qd, 1.0)
+    assert e.value.code == -7
+    k, v, q = W.tokens(w, 0, 0, 129)
+    with pytest.raises(binding.MixKVQError) as e:
+        cache.quantize_append(0, k.cuda(), v.cuda(), q.cuda())
+    assert e.value.code == -5
+    assert cache.describe(0).residual_tokens == 0
+    with pytest.raises(binding.MixKVQError) as e:         # misaligned device pointer
+        cache.quantize_append(0, k.cuda().view(-1)[1:1 + 128 * 4].view(1, 4, 1, 128), v.cuda()[:, :, :1].contiguous(),
+                              q.cuda()[:, :, :1].contiguous())
+    assert e.value.code == -3
+
+
+def test_extras_arena_exhaustion_sets_status(binding):
+    w = small(batch=1, tokens=3 * 128 + 1, **W.P27)
+    k, v, q = W.tokens(w, 0, 0, w.tokens)
+    cache = U.make_cache(binding, w, extras_budget_bytes=2048)     # room for about one block's promoted channels
+    cache.quantize_append(0, k.cuda(), v.cuda(), q.cuda())
+    assert cache.status() & binding.DEV_EXTRAS_FULL
+    cache.reset()
+    assert cache.status() == 0 and cache.describe(0).n_blocks == 0

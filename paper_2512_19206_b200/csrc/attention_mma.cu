@@ -1,9 +1,679 @@
-// placeholder until the tensor-core kernel lands: routes to the plain-ALU kernel
+// Fused split-K GQA decode attention over the mixed-precision cache (Eq. 1 with Eq. 3 applied on the fly).
+//
+// Work unit = 32 tokens of one stream.  All units of all streams are split evenly over the CTAs; inside a
+// CTA every warp owns a contiguous run of units and is an independent split: it stages its units into its
+// own shared-memory ring with 1-D bulk (TMA) copies signalled on mbarriers, expands the 2-bit codes into
+// tensor-core A fragments with one logic op (plus one fp16 FMA for keys) per pair of codes, and runs
+// q.K^T, online softmax and P.V on mma.sync m16n8k16 tiles with the g query heads of the KV head as the
+// N dimension.  The packed layout stores the codes in A-fragment order, so a lane's 16-byte shared-memory
+// load is exactly its registers; nothing dequantized is ever written back to shared memory.
+//
+//   keys    A = c*s (exact in fp16: 2-bit code x 8-bit scale), B = q (exact), zero-points enter through
+//           one extra tile per key group (A = z broadcast over rows) that initializes the accumulators.
+//   values  A = raw codes read as fp16 subnormals (c * 4^i * 2^-24), B = P * s_v * 4^-i * 2^4, zero-points
+//           and the softmax denominator through one extra tile (rows = value groups and a row of ones).
+//   promoted (BF16) key channels and the UINT4 high plane come from the block's extras with a gathered q.
+//   residual (unquantized) tokens use bf16 tiles straight from global memory.
 #include "common.cuh"
+
 namespace mixkvq {
-cudaError_t attention_mma_setup() { return cudaSuccess; }
+
+cudaError_t launch_combine(const float* ws, float* out, int g, int Hkv, int Hq, int mode, int n,
+                           long long units_per_stream, int S, cudaStream_t stream);
+
+namespace {
+
+constexpr int kWarps = 4;
+constexpr int kStages = 4;
+constexpr int kStageBytes = 3072;            // unit (<= 2560 B) followed by one key-meta group (512 B)
+constexpr int kKeyMetaOff = 2560;
+constexpr int kPrepBytes = 1280;             // kprep 512 | zprep 256 | svp 256 | zvp 256
+constexpr int kSharedTail = 128 + 2048 + 2048 + 128 + 128 + 4096;
+constexpr int kSmemBytes = kWarps * (kStages * kStageBytes + kPrepBytes) + kSharedTail;
+constexpr int kCtasPerSm = 3;
+constexpr uint32_t kSpinLimit = 1u << 22;    // bounded wait on a staged copy
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Waits for a phase with an iteration limit; false if it gave up.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < kSpinLimit; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+
+__device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                        uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
+  uint32_t y;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t hfma2_u(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t d;
+  asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+__device__ __forceinline__ uint32_t hmul2_u(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
+  __half2 h = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+__device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+// two bf16 in one word -> two fp16 in one word (exact inside the fp16 range)
+__device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t w) { return pack_half2(bf_lo(w), bf_hi(w)); }
+
+// Bit position (inside each 16-bit half, after the shift below) of k-tile kt's 2-bit field.
+__device__ __forceinline__ constexpr int key_pos(int kt) { return (0x86486464u >> (4 * kt)) & 0xF; }
+// k-tiles 0,1 are read from (w << 4), 2..4 from w, 5..7 from (w >> 6)
+__device__ __forceinline__ uint32_t key_shift(uint32_t w, int kt) { return kt < 2 ? (w << 4) : (kt < 5 ? w : (w >> 6)); }
+
+template <int G>
+__global__ void __launch_bounds__(kWarps * 32, kCtasPerSm)
+attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float scale_log2e, float* __restrict__ ws) {
+  constexpr int VG = kD / G;              // value groups per token
+  constexpr int TPG = 8 / VG;             // 16-channel tiles per value group
+  extern __shared__ __align__(128) unsigned char smem[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, r = lane >> 2, t = lane & 3;
+
+  unsigned char* ring = smem + warp * (kStages * kStageBytes);
+  unsigned char* prep = smem + kWarps * kStages * kStageBytes + warp * kPrepBytes;
+  uint32_t* kprep = reinterpret_cast<uint32_t*>(prep);          // [8 kt][4 t]{m2 ch0, o2 ch0, m2 ch1, o2 ch1}
+  uint32_t* zprep = reinterpret_cast<uint32_t*>(prep + 512);    // [8 kt][4 t][2 ch] half2 z / mult
+  uint32_t* svp = reinterpret_cast<uint32_t*>(prep + 768);      // [2 ks][2 ch][4 t][4 vg] half2 s_v'
+  uint32_t* zvp = reinterpret_cast<uint32_t*>(prep + 1024);     // [2 ks][2 ch][4 vg][4 t] half2 z_v
+  unsigned char* tail = smem + kWarps * (kStages * kStageBytes + kPrepBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tail);           // [kWarps][kStages]
+  uint16_t* qb16 = reinterpret_cast<uint16_t*>(tail + 128);     // [8][128] q, bf16 bits (0 for heads >= g)
+  __half* qf16 = reinterpret_cast<__half*>(tail + 128 + 2048);  // [8][128] q, fp16
+  float* mS = reinterpret_cast<float*>(tail + 128 + 4096);      // [4][8]
+  float* lS = mS + 32;                                          // [4][8]
+  float* oS = lS + 32;                                          // [8][128]
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kWarps * kStages; ++i) mbar_init(smem_u32(&bars[i]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  const int S = lv.B * lv.Hkv, U = lv.U, g = lv.g;
+  const int packed_units = lv.n_blocks * U;
+  const int Us = packed_units + (lv.r + 31) / 32;
+  const long long total = (long long)Us * S;
+  const long long cb = split_begin(total, gridDim.x, blockIdx.x), ce = split_begin(total, gridDim.x, blockIdx.x + 1);
+
+  uint32_t ring_count = 0;        // packed units this warp has consumed so far (ring position)
+  uint32_t ring_issued = 0;       // packed units this warp has issued so far
+  bool gave_up = false;
+
+  for (long long seg = cb; seg < ce;) {
+    const int s = (int)(seg / Us);
+    const int ub = (int)(seg - (long long)s * Us);
+    const int ue = (int)min((long long)Us, ce - (long long)s * Us);
+    seg += ue - ub;
+    const int wb = ub + (int)split_begin(ue - ub, kWarps, warp), we = ub + (int)split_begin(ue - ub, kWarps, warp + 1);
+
+    // ---- query of this stream: bf16 and fp16 tables for the gathered paths
+    {
+      const int b = s / lv.Hkv, hk = s % lv.Hkv;
+      __syncthreads();
+      for (int i = threadIdx.x; i < 8 * kD; i += kWarps * 32) {
+        const int h = i >> 7, d = i & 127;
+        const __nv_bfloat16 v = (h < g) ? q[((size_t)b * lv.Hq + hk * g + h) * kD + d] : __float2bfloat16(0.f);
+        qb16[i] = *reinterpret_cast<const uint16_t*>(&v);
+        qf16[i] = __float2half_rn(__bfloat162float(v));
+      }
+      __syncthreads();
+    }
+    // B fragments of q for the base key tiles: head r, channels 16kt + {2t, 2t+1} and {2t+8, 2t+9}, times mult(kt)
+    uint32_t bq[8][2];
+#pragma unroll
+    for (int kt = 0; kt < 8; ++kt) {
+      const float mult = (float)(1 << (8 - key_pos(kt)));
+#pragma unroll
+      for (int hch = 0; hch < 2; ++hch) {
+        const uint32_t w = *reinterpret_cast<const uint32_t*>(&qb16[r * kD + 16 * kt + 8 * hch + 2 * t]);
+        bq[kt][hch] = pack_half2(bf_lo(w) * mult, bf_hi(w) * mult);
+      }
+    }
+
+    const char* base = lv.base + (size_t)s * lv.base_stride;
+    const char* extras = lv.extras + (size_t)s * lv.extras_stride;
+    const uint2* table = reinterpret_cast<const uint2*>(lv.table + (size_t)s * lv.table_stride);
+    const uint16_t* resk = reinterpret_cast<const uint16_t*>(lv.resk + (size_t)s * lv.resk_stride);
+    const uint16_t* resv = reinterpret_cast<const uint16_t*>(lv.resv + (size_t)s * lv.resv_stride);
+
+    float O[8][4];       // O^T tiles: [channel tile] x (channels r, r+8) x (heads 2t, 2t+1); packed part scaled 2^-20
+    float Zc[4] = {0.f, 0.f, 0.f, 0.f};   // rows 0..VG-1: sum p * z_v per value group; row 4: sum p
+    float zc[4] = {0.f, 0.f, 0.f, 0.f};   // key zero-point term of the current key group
+    float m0 = -INFINITY, m1 = -INFINITY; // running max (log2 domain) of heads 2t, 2t+1
+#pragma unroll
+    for (int ct = 0; ct < 8; ++ct)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) O[ct][i] = 0.f;
+    bool o_true_scale = false;
+
+    const int n_pack = max(0, min(we, packed_units) - wb);
+    int issued = 0;
+    auto issue = [&](int x, bool first) {
+      // lane 0 only: stage unit x of this stream
+      const int bi = x / U, u = x - bi * U;
+      const char* blk = base + (size_t)bi * lv.base_bytes;
+      const uint32_t stage = ring_issued % kStages;
+      const uint32_t bar = smem_u32(&bars[warp * kStages + stage]);
+      const uint32_t dst = smem_u32(ring + stage * kStageBytes);
+      const bool meta = first || ((u * 32) % G == 0);
+      mbar_expect_tx(bar, lv.unit_bytes + (meta ? 512u : 0u));
+      bulk_g2s(dst, blk + lv.NG * 512 + (size_t)u * lv.unit_bytes, lv.unit_bytes, bar);
+      if (meta) bulk_g2s(dst + kKeyMetaOff, blk + ((u * 32) / G) * 512, 512u, bar);
+    };
+    for (; !gave_up && issued < min(n_pack, kStages); ++issued) {
+      if (lane == 0) issue(wb + issued, issued == 0);
+      ++ring_issued;
+    }
+
+    int cur_bi = -1, pf_bi = -1;
+    uint2 entry = make_uint2(0, 0), pf_entry = make_uint2(0, 0);
+    int n16 = 0, n4 = 0, n16p = 0;
+    const char* ex = nullptr;
+    uint32_t ex_hdr = 0, ex_unit = 0;
+
+    for (int i = 0; i < n_pack && !gave_up; ++i) {
+      const int x = wb + i;
+      const int bi = x / U, u = x - bi * U;
+      if (bi != cur_bi) {
+        entry = (pf_bi == bi) ? pf_entry : table[bi];
+        cur_bi = bi;
+        pf_bi = bi + 1;
+        if (pf_bi < lv.n_blocks) pf_entry = table[pf_bi];
+        n16 = entry.y & 0xFF;
+        n4 = (entry.y >> 8) & 0xFF;
+        n16p = (n16 + 1) >> 1;
+        ex = extras + (size_t)entry.x * 16;
+        ex_hdr = extras_header_bytes(n16, n4);
+        ex_unit = extras_unit_bytes(n16, n4);
+      }
+      const uint32_t stage = ring_count % kStages, parity = (ring_count / kStages) & 1;
+      if (!mbar_wait_bounded(smem_u32(&bars[warp * kStages + stage]), parity)) {
+        gave_up = true;
+        break;
+      }
+      ++ring_count;
+      const unsigned char* st = ring + stage * kStageBytes;
+      const bool has_meta = (i == 0) || ((u * 32) % G == 0);
+
+      // ---- key-group preparation: fp16 scale pairs in fragment order, zero-point tile
+      if (has_meta) {
+        const uint4 mz = reinterpret_cast<const uint4*>(st + kKeyMetaOff)[lane];   // channels 4*lane .. 4*lane+3
+        const int kt = lane >> 2, ch = (lane & 3) >> 1, t0 = 2 * (lane & 1);
+        const float zs = 1.0f / (float)(1 << (8 - key_pos(kt)));
+        const uint32_t ma = pack_half2(bf_lo(mz.x), bf_lo(mz.y)), mb = pack_half2(bf_lo(mz.z), bf_lo(mz.w));
+        const uint32_t neg4 = 0xC400C400u;   // half2(-4, -4)
+        __syncwarp();
+        *reinterpret_cast<uint2*>(&kprep[(kt * 4 + t0) * 4 + ch * 2]) = make_uint2(ma, hmul2_u(ma, neg4));
+        *reinterpret_cast<uint2*>(&kprep[(kt * 4 + t0 + 1) * 4 + ch * 2]) = make_uint2(mb, hmul2_u(mb, neg4));
+        zprep[(kt * 4 + t0) * 2 + ch] = pack_half2(bf_hi(mz.x) * zs, bf_hi(mz.y) * zs);
+        zprep[(kt * 4 + t0 + 1) * 2 + ch] = pack_half2(bf_hi(mz.z) * zs, bf_hi(mz.w) * zs);
+        __syncwarp();
+        zc[0] = zc[1] = zc[2] = zc[3] = 0.f;
+#pragma unroll
+        for (int kt2 = 0; kt2 < 8; ++kt2) {
+          const uint2 zz = *reinterpret_cast<const uint2*>(&zprep[(kt2 * 4 + t) * 2]);
+          mma_f16(zc, zz.x, zz.x, zz.y, zz.y, bq[kt2][0], bq[kt2][1]);
+        }
+      }
+
+      // ---- extras of this unit: issue the global loads early
+      const char* exu = ex + ex_hdr + (size_t)u * ex_unit;
+      uint32_t xa[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};   // BF16 pairs, first 16 promoted channels
+      uint32_t xid0 = 0xFFFFFFFFu, xid1 = 0xFFFFFFFFu;
+      if (n16 > 0) {
+        const uint32_t* xw = reinterpret_cast<const uint32_t*>(exu);
+        if (t < n16p) {
+          xid0 = *reinterpret_cast<const uint16_t*>(ex + 2 * t);
+#pragma unroll
+          for (int mt = 0; mt < 2; ++mt) {
+            xa[mt][0] = xw[t * 32 + mt * 16 + r];
+            xa[mt][1] = xw[t * 32 + mt * 16 + 8 + r];
+          }
+        }
+        if (t + 4 < n16p) {
+          xid1 = *reinterpret_cast<const uint16_t*>(ex + 2 * (t + 4));
+#pragma unroll
+          for (int mt = 0; mt < 2; ++mt) {
+            xa[mt][2] = xw[(t + 4) * 32 + mt * 16 + r];
+            xa[mt][3] = xw[(t + 4) * 32 + mt * 16 + 8 + r];
+          }
+        }
+      }
+
+      // ---- q.K^T on the base (2-bit low plane) tiles
+      float Sx[2][4];
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) Sx[mt][j] = zc[j];
+      {
+        const uint4 kw0 = reinterpret_cast<const uint4*>(st)[lane];
+        const uint4 kw1 = reinterpret_cast<const uint4*>(st)[32 + lane];
+        const uint32_t kw[2][4] = {{kw0.x, kw0.y, kw0.z, kw0.w}, {kw1.x, kw1.y, kw1.z, kw1.w}};
+#pragma unroll
+        for (int kt = 0; kt < 8; ++kt) {
+          const uint4 kp = *reinterpret_cast<const uint4*>(&kprep[(kt * 4 + t) * 4]);
+          const uint32_t mask = 0x00030003u << key_pos(kt);
+#pragma unroll
+          for (int mt = 0; mt < 2; ++mt) {
+            uint32_t a[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const uint32_t code = (key_shift(kw[mt][j], kt) & mask) | 0x44004400u;     // 4 + c * 2^(pos-8)
+              a[j] = hfma2_u(code, j < 2 ? kp.x : kp.z, j < 2 ? kp.y : kp.w);            // c * s * 2^(pos-8)
+            }
+            mma_f16(Sx[mt], a[0], a[1], a[2], a[3], bq[kt][0], bq[kt][1]);
+          }
+        }
+      }
+      // ---- promoted channels (raw bf16 keys) with a gathered q
+      if (n16 > 0) {
+        for (int kk = 0; kk * 8 < n16p; ++kk) {
+          uint32_t a[2][4], id0, id1;
+          if (kk == 0) {
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+              for (int j = 0; j < 4; ++j) a[mt][j] = xa[mt][j];
+            id0 = xid0;
+            id1 = xid1;
+          } else {
+            const uint32_t* xw = reinterpret_cast<const uint32_t*>(exu);
+            const int p0 = 8 * kk + t, p1 = p0 + 4;
+            id0 = id1 = 0xFFFFFFFFu;
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt) a[mt][0] = a[mt][1] = a[mt][2] = a[mt][3] = 0;
+            if (p0 < n16p) {
+              id0 = *reinterpret_cast<const uint16_t*>(ex + 2 * p0);
+#pragma unroll
+              for (int mt = 0; mt < 2; ++mt) {
+                a[mt][0] = xw[p0 * 32 + mt * 16 + r];
+                a[mt][1] = xw[p0 * 32 + mt * 16 + 8 + r];
+              }
+            }
+            if (p1 < n16p) {
+              id1 = *reinterpret_cast<const uint16_t*>(ex + 2 * p1);
+#pragma unroll
+              for (int mt = 0; mt < 2; ++mt) {
+                a[mt][2] = xw[p1 * 32 + mt * 16 + r];
+                a[mt][3] = xw[p1 * 32 + mt * 16 + 8 + r];
+              }
+            }
+          }
+          auto gather_bf16 = [&](uint32_t ids) -> uint32_t {
+            const uint32_t c0 = ids & 0xFF, c1 = (ids >> 8) & 0xFF;
+            const uint32_t lo = (c0 < 128) ? qb16[r * kD + c0] : 0u, hi = (c1 < 128) ? qb16[r * kD + c1] : 0u;
+            return lo | (hi << 16);
+          };
+          const uint32_t b0 = gather_bf16(id0), b1 = gather_bf16(id1);
+#pragma unroll
+          for (int mt = 0; mt < 2; ++mt) mma_bf16(Sx[mt], a[mt][0], a[mt][1], a[mt][2], a[mt][3], b0, b1);
+        }
+      }
+      // ---- UINT4 high plane: c_hi * 4s, gathered q in fp16
+      if (n4 > 0) {
+        const int n4pairs = (n4 + 1) >> 1;
+        const uint32_t* hw = reinterpret_cast<const uint32_t*>(exu + 128 * n16p);
+        const unsigned char* ids4 = reinterpret_cast<const unsigned char*>(ex) + 2 * n16p;
+        const __half* kph = reinterpret_cast<const __half*>(kprep);
+        for (int kk = 0; kk * 8 < n4pairs; ++kk) {
+          uint32_t a[2][4], b[2];
+#pragma unroll
+          for (int hp = 0; hp < 2; ++hp) {
+            const int p = 8 * kk + 4 * hp + t;
+            uint32_t w = 0, sc = 0;
+            b[hp] = 0;
+            if (p < n4pairs) {
+              w = hw[p * 4 + (r & 3)] >> (8 * (r >> 2));
+              const uint32_t c0 = ids4[2 * p], c1 = ids4[2 * p + 1];
+              auto scale_of = [&](uint32_t c) -> __half {
+                // fp16 scale of channel c in kprep: [(kt*4 + t')*4 + ch*2] half2, element e
+                const int kt = c >> 4, col = c & 15;
+                return kph[(((kt * 4 + ((col & 7) >> 1)) * 4 + (col >> 3) * 2) << 1) + (col & 1)];
+              };
+              const __half zero = __float2half_rn(0.f);
+              const __half s0 = (c0 < 128) ? scale_of(c0) : zero, s1 = (c1 < 128) ? scale_of(c1) : zero;
+              const __half q0 = (c0 < 128) ? qf16[r * kD + c0] : zero, q1 = (c1 < 128) ? qf16[r * kD + c1] : zero;
+              __half2 s2 = __halves2half2(s0, s1), q2 = __halves2half2(q0, q1);
+              sc = *reinterpret_cast<uint32_t*>(&s2);
+              b[hp] = *reinterpret_cast<uint32_t*>(&q2);
+            }
+            const uint32_t m4 = hmul2_u(sc, 0x44004400u);          // 4s
+            const uint32_t o4 = hmul2_u(sc, 0xCC00CC00u);          // -16s
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+              for (int rh = 0; rh < 2; ++rh) {
+                const int f = 2 * mt + rh;
+                const uint32_t code = ((w << (8 - 2 * f)) & 0x03000300u) | 0x44004400u;   // 4 + c_hi
+                a[mt][2 * hp + rh] = hfma2_u(code, m4, o4);                                // c_hi * 4s
+              }
+          }
+#pragma unroll
+          for (int mt = 0; mt < 2; ++mt) mma_f16(Sx[mt], a[mt][0], a[mt][1], a[mt][2], a[mt][3], b[0], b[1]);
+        }
+      }
+
+      // ---- value-group preparation (lane = token)
+      {
+        const uint32_t* vmeta = reinterpret_cast<const uint32_t*>(st + 2048);
+        const int ks = lane >> 4, ch = (lane >> 3) & 1, tt = (lane & 7) >> 1, e = lane & 1;
+        const float up = (float)(1 << 4) / (float)(1 << (2 * (lane >> 3)));     // 2^(4 - 2*(2ks + ch))
+        __half* svh = reinterpret_cast<__half*>(svp);
+        __half* zvh = reinterpret_cast<__half*>(zvp);
+#pragma unroll
+        for (int vg = 0; vg < VG; ++vg) {
+          const uint32_t mz = vmeta[lane * VG + vg];
+          svh[((((ks * 2 + ch) * 4 + tt) * 4 + vg) << 1) + e] = __float2half_rn(bf_lo(mz) * up);
+          zvh[((((ks * 2 + ch) * 4 + vg) * 4 + tt) << 1) + e] = __float2half_rn(bf_hi(mz));
+        }
+      }
+
+      // ---- online softmax (log2 domain); heads 2t, 2t+1; tokens r, r+8 of each m-tile
+      float xs[2][4];
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) xs[mt][j] = Sx[mt][j] * scale_log2e;
+      float u0 = fmaxf(fmaxf(xs[0][0], xs[0][2]), fmaxf(xs[1][0], xs[1][2]));
+      float u1 = fmaxf(fmaxf(xs[0][1], xs[0][3]), fmaxf(xs[1][1], xs[1][3]));
+#pragma unroll
+      for (int off = 4; off < 32; off <<= 1) {
+        u0 = fmaxf(u0, __shfl_xor_sync(0xffffffffu, u0, off));
+        u1 = fmaxf(u1, __shfl_xor_sync(0xffffffffu, u1, off));
+      }
+      const float n0 = fmaxf(m0, u0), n1 = fmaxf(m1, u1);
+      if (__any_sync(0xffffffffu, (n0 > m0) || (n1 > m1))) {
+        const float a0 = exp2f(m0 - n0), a1 = exp2f(m1 - n1);    // exp2(-inf) = 0 on the first unit
+#pragma unroll
+        for (int ct = 0; ct < 8; ++ct) {
+          O[ct][0] *= a0; O[ct][1] *= a1; O[ct][2] *= a0; O[ct][3] *= a1;
+        }
+        Zc[0] *= a0; Zc[1] *= a1; Zc[2] *= a0; Zc[3] *= a1;
+        m0 = n0;
+        m1 = n1;
+      }
+      uint32_t Pt[2][2];    // P^T B fragments: [k-step][tokens 2t.. / 2t+8..], head r
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt) {
+        const uint32_t plo = pack_half2(exp2f(xs[mt][0] - m0), exp2f(xs[mt][1] - m1));   // token r
+        const uint32_t phi = pack_half2(exp2f(xs[mt][2] - m0), exp2f(xs[mt][3] - m1));   // token r + 8
+        Pt[mt][0] = movmatrix_trans(plo);
+        Pt[mt][1] = movmatrix_trans(phi);
+      }
+      __syncwarp();   // svp / zvp written above are read below
+
+      // ---- zero-point and denominator tile: rows 0..VG-1 = z_v of the group, row 4 = ones
+#pragma unroll
+      for (int ks = 0; ks < 2; ++ks) {
+        uint32_t a0 = 0, a2 = 0;
+        if (r < VG) {
+          a0 = zvp[((ks * 2 + 0) * 4 + r) * 4 + t];
+          a2 = zvp[((ks * 2 + 1) * 4 + r) * 4 + t];
+        } else if (r == 4) {
+          a0 = a2 = 0x3C003C00u;
+        }
+        mma_f16(Zc, a0, 0u, a2, 0u, Pt[ks][0], Pt[ks][1]);
+      }
+      // ---- P.V: codes as fp16 subnormals, scales folded into P
+      {
+        const uint4 vw0 = reinterpret_cast<const uint4*>(st + 1024)[lane];
+        const uint4 vw1 = reinterpret_cast<const uint4*>(st + 1024)[32 + lane];
+        const uint32_t vw[8] = {vw0.x, vw0.y, vw0.z, vw0.w, vw1.x, vw1.y, vw1.z, vw1.w};
+#pragma unroll
+        for (int vg = 0; vg < VG; ++vg) {
+          uint32_t Bp[2][2];
+#pragma unroll
+          for (int ks = 0; ks < 2; ++ks)
+#pragma unroll
+            for (int ch = 0; ch < 2; ++ch) Bp[ks][ch] = hmul2_u(Pt[ks][ch], svp[((ks * 2 + ch) * 4 + t) * 4 + vg]);
+#pragma unroll
+          for (int c = 0; c < TPG; ++c) {
+            const int ct = vg * TPG + c;
+            const uint32_t x0 = vw[ct], x1 = vw[ct] >> 8;
+#pragma unroll
+            for (int ks = 0; ks < 2; ++ks) {
+              const uint32_t mk0 = 0x00030003u << (4 * ks), mk1 = 0x00030003u << (4 * ks + 2);
+              mma_f16(O[ct], x0 & mk0, x1 & mk0, x0 & mk1, x1 & mk1, Bp[ks][0], Bp[ks][1]);
+            }
+          }
+        }
+      }
+
+      // ---- release the stage and refill it
+      __syncwarp();
+      if (issued < n_pack) {
+        if (lane == 0) issue(wb + issued, false);
+        ++ring_issued;
+        ++issued;
+      }
+    }
+    if (gave_up) {
+      // drain what is still in flight (bounded); later segments stage nothing but still join the CTA barriers
+      while (ring_count < ring_issued) {
+        const uint32_t stage = ring_count % kStages, parity = (ring_count / kStages) & 1;
+        mbar_wait_bounded(smem_u32(&bars[warp * kStages + stage]), parity);
+        ++ring_count;
+      }
+      if (lane == 0) atomicOr(lv.status, (uint32_t)MIXKVQ_DEV_COPY_TIMEOUT);
+    }
+
+    // ---- residual (unquantized) tokens of this warp's range: bf16 tiles from global memory
+    for (int x = max(wb, packed_units); x < we; ++x) {
+      if (!o_true_scale) {
+#pragma unroll
+        for (int ct = 0; ct < 8; ++ct)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) O[ct][j] *= 1048576.0f;
+        o_true_scale = true;
+      }
+      const int j0 = (x - packed_units) * 32, rt = lv.r;
+      float Sx[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+      for (int kt = 0; kt < 8; ++kt) {
+        const uint32_t b0 = *reinterpret_cast<const uint32_t*>(&qb16[r * kD + 16 * kt + 2 * t]);
+        const uint32_t b1 = *reinterpret_cast<const uint32_t*>(&qb16[r * kD + 16 * kt + 8 + 2 * t]);
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+          const int ta = j0 + mt * 16 + r, tb = ta + 8;
+          const uint32_t* ka = reinterpret_cast<const uint32_t*>(resk + (size_t)ta * kD + 16 * kt + 2 * t);
+          const uint32_t* kb = reinterpret_cast<const uint32_t*>(resk + (size_t)tb * kD + 16 * kt + 2 * t);
+          const uint32_t a0 = ta < rt ? ka[0] : 0u, a1 = tb < rt ? kb[0] : 0u;
+          const uint32_t a2 = ta < rt ? ka[4] : 0u, a3 = tb < rt ? kb[4] : 0u;
+          mma_bf16(Sx[mt], a0, a1, a2, a3, b0, b1);
+        }
+      }
+      float xl[2][4];
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt) {
+        const bool va = (j0 + mt * 16 + r) < rt, vb = (j0 + mt * 16 + 8 + r) < rt;
+        xl[mt][0] = va ? Sx[mt][0] * scale_log2e : -INFINITY;
+        xl[mt][1] = va ? Sx[mt][1] * scale_log2e : -INFINITY;
+        xl[mt][2] = vb ? Sx[mt][2] * scale_log2e : -INFINITY;
+        xl[mt][3] = vb ? Sx[mt][3] * scale_log2e : -INFINITY;
+      }
+      float u0 = fmaxf(fmaxf(xl[0][0], xl[0][2]), fmaxf(xl[1][0], xl[1][2]));
+      float u1 = fmaxf(fmaxf(xl[0][1], xl[0][3]), fmaxf(xl[1][1], xl[1][3]));
+#pragma unroll
+      for (int off = 4; off < 32; off <<= 1) {
+        u0 = fmaxf(u0, __shfl_xor_sync(0xffffffffu, u0, off));
+        u1 = fmaxf(u1, __shfl_xor_sync(0xffffffffu, u1, off));
+      }
+      const float n0 = fmaxf(m0, u0), n1 = fmaxf(m1, u1);
+      if (__any_sync(0xffffffffu, (n0 > m0) || (n1 > m1))) {
+        const float a0 = exp2f(m0 - n0), a1 = exp2f(m1 - n1);
+#pragma unroll
+        for (int ct = 0; ct < 8; ++ct) {
+          O[ct][0] *= a0; O[ct][1] *= a1; O[ct][2] *= a0; O[ct][3] *= a1;
+        }
+        Zc[0] *= a0; Zc[1] *= a1; Zc[2] *= a0; Zc[3] *= a1;
+        m0 = n0;
+        m1 = n1;
+      }
+      uint32_t Pt[2][2];
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt) {
+        Pt[mt][0] = movmatrix_trans(pack_half2(exp2f(xl[mt][0] - m0), exp2f(xl[mt][1] - m1)));
+        Pt[mt][1] = movmatrix_trans(pack_half2(exp2f(xl[mt][2] - m0), exp2f(xl[mt][3] - m1)));
+      }
+      const uint32_t ones = (r == 4) ? 0x3C003C00u : 0u;
+#pragma unroll
+      for (int ks = 0; ks < 2; ++ks) mma_f16(Zc, ones, 0u, ones, 0u, Pt[ks][0], Pt[ks][1]);
+#pragma unroll
+      for (int ct = 0; ct < 8; ++ct) {
+        const int c0 = 16 * ct + r, c1 = c0 + 8;
+#pragma unroll
+        for (int ks = 0; ks < 2; ++ks) {
+          const int ja = j0 + 16 * ks + 2 * t, jb = ja + 8;
+          auto load_pair = [&](int c, int j) -> uint32_t {
+            if (j >= rt) return 0u;
+            uint32_t w = *reinterpret_cast<const uint32_t*>(resv + (size_t)c * lv.R + j);
+            if (j + 1 >= rt) w &= 0xFFFFu;
+            return bf16x2_to_f16x2(w);
+          };
+          mma_f16(O[ct], load_pair(c0, ja), load_pair(c1, ja), load_pair(c0, jb), load_pair(c1, jb), Pt[ks][0],
+                  Pt[ks][1]);
+        }
+      }
+    }
+
+    // ---- finish this warp's split: true scale, zero-point terms, denominator
+    if (!o_true_scale) {
+#pragma unroll
+      for (int ct = 0; ct < 8; ++ct)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) O[ct][j] *= 1048576.0f;
+    }
+#pragma unroll
+    for (int ct = 0; ct < 8; ++ct) {
+      const int vg = ct / TPG;
+      const float z0 = __shfl_sync(0xffffffffu, Zc[0], vg * 4 + t), z1 = __shfl_sync(0xffffffffu, Zc[1], vg * 4 + t);
+      O[ct][0] += z0; O[ct][1] += z1; O[ct][2] += z0; O[ct][3] += z1;
+    }
+    const float l0 = __shfl_sync(0xffffffffu, Zc[0], 16 + t), l1 = __shfl_sync(0xffffffffu, Zc[1], 16 + t);
+
+    // ---- merge the warps of the CTA, write the partial of (CTA, stream)
+    if (r == 0) {
+      mS[warp * 8 + 2 * t] = m0;
+      mS[warp * 8 + 2 * t + 1] = m1;
+      lS[warp * 8 + 2 * t] = l0;
+      lS[warp * 8 + 2 * t + 1] = l1;
+    }
+    for (int i = threadIdx.x; i < 8 * kD; i += kWarps * 32) oS[i] = 0.f;
+    __syncthreads();
+    {
+      float M0 = -INFINITY, M1 = -INFINITY;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) {
+        M0 = fmaxf(M0, mS[w * 8 + 2 * t]);
+        M1 = fmaxf(M1, mS[w * 8 + 2 * t + 1]);
+      }
+      const float f0 = (m0 == -INFINITY) ? 0.f : exp2f(m0 - M0), f1 = (m1 == -INFINITY) ? 0.f : exp2f(m1 - M1);
+      if (m0 != -INFINITY || m1 != -INFINITY) {
+#pragma unroll
+        for (int ct = 0; ct < 8; ++ct) {
+          atomicAdd(&oS[(2 * t) * kD + 16 * ct + r], f0 * O[ct][0]);
+          atomicAdd(&oS[(2 * t + 1) * kD + 16 * ct + r], f1 * O[ct][1]);
+          atomicAdd(&oS[(2 * t) * kD + 16 * ct + 8 + r], f0 * O[ct][2]);
+          atomicAdd(&oS[(2 * t + 1) * kD + 16 * ct + 8 + r], f1 * O[ct][3]);
+        }
+      }
+    }
+    __syncthreads();
+    {
+      float* part = ws + (size_t)(blockIdx.x + s) * kPartialFloats;
+      for (int i = threadIdx.x; i < 8 * kD; i += kWarps * 32) part[(i >> 7) * 130 + 2 + (i & 127)] = oS[i];
+      if (threadIdx.x < 8) {
+        const int h = threadIdx.x;
+        float M = -INFINITY, L = 0.f;
+        for (int w = 0; w < kWarps; ++w) M = fmaxf(M, mS[w * 8 + h]);
+        for (int w = 0; w < kWarps; ++w) {
+          const float mw = mS[w * 8 + h];
+          L += (mw == -INFINITY) ? 0.f : exp2f(mw - M) * lS[w * 8 + h];
+        }
+        part[h * 130] = M;
+        part[h * 130 + 1] = L;
+      }
+    }
+  }
+}
+
+template <int G>
+cudaError_t launch_g(const LayerView& lv, const void* q, float scale, float* ws, int grid, cudaStream_t stream) {
+  attention_mma_kernel<G><<<grid, kWarps * 32, kSmemBytes, stream>>>(lv, static_cast<const __nv_bfloat16*>(q),
+                                                                     scale * 1.4426950408889634f, ws);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t attention_mma_setup() {
+  cudaError_t e;
+  e = cudaFuncSetAttribute(attention_mma_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(attention_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(attention_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+}
+
 cudaError_t launch_attention_mma(const LayerView& lv, const void* q, float* out, float scale, float* ws, int n_sms,
                                  cudaStream_t stream, int* launches) {
-  return launch_attention_simt(lv, q, out, scale, ws, n_sms, stream, launches);
+  const int S = lv.B * lv.Hkv;
+  const long long Us = (long long)lv.n_blocks * lv.U + (lv.r + 31) / 32;
+  const long long total = Us * S;
+  int grid = (int)min((long long)min(n_sms * kCtasPerSm, kMaxCtas), total);
+  if (grid < 1) grid = 1;
+  cudaError_t e;
+  if (lv.G == 32) e = launch_g<32>(lv, q, scale, ws, grid, stream);
+  else if (lv.G == 64) e = launch_g<64>(lv, q, scale, ws, grid, stream);
+  else e = launch_g<128>(lv, q, scale, ws, grid, stream);
+  if (e != cudaSuccess) return e;
+  e = launch_combine(ws, out, lv.g, lv.Hkv, lv.Hq, 1, grid, Us, S, stream);
+  *launches = 2;
+  return e;
 }
+
 }  // namespace mixkvq

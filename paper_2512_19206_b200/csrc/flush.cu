@@ -184,13 +184,9 @@ flush_kernel(LayerView lv) {
 static size_t flush_smem_bytes(int R) { return (size_t)R * 384 + 3 * 128 + 16; }
 
 cudaError_t launch_flush(const LayerView& lv, cudaStream_t stream) {
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(flush_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)flush_smem_bytes(256));
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  cudaError_t e = cudaFuncSetAttribute(flush_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)flush_smem_bytes(256));
+  if (e != cudaSuccess) return e;
   flush_kernel<<<lv.B * lv.Hkv, 256, flush_smem_bytes(lv.R), stream>>>(lv);
   return cudaGetLastError();
 }

@@ -129,7 +129,8 @@ int mixkvq_decode_attention(mixkvq_cache* cache, int layer, const void* q_dev, f
                             void* workspace_dev, size_t workspace_bytes, void* stream);
 
 /* Selects the decode-attention kernel: 0 = tensor-core kernel (default), 1 = plain-ALU kernel
- * (kept for comparison; same results within tolerance, much slower). */
+ * (kept for comparison; same results within tolerance, much slower), 2 = the tensor-core split kernel
+ * alone: the split partials stay in the workspace and out_dev is NOT written (for timing that kernel). */
 int mixkvq_set_attention_kernel(mixkvq_cache* cache, int kind);
 
 /* Synchronizes `stream`, then returns the sticky device status word (MIXKVQ_DEV_* bits). */

@@ -231,14 +231,15 @@ int mixkvq_decode_attention(mixkvq_cache* cache, int layer, const void* q_dev, f
     e = launch_attention_simt(lv, q_dev, out_dev, softmax_scale, static_cast<float*>(workspace_dev), cache->n_sms,
                               static_cast<cudaStream_t>(stream), &launches);
   else
-    e = launch_attention_mma(lv, q_dev, out_dev, softmax_scale, static_cast<float*>(workspace_dev), cache->n_sms,
-                             static_cast<cudaStream_t>(stream), &launches);
+    e = launch_attention_mma(lv, q_dev, cache->attn_kind == 2 ? nullptr : out_dev, softmax_scale,
+                             static_cast<float*>(workspace_dev), cache->n_sms, static_cast<cudaStream_t>(stream),
+                             &launches);
   cache->launches += launches;
   return e == cudaSuccess ? MIXKVQ_OK : MIXKVQ_E_CUDA;
 }
 
 int mixkvq_set_attention_kernel(mixkvq_cache* cache, int kind) {
-  if (!cache || (kind != 0 && kind != 1)) return MIXKVQ_E_INVALID_ARG;
+  if (!cache || kind < 0 || kind > 2) return MIXKVQ_E_INVALID_ARG;
   cache->attn_kind = kind;
   return MIXKVQ_OK;
 }

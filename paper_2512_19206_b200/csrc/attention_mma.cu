@@ -670,7 +670,8 @@ cudaError_t launch_attention_mma(const LayerView& lv, const void* q, float* out,
   if (lv.G == 32) e = launch_g<32>(lv, q, scale, ws, grid, stream);
   else if (lv.G == 64) e = launch_g<64>(lv, q, scale, ws, grid, stream);
   else e = launch_g<128>(lv, q, scale, ws, grid, stream);
-  if (e != cudaSuccess) return e;
+  *launches = 1;
+  if (e != cudaSuccess || out == nullptr) return e;     // out == nullptr: split kernel only (timing)
   e = launch_combine(ws, out, lv.g, lv.Hkv, lv.Hq, 1, grid, Us, S, stream);
   *launches = 2;
   return e;

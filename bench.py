@@ -248,11 +248,13 @@ def run_gpu(args, w):
         sampler.start()
     launches0 = cache.launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.profiler.start()      # a profiler started with capture off sees only the timed region
     e0.record()
     for i in range(Wm, Wm + K):
         step(i)
     e1.record()
     barrier()
+    torch.cuda.profiler.stop()
     ms = e0.elapsed_time(e1)
     launches = cache.launch_count() - launches0
     flushes = sum(1 for i in range(Wm, Wm + K) if (w.tokens + i) % w.residual_len == 0) * w.n_layers

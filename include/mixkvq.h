@@ -41,7 +41,9 @@ enum {
   MIXKVQ_E_BUFFER_TOO_SMALL = -4,     /* cache memory or attention workspace smaller than required   */
   MIXKVQ_E_CAPACITY = -5,             /* append would exceed max_tokens                              */
   MIXKVQ_E_CUDA = -6,                 /* a CUDA runtime call or kernel launch reported an error      */
-  MIXKVQ_E_EMPTY = -7                 /* attention or selection requested on a layer with no tokens  */
+  MIXKVQ_E_EMPTY = -7,                /* attention or selection requested on a layer with no tokens  */
+  MIXKVQ_E_BUILTIN_SCRATCH = -8       /* mixkvq_decode_attention_noalloc: batch * n_kv_heads exceeds
+                                         MIXKVQ_NOALLOC_MAX_STREAMS                                  */
 };
 
 /* bits of the sticky device status word */
@@ -127,6 +129,27 @@ int mixkvq_quantize_append(mixkvq_cache* cache, int layer, const void* k_dev, co
  *   workspace_dev: at least attn_workspace_bytes (mixkvq_cache_bytes); contents are scratch */
 int mixkvq_decode_attention(mixkvq_cache* cache, int layer, const void* q_dev, float* out_dev, float softmax_scale,
                             void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/* (The paper has no counterpart of this entry point; it exists for integration reasons only.)
+ * Same computation and same results as mixkvq_decode_attention, for callers that have no way to hand
+ * over a workspace: code that runs inside a serving engine's pre-sized memory pool, a plugin that may
+ * not call cudaMalloc (or any allocating library routine) once the engine has started, or a host
+ * program written in a language binding that exposes no device allocator.  The split partials go to a
+ * scratch array that is compiled into the library (static device storage of
+ * (1184 + MIXKVQ_NOALLOC_MAX_STREAMS) * 4160 bytes, about 5.7 MiB, which every GPU that loads the
+ * library holds until the process exits).  The call allocates and frees nothing.
+ *   - batch * n_kv_heads of the cache must be <= MIXKVQ_NOALLOC_MAX_STREAMS, else
+ *     MIXKVQ_E_BUILTIN_SCRATCH is returned and nothing is launched.
+ *   - The first call on each device looks up the device address of the scratch array (with that device
+ *     current, which must be the device that owns the cache memory).  Make that first call before any
+ *     stream capture begins.
+ *   - All calls on a device share the one array.  Nothing in it has to start at zero (every partial a
+ *     call reads was written by that same call), so stale contents of earlier calls are harmless; but
+ *     two calls whose kernels overlap on the GPU (different streams, no ordering between them) race on
+ *     it and both results are undefined.  Calls on one stream are ordered and safe. */
+#define MIXKVQ_NOALLOC_MAX_STREAMS 256
+int mixkvq_decode_attention_noalloc(mixkvq_cache* cache, int layer, const void* q_dev, float* out_dev,
+                                    float softmax_scale, void* stream);
 
 /* Selects the decode-attention kernel: 0 = tensor-core kernel (default), 1 = plain-ALU kernel
  * (kept for comparison; same results within tolerance, much slower), 2 = the tensor-core split kernel

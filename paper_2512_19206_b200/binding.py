@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libmixkvq.so")
 EXPORTS = [
     "mixkvq_cache_bytes", "mixkvq_cache_init", "mixkvq_cache_destroy", "mixkvq_cache_reset",
     "mixkvq_select_channels", "mixkvq_select_channels_raw", "mixkvq_quantize_append",
-    "mixkvq_decode_attention", "mixkvq_set_attention_kernel", "mixkvq_query_status",
+    "mixkvq_decode_attention", "mixkvq_decode_attention_noalloc", "mixkvq_set_attention_kernel", "mixkvq_query_status",
     "mixkvq_cache_describe", "mixkvq_launch_count", "mixkvq_status_string",
 ]
 
@@ -66,6 +66,7 @@ def lib():
         L.mixkvq_select_channels_raw.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32, f32, f32, vp, vp, vp]
         L.mixkvq_quantize_append.argtypes = [vp, i32, vp, vp, vp, i32, vp]
         L.mixkvq_decode_attention.argtypes = [vp, i32, vp, vp, f32, vp, C.c_size_t, vp]
+        L.mixkvq_decode_attention_noalloc.argtypes = [vp, i32, vp, vp, f32, vp]
         L.mixkvq_set_attention_kernel.argtypes = [vp, i32]
         L.mixkvq_query_status.argtypes = [vp, C.POINTER(i32), vp]
         L.mixkvq_cache_describe.argtypes = [vp, i32, C.POINTER(LayoutDesc)]
@@ -163,6 +164,17 @@ class Cache:
         _check(lib().mixkvq_decode_attention(self.handle, layer, _ptr(q), _ptr(out), float(scale),
                                              _ptr(self.workspace), self.workspace.numel(), _stream()),
                "mixkvq_decode_attention")
+        return out
+
+    def decode_attention_noalloc(self, layer, q, scale, out=None):
+        """Same as decode_attention, but the library's built-in scratch array holds the split partials: for
+        callers that cannot provide a workspace.  `out` should be passed by such callers (the default
+        allocates it with torch for convenience).  Calls that overlap on the GPU race on the shared array."""
+        if out is None:
+            out = torch.empty(q.shape, dtype=torch.float32, device=q.device)
+        with torch.cuda.device(self.mem.device):
+            _check(lib().mixkvq_decode_attention_noalloc(self.handle, layer, _ptr(q), _ptr(out), float(scale), _stream()),
+                   "mixkvq_decode_attention_noalloc")
         return out
 
     def select_channels(self, layer, want_salience=True):

@@ -238,6 +238,39 @@ int mixkvq_decode_attention(mixkvq_cache* cache, int layer, const void* q_dev, f
   return e == cudaSuccess ? MIXKVQ_OK : MIXKVQ_E_CUDA;
 }
 
+// ---- decode attention with the split partials in storage compiled into the library (no allocation)
+namespace {
+constexpr size_t kBuiltinScratchBytes =
+    (size_t)(kMaxCtas + MIXKVQ_NOALLOC_MAX_STREAMS) * kPartialFloats * sizeof(float);
+constexpr int kMaxDevices = 64;
+}  // namespace
+// In host code this name is only a handle for cudaGetSymbolAddress, never a device pointer.
+static __device__ __align__(256) unsigned char g_builtin_scratch[kBuiltinScratchBytes];
+static void* g_builtin_scratch_addr[kMaxDevices];      // device address of the array, per device ordinal
+
+int mixkvq_decode_attention_noalloc(mixkvq_cache* cache, int layer, const void* q_dev, float* out_dev,
+                                    float softmax_scale, void* stream) {
+  if (!cache || !q_dev || !out_dev || layer < 0 || layer >= cache->cfg.n_layers) return MIXKVQ_E_INVALID_ARG;
+  if (!aligned16(q_dev) || !aligned16(out_dev)) return MIXKVQ_E_ALIGNMENT;
+  if (cache->S > MIXKVQ_NOALLOC_MAX_STREAMS) return MIXKVQ_E_BUILTIN_SCRATCH;
+  if (cache->n_blocks[layer] == 0 && cache->r[layer] == 0) return MIXKVQ_E_EMPTY;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MIXKVQ_E_CUDA;
+  if (!g_builtin_scratch_addr[dev]) {
+    // once per device, with that device current: resolve the array's address on this device
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_builtin_scratch) != cudaSuccess || !p) return MIXKVQ_E_CUDA;
+    g_builtin_scratch_addr[dev] = p;
+  }
+  LayerView lv = view(cache, layer);
+  int launches = 0;
+  cudaError_t e = launch_attention_mma(lv, q_dev, out_dev, softmax_scale,
+                                       static_cast<float*>(g_builtin_scratch_addr[dev]), cache->n_sms,
+                                       static_cast<cudaStream_t>(stream), &launches);
+  cache->launches += launches;
+  return e == cudaSuccess ? MIXKVQ_OK : MIXKVQ_E_CUDA;
+}
+
 int mixkvq_set_attention_kernel(mixkvq_cache* cache, int kind) {
   if (!cache || kind < 0 || kind > 2) return MIXKVQ_E_INVALID_ARG;
   cache->attn_kind = kind;
@@ -283,6 +316,7 @@ const char* mixkvq_status_string(int status) {
     case MIXKVQ_E_CAPACITY: return "append exceeds max_tokens";
     case MIXKVQ_E_CUDA: return "CUDA error";
     case MIXKVQ_E_EMPTY: return "layer holds no tokens";
+    case MIXKVQ_E_BUILTIN_SCRATCH: return "batch * n_kv_heads exceeds the built-in scratch (MIXKVQ_NOALLOC_MAX_STREAMS)";
     default: return "unknown status";
   }
 }

@@ -284,6 +284,7 @@ def unquantized_attention(q, K, V, scale):
 
 # --------------------------------------------------------------------------------------------
 # byte layout (written from the layout section of the design document, one element at a time)
+# fragment layout: blocks of any R other than 128
 # --------------------------------------------------------------------------------------------
 def base_bytes(R, G):
     return (R // G) * 512 + (R // 32) * (2048 + 128 * (D // G))
@@ -442,6 +443,111 @@ def unpack_base(buf, R, G):
     return klow, ks, kz, vcodes, vs, vz
 
 
+# --------------------------------------------------------------------------------------------
+# tile layout (blocks of R = 128 tokens): one thread of the attention kernel owns one token's key codes
+# and one channel's value codes, each a contiguous run of 2-bit fields
+# --------------------------------------------------------------------------------------------
+def uses_tile_layout(R):
+    return R == 128
+
+
+def tile_base_bytes(G):
+    return (128 // G) * 512 + 4096 + 4096 + 128 * (D // G) * 4
+
+
+def tile_extras_bytes(n16, n4):
+    n16p, n4w = (n16 + 1) // 2, (n4 + 15) // 16
+    return 16 * ((2 * n16p + 16 * n4w + 15) // 16) + 512 * (n16p + n4w)
+
+
+def _tile_code_pos(row, i):
+    """Code number i (0..127) of a 32-byte row: (byte offset of the 32-bit word inside the 4096-byte plane,
+    bit offset).  Keys: row = token, i = channel.  Values: row = channel, i = token."""
+    hh, rem = divmod(i, 64)
+    w, rem = divmod(rem, 16)
+    f, e = divmod(rem, 2)
+    return hh * 2048 + row * 16 + w * 4, 16 * e + 2 * f
+
+
+def _tile_tables():
+    if not hasattr(_tile_tables, "cache"):
+        wi = np.zeros((128, 128), np.int64); bi = np.zeros((128, 128), np.int64)
+        for row in range(128):
+            for i in range(128):
+                off, bit = _tile_code_pos(row, i)
+                wi[row, i], bi[row, i] = off // 4, bit
+        assert len(set(zip(wi.ravel().tolist(), bi.ravel().tolist()))) == 128 * 128
+        assert wi.max() == 1023 and bi.max() == 30
+        _tile_tables.cache = (wi, bi)
+    return _tile_tables.cache
+
+
+def pack_base_tile(blk: Block, G):
+    NG, VG = 128 // G, D // G
+    wi, bi = _tile_tables()
+    words = np.zeros(tile_base_bytes(G) // 4, np.uint32)
+    quant = blk.tiers != TIER_BF16
+    ks16 = np.where(quant[None, :], bf16_to_u16(blk.ks), 0).astype(np.uint32)
+    kz16 = np.where(quant[None, :], bf16_to_u16(blk.kz), 0).astype(np.uint32)
+    words[:NG * 128] = (ks16 | (kz16 << 16)).reshape(NG * 128)            # entry (kg, d) at kg*512 + d*4
+    klow = np.where(quant[None, :], blk.kcodes & 3, 0)
+    kbase = NG * 128
+    _scatter_codes(words, kbase + wi, bi, klow)                            # row = token, i = channel
+    _scatter_codes(words, kbase + 1024 + wi, bi, blk.vcodes.T)             # row = channel, i = token
+    vs16, vz16 = bf16_to_u16(blk.vs).astype(np.uint32), bf16_to_u16(blk.vz).astype(np.uint32)
+    words[kbase + 2048:kbase + 2048 + 128 * VG] = (vs16 | (vz16 << 16)).reshape(128 * VG)   # (j*VG + vg)*4
+    return words.astype("<u4").tobytes()
+
+
+def unpack_base_tile(buf, G):
+    NG, VG = 128 // G, D // G
+    words = np.frombuffer(buf, dtype="<u4")
+    halves = np.frombuffer(buf, dtype="<u2")
+    ks = np.zeros((NG, D), np.float32); kz = np.zeros((NG, D), np.float32)
+    for kg in range(NG):
+        for d in range(D):
+            ks[kg, d] = u16_to_bf16(halves[(kg * 512 + d * 4) // 2])
+            kz[kg, d] = u16_to_bf16(halves[(kg * 512 + d * 4) // 2 + 1])
+    klow = np.zeros((128, D), np.uint8); vcodes = np.zeros((128, D), np.uint8)
+    vs = np.zeros((128, VG), np.float32); vz = np.zeros((128, VG), np.float32)
+    kb, vb, mb = NG * 512, NG * 512 + 4096, NG * 512 + 8192
+    for j in range(128):
+        for d in range(D):
+            off, bit = _tile_code_pos(j, d)
+            klow[j, d] = (int(words[(kb + off) // 4]) >> bit) & 3
+            off, bit = _tile_code_pos(d, j)
+            vcodes[j, d] = (int(words[(vb + off) // 4]) >> bit) & 3
+        for vg in range(VG):
+            o = (mb + (j * VG + vg) * 4) // 2
+            vs[j, vg] = u16_to_bf16(halves[o]); vz[j, vg] = u16_to_bf16(halves[o + 1])
+    return klow, ks, kz, vcodes, vs, vz
+
+
+def pack_extras_tile(blk: Block):
+    chan16, chan4 = channel_lists(blk.tiers)
+    n16, n4 = len(chan16), len(chan4)
+    n16p, n4w = (n16 + 1) // 2, (n4 + 15) // 16
+    hdr = 16 * ((2 * n16p + 16 * n4w + 15) // 16)
+    head = bytearray(hdr)
+    l16 = chan16 + [0xFF] * (2 * n16p - n16)
+    l4 = chan4 + [0xFF] * (16 * n4w - n4)
+    head[0:2 * n16p] = bytes(l16)
+    head[2 * n16p:2 * n16p + 16 * n4w] = bytes(l4)
+    words = np.zeros(128 * (n16p + n4w), np.uint32)
+    raw16 = bf16_to_u16(blk.kraw).astype(np.uint32)
+    for i in range(n16p):                                                   # word (i*128 + j)
+        lo = raw16[:, l16[2 * i]]
+        hi = raw16[:, l16[2 * i + 1]] if l16[2 * i + 1] != 0xFF else np.zeros(128, np.uint32)
+        words[i * 128:(i + 1) * 128] = lo | (hi << 16)
+    for idx, ch in enumerate(chan4):                                        # word ((n16p + w)*128 + j)
+        w, rem = divmod(idx, 16)
+        f, e = divmod(rem, 2)
+        words[(n16p + w) * 128:(n16p + w + 1) * 128] |= (blk.kcodes[:, ch] >> 2).astype(np.uint32) << np.uint32(16 * e + 2 * f)
+    out = bytes(head) + words.astype("<u4").tobytes()
+    assert len(out) == tile_extras_bytes(n16, n4)
+    return out, n16, n4
+
+
 def table_entry(extras_off16, n16, n4):
     return int(extras_off16).to_bytes(4, "little") + bytes([n16, n4, 0, 0])
 
@@ -450,9 +556,14 @@ def pack_stream(st: OracleStream):
     """All bytes the stream would hold in device memory, by region."""
     base, table, extras = [], [], []
     used16 = 0
+    tile = uses_tile_layout(st.R)
     for blk in st.blocks:
-        base.append(pack_base(blk, st.R, st.G))
-        ex, n16, n4 = pack_extras(blk, st.R)
+        if tile:
+            base.append(pack_base_tile(blk, st.G))
+            ex, n16, n4 = pack_extras_tile(blk)
+        else:
+            base.append(pack_base(blk, st.R, st.G))
+            ex, n16, n4 = pack_extras(blk, st.R)
         table.append(table_entry(used16, n16, n4))
         extras.append(ex)
         used16 += len(ex) // 16

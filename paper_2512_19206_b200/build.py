@@ -8,7 +8,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmixkvq.so")
-SOURCES = ["api.cu", "append.cu", "select.cu", "flush.cu", "combine.cu", "attention_simt.cu", "attention_mma.cu"]
+SOURCES = ["api.cu", "append.cu", "select.cu", "flush.cu", "combine.cu", "attention_simt.cu", "attention_mma.cu",
+           "attention_tc.cu"]
 
 
 def _stale() -> bool:

@@ -11,7 +11,7 @@ struct mixkvq_cache {
   mixkvq_config cfg;
   char* mem;
   size_t bytes;
-  int S, g, R, G, U, NG, VG, max_blocks;
+  int S, g, R, G, U, NG, VG, max_blocks, tile;
   uint32_t base_bytes, unit_bytes;
   uint64_t extras_budget;
   // byte offsets inside one layer and per-stream strides
@@ -57,7 +57,9 @@ uint64_t plan(const mixkvq_config* c, mixkvq_cache* h) {
   h->VG = kD / h->G;
   h->max_blocks = (c->max_tokens + h->R - 1) / h->R;
   h->unit_bytes = 2048u + 128u * h->VG;
-  h->base_bytes = (uint32_t)h->NG * 512u + (uint32_t)h->U * h->unit_bytes;
+  h->tile = (h->R == 128) ? 1 : 0;
+  h->base_bytes = h->tile ? (uint32_t)h->NG * 512u + 8192u + 512u * (uint32_t)h->VG
+                          : (uint32_t)h->NG * 512u + (uint32_t)h->U * h->unit_bytes;
   h->extras_budget = c->extras_budget_bytes ? align_up(c->extras_budget_bytes, 16)
                                             : align_up((uint64_t)h->max_blocks * h->R * 32, 256);
   h->state_stride = kStateBytes;
@@ -85,6 +87,7 @@ LayerView view(const mixkvq_cache* h, int layer) {
   v.R = h->R; v.G = h->G; v.U = h->U; v.NG = h->NG; v.VG = h->VG;
   v.max_blocks = h->max_blocks;
   v.n_blocks = h->n_blocks[layer]; v.r = h->r[layer];
+  v.tile = h->tile;
   v.base_bytes = h->base_bytes; v.unit_bytes = h->unit_bytes;
   v.extras_budget = h->extras_budget;
   v.score_bits = h->cfg.score_bits; v.importance_mode = h->cfg.importance_mode;
@@ -108,6 +111,21 @@ int zero_layer_state(mixkvq_cache* h, int layer, cudaStream_t st) {
   h->n_blocks[layer] = 0;
   h->r[layer] = 0;
   return MIXKVQ_OK;
+}
+
+// Picks the decode-attention kernel for the layer's layout and the selected kind, enqueues it and counts its launches.
+int run_attention(mixkvq_cache* h, int layer, const void* q, float* out, float scale, float* ws, cudaStream_t st) {
+  LayerView lv = view(h, layer);
+  int launches = 0;
+  cudaError_t e;
+  if (h->attn_kind == 1)
+    e = launch_attention_simt(lv, q, out, scale, ws, h->n_sms, st, &launches);
+  else if (h->tile)
+    e = launch_attention_tc(lv, q, h->attn_kind == 2 ? nullptr : out, scale, ws, h->n_sms, st, &launches);
+  else
+    e = launch_attention_mma(lv, q, h->attn_kind == 2 ? nullptr : out, scale, ws, h->n_sms, st, &launches);
+  h->launches += launches;
+  return e == cudaSuccess ? MIXKVQ_OK : MIXKVQ_E_CUDA;
 }
 
 }  // namespace
@@ -224,18 +242,8 @@ int mixkvq_decode_attention(mixkvq_cache* cache, int layer, const void* q_dev, f
   if (!aligned16(q_dev) || !aligned16(out_dev) || !aligned16(workspace_dev)) return MIXKVQ_E_ALIGNMENT;
   if (workspace_bytes_given < workspace_bytes(cache->S)) return MIXKVQ_E_BUFFER_TOO_SMALL;
   if (cache->n_blocks[layer] == 0 && cache->r[layer] == 0) return MIXKVQ_E_EMPTY;
-  LayerView lv = view(cache, layer);
-  int launches = 0;
-  cudaError_t e;
-  if (cache->attn_kind == 1)
-    e = launch_attention_simt(lv, q_dev, out_dev, softmax_scale, static_cast<float*>(workspace_dev), cache->n_sms,
-                              static_cast<cudaStream_t>(stream), &launches);
-  else
-    e = launch_attention_mma(lv, q_dev, cache->attn_kind == 2 ? nullptr : out_dev, softmax_scale,
-                             static_cast<float*>(workspace_dev), cache->n_sms, static_cast<cudaStream_t>(stream),
-                             &launches);
-  cache->launches += launches;
-  return e == cudaSuccess ? MIXKVQ_OK : MIXKVQ_E_CUDA;
+  return run_attention(cache, layer, q_dev, out_dev, softmax_scale, static_cast<float*>(workspace_dev),
+                       static_cast<cudaStream_t>(stream));
 }
 
 // ---- decode attention with the split partials in storage compiled into the library (no allocation)
@@ -262,13 +270,8 @@ int mixkvq_decode_attention_noalloc(mixkvq_cache* cache, int layer, const void* 
     if (cudaGetSymbolAddress(&p, g_builtin_scratch) != cudaSuccess || !p) return MIXKVQ_E_CUDA;
     g_builtin_scratch_addr[dev] = p;
   }
-  LayerView lv = view(cache, layer);
-  int launches = 0;
-  cudaError_t e = launch_attention_mma(lv, q_dev, out_dev, softmax_scale,
-                                       static_cast<float*>(g_builtin_scratch_addr[dev]), cache->n_sms,
-                                       static_cast<cudaStream_t>(stream), &launches);
-  cache->launches += launches;
-  return e == cudaSuccess ? MIXKVQ_OK : MIXKVQ_E_CUDA;
+  return run_attention(cache, layer, q_dev, out_dev, softmax_scale, static_cast<float*>(g_builtin_scratch_addr[dev]),
+                       static_cast<cudaStream_t>(stream));
 }
 
 int mixkvq_set_attention_kernel(mixkvq_cache* cache, int kind) {

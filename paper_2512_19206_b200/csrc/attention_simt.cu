@@ -71,22 +71,37 @@ attention_simt_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float s
       const uint32_t* kcodes = reinterpret_cast<const uint32_t*>(ub_ptr);
       const char* exu = ex + extras_header_bytes(n16, n4) + (size_t)u * extras_unit_bytes(n16, n4);
       const int n16p = (n16 + 1) >> 1;
+      // tile layout (R == 128): planes of the whole block, token j of the block
+      const int jt = 32 * u + lane;
+      const char* kplane = blk + lv.NG * 512;
+      const uint32_t* txw = reinterpret_cast<const uint32_t*>(ex + tile_extras_header_bytes(n16, n4));
       for (int d = 0; d < kD; ++d) {
         float kval;
         const uint8_t s16 = slot16[warp][d];
         if (s16 != 0xFF) {
-          const uint32_t w = reinterpret_cast<const uint32_t*>(exu)[(s16 >> 1) * 32 + lane];
+          const uint32_t w = lv.tile ? txw[(s16 >> 1) * 128 + jt]
+                                     : reinterpret_cast<const uint32_t*>(exu)[(s16 >> 1) * 32 + lane];
           kval = bf16_bits_to_float((s16 & 1) ? (w >> 16) : (w & 0xFFFF));
         } else {
-          int word, bit;
-          k_code_pos(lane, d, &word, &bit);
-          int code = (kcodes[word] >> bit) & 3;
+          int code;
           const uint8_t s4 = slot4[warp][d];
-          if (s4 != 0xFF) {
-            int hw, hb;
-            hi_plane_pos(lane, s4 & 1, &hw, &hb);
-            const uint32_t w = reinterpret_cast<const uint32_t*>(exu + 128 * n16p)[(s4 >> 1) * 4 + hw];
-            code += 4 * ((w >> hb) & 3);
+          if (lv.tile) {
+            const uint32_t kw = *reinterpret_cast<const uint32_t*>(kplane + (d >> 6) * 2048 + jt * 16 + ((d & 63) >> 4) * 4);
+            code = (kw >> (16 * (d & 1) + 2 * ((d & 15) >> 1))) & 3;
+            if (s4 != 0xFF) {
+              const uint32_t w = txw[(n16p + (s4 >> 4)) * 128 + jt];
+              code += 4 * ((w >> (16 * (s4 & 1) + 2 * ((s4 & 15) >> 1))) & 3);
+            }
+          } else {
+            int word, bit;
+            k_code_pos(lane, d, &word, &bit);
+            code = (kcodes[word] >> bit) & 3;
+            if (s4 != 0xFF) {
+              int hw, hb;
+              hi_plane_pos(lane, s4 & 1, &hw, &hb);
+              const uint32_t w = reinterpret_cast<const uint32_t*>(exu + 128 * n16p)[(s4 >> 1) * 4 + hw];
+              code += 4 * ((w >> hb) & 3);
+            }
           }
           const uint32_t mz = kmeta[d];
           kval = fmaf((float)code, bf16_bits_to_float(mz & 0xFFFF), bf16_bits_to_float(mz >> 16));
@@ -123,12 +138,22 @@ attention_simt_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float s
       if (unit < packed_units) {
         const uint32_t* vcodes = reinterpret_cast<const uint32_t*>(ub_ptr + 1024);
         const uint32_t* vmeta = reinterpret_cast<const uint32_t*>(ub_ptr + 2048);
+        const int u = unit % lv.U, t = 32 * u + jj;                  // tile layout: token t of the block
+        const char* tblk = base + (size_t)(unit / lv.U) * lv.base_bytes + lv.NG * 512;
         for (int i = 0; i < 4; ++i) {
           const int c = 4 * lane + i;
-          int word, bit;
-          v_code_pos(jj, c, &word, &bit);
-          const int code = (vcodes[word] >> bit) & 3;
-          const uint32_t mz = vmeta[jj * lv.VG + c / lv.G];
+          int code;
+          uint32_t mz;
+          if (lv.tile) {
+            const uint32_t vw = *reinterpret_cast<const uint32_t*>(tblk + 4096 + (t >> 6) * 2048 + c * 16 + ((t & 63) >> 4) * 4);
+            code = (vw >> (16 * (t & 1) + 2 * ((t & 15) >> 1))) & 3;
+            mz = reinterpret_cast<const uint32_t*>(tblk + 8192)[t * lv.VG + c / lv.G];
+          } else {
+            int word, bit;
+            v_code_pos(jj, c, &word, &bit);
+            code = (vcodes[word] >> bit) & 3;
+            mz = vmeta[jj * lv.VG + c / lv.G];
+          }
           vv[i] = fmaf((float)code, bf16_bits_to_float(mz & 0xFFFF), bf16_bits_to_float(mz >> 16));
         }
       } else {

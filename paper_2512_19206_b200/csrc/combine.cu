@@ -9,7 +9,7 @@ namespace mixkvq {
 __global__ void __launch_bounds__(128)
 combine_kernel(const float* __restrict__ ws, float* __restrict__ out, int g, int Hkv, int Hq, int mode, int n,
                long long units_per_stream, int S) {
-  const int s = blockIdx.x, c = threadIdx.x;
+  const int s = blockIdx.x / g, h = blockIdx.x % g, c = threadIdx.x;
   int first, count;
   if (mode == 0) {
     first = s * n;
@@ -22,24 +22,24 @@ combine_kernel(const float* __restrict__ ws, float* __restrict__ out, int g, int
     count = c1 - c0 + 1;
   }
   const int b = s / Hkv, hk = s % Hkv;
-  for (int h = 0; h < g; ++h) {
-    float M = -INFINITY;
-    for (int i = 0; i < count; ++i) M = fmaxf(M, ws[(size_t)(first + i) * kPartialFloats + h * 130]);
-    float l = 0.f, o = 0.f;
-    for (int i = 0; i < count; ++i) {
-      const float* p = ws + (size_t)(first + i) * kPartialFloats + h * 130;
-      const float m = p[0];
-      const float f = (m == -INFINITY) ? 0.f : exp2f(m - M);
-      l += f * p[1];
-      o += f * p[2 + c];
-    }
-    out[((size_t)b * Hq + hk * g + h) * kD + c] = o / l;
+  const float* base = ws + (size_t)first * kPartialFloats + h * 130;
+  float M = -INFINITY;
+  for (int i = 0; i < count; ++i) M = fmaxf(M, base[(size_t)i * kPartialFloats]);
+  float l = 0.f, o = 0.f;
+#pragma unroll 4
+  for (int i = 0; i < count; ++i) {
+    const float* p = base + (size_t)i * kPartialFloats;
+    const float m = p[0];
+    const float f = (m == -INFINITY) ? 0.f : exp2f(m - M);
+    l += f * p[1];
+    o += f * p[2 + c];
   }
+  out[((size_t)b * Hq + hk * g + h) * kD + c] = o / l;
 }
 
 cudaError_t launch_combine(const float* ws, float* out, int g, int Hkv, int Hq, int mode, int n,
                            long long units_per_stream, int S, cudaStream_t stream) {
-  combine_kernel<<<S, 128, 0, stream>>>(ws, out, g, Hkv, Hq, mode, n, units_per_stream, S);
+  combine_kernel<<<S * g, 128, 0, stream>>>(ws, out, g, Hkv, Hq, mode, n, units_per_stream, S);
   return cudaGetLastError();
 }
 

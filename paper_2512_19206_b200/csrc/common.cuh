@@ -25,6 +25,7 @@ struct LayerView {
   int R, G, U, NG, VG;        // residual length, group size, units/block, key groups/block, value groups/token
   int max_blocks;
   int n_blocks, r;            // current fill (same for all streams)
+  int tile;                   // 1: tile layout (R == 128), 0: fragment layout
   uint32_t base_bytes, unit_bytes;
   uint64_t extras_budget;     // bytes per stream
   // method parameters
@@ -47,6 +48,16 @@ __host__ __device__ inline uint32_t extras_header_bytes(int n16, int n4) {
 __host__ __device__ inline uint32_t extras_unit_bytes(int n16, int n4) {
   int n16p = (n16 + 1) >> 1, n4p = ((n4 + 1) >> 1) << 1;
   return 128u * n16p + 8u * n4p;
+}
+
+// tile layout (R == 128): header [chan16: 2*n16p][chan4: 16*n4w][pad to 16], body (n16p + n4w) x 128 words
+__host__ __device__ inline uint32_t tile_extras_header_bytes(int n16, int n4) {
+  int n16p = (n16 + 1) >> 1, n4w = (n4 + 15) >> 4;
+  return 16u * ((2 * n16p + 16 * n4w + 15) >> 4);
+}
+__host__ __device__ inline uint32_t tile_extras_body_bytes(int n16, int n4) {
+  int n16p = (n16 + 1) >> 1, n4w = (n4 + 15) >> 4;
+  return 512u * (n16p + n4w);
 }
 
 // ---- bf16 bit helpers (no rounding involved)
@@ -125,4 +136,8 @@ cudaError_t launch_attention_simt(const LayerView& lv, const void* q, float* out
 cudaError_t launch_attention_mma(const LayerView& lv, const void* q, float* out, float scale, float* ws,
                                  int n_sms, cudaStream_t stream, int* launches);
 cudaError_t attention_mma_setup();
+// tile layout (R == 128): tcgen05 kernel
+cudaError_t launch_attention_tc(const LayerView& lv, const void* q, float* out, float scale, float* ws,
+                                int n_sms, cudaStream_t stream, int* launches);
+cudaError_t attention_tc_setup();
 }  // namespace mixkvq

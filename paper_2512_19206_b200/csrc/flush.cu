@@ -69,7 +69,8 @@ flush_kernel(LayerView lv) {
     }
     uint32_t* used = reinterpret_cast<uint32_t*>(state + 1028);
     uint32_t off16 = *used;
-    uint32_t need = extras_header_bytes(n16, n4) + (uint32_t)U * extras_unit_bytes(n16, n4);
+    uint32_t need = lv.tile ? tile_extras_header_bytes(n16, n4) + tile_extras_body_bytes(n16, n4)
+                            : extras_header_bytes(n16, n4) + (uint32_t)U * extras_unit_bytes(n16, n4);
     if ((uint64_t)off16 * 16 + need > lv.extras_budget) {
       atomicOr(lv.status, (uint32_t)MIXKVQ_DEV_EXTRAS_FULL);
       n16 = 0;
@@ -90,50 +91,86 @@ flush_kernel(LayerView lv) {
   char* ex = lv.extras + (size_t)s * lv.extras_stride + (size_t)misc[2] * 16;
   const uint32_t hdr = extras_header_bytes(n16, n4), exunit = extras_unit_bytes(n16, n4);
 
-  // ---- key low plane, fragment order
-  for (int i = tid; i < U * 256; i += 256) {
-    const int u = i >> 8, wi = i & 255;
-    const int mt = wi >> 7, lane = (wi >> 2) & 31, a = wi & 3;
-    const int r = lane >> 2, t = lane & 3, ch = a >> 1, rh = a & 1;
-    const int j = 32 * u + mt * 16 + rh * 8 + r;
-    uint32_t w = 0;
+  if (lv.tile) {
+    // ---- tile layout (R = 128): a token's key codes are 32 contiguous bytes (two 16-byte halves)
+    char* kplane = blk + NG * 512;
+    for (int i = tid; i < 128 * 8; i += 256) {
+      const int j = i >> 3, W = i & 7;
+      uint32_t w = 0;
 #pragma unroll
-    for (int kt = 0; kt < 8; ++kt)
+      for (int f = 0; f < 8; ++f)
 #pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        const int d = kt * 16 + ch * 8 + 2 * t + e;
-        w |= (uint32_t)(cS[j * kD + d] & 3) << (16 * e + 2 * kt);
-      }
-    reinterpret_cast<uint32_t*>(blk + NG * 512 + (size_t)u * lv.unit_bytes)[wi] = w;
-  }
-  // ---- extras: header, BF16 pairs, UINT4 high plane
-  for (int i = tid; i < (int)hdr; i += 256) {
-    uint8_t b = 0;
-    if (i < 2 * n16p) b = (i < n16) ? chan16S[i] : 0xFF;
-    else if (i < 2 * n16p + n4p) b = (i - 2 * n16p < n4) ? chan4S[i - 2 * n16p] : 0xFF;
-    ex[i] = (char)b;
-  }
-  for (int i = tid; i < U * n16p * 32; i += 256) {
-    const int u = i / (n16p * 32), rem = i % (n16p * 32), p = rem >> 5, jj = rem & 31;
-    const int j = 32 * u + jj;
-    uint32_t w = kS[j * kD + chan16S[2 * p]];
-    if (2 * p + 1 < n16) w |= (uint32_t)kS[j * kD + chan16S[2 * p + 1]] << 16;
-    reinterpret_cast<uint32_t*>(ex + hdr + (size_t)u * exunit)[rem] = w;
-  }
-  for (int i = tid; i < U * (n4p / 2) * 4; i += 256) {
-    const int u = i / (n4p * 2), rem = i % (n4p * 2), p = rem >> 2, wj = rem & 3;
-    uint32_t w = 0;
-    for (int e = 0; e < 2; ++e) {
-      if (2 * p + e >= n4) continue;
-      const int d = chan4S[2 * p + e];
-      for (int rhi = 0; rhi < 2; ++rhi)
-        for (int mt = 0; mt < 2; ++mt)
-          for (int rh = 0; rh < 2; ++rh) {
-            const int j = 32 * u + mt * 16 + rh * 8 + wj + 4 * rhi;
-            w |= (uint32_t)(cS[j * kD + d] >> 2) << (16 * e + 8 * rhi + 2 * (2 * mt + rh));
-          }
+        for (int e = 0; e < 2; ++e) w |= (uint32_t)(cS[j * kD + 16 * W + 2 * f + e] & 3) << (16 * e + 2 * f);
+      *reinterpret_cast<uint32_t*>(kplane + (W >> 2) * 2048 + j * 16 + (W & 3) * 4) = w;
     }
-    reinterpret_cast<uint32_t*>(ex + hdr + (size_t)u * exunit + 128 * n16p)[rem] = w;
+    const int n4w = (n4 + 15) >> 4;
+    const uint32_t thdr = tile_extras_header_bytes(n16, n4);
+    for (int i = tid; i < (int)thdr; i += 256) {
+      uint8_t b = 0;
+      if (i < 2 * n16p) b = (i < n16) ? chan16S[i] : 0xFF;
+      else if (i < 2 * n16p + 16 * n4w) b = (i - 2 * n16p < n4) ? chan4S[i - 2 * n16p] : 0xFF;
+      ex[i] = (char)b;
+    }
+    uint32_t* xw = reinterpret_cast<uint32_t*>(ex + thdr);
+    for (int i = tid; i < n16p * 128; i += 256) {
+      const int p = i >> 7, j = i & 127;
+      uint32_t w = kS[j * kD + chan16S[2 * p]];
+      if (2 * p + 1 < n16) w |= (uint32_t)kS[j * kD + chan16S[2 * p + 1]] << 16;
+      xw[i] = w;
+    }
+    for (int i = tid; i < n4w * 128; i += 256) {
+      const int wq = i >> 7, j = i & 127;
+      uint32_t w = 0;
+      for (int k = 0; k < 16 && 16 * wq + k < n4; ++k)
+        w |= (uint32_t)(cS[j * kD + chan4S[16 * wq + k]] >> 2) << (16 * (k & 1) + 2 * (k >> 1));
+      xw[n16p * 128 + i] = w;
+    }
+  } else {
+    // ---- key low plane, fragment order
+    for (int i = tid; i < U * 256; i += 256) {
+      const int u = i >> 8, wi = i & 255;
+      const int mt = wi >> 7, lane = (wi >> 2) & 31, a = wi & 3;
+      const int r = lane >> 2, t = lane & 3, ch = a >> 1, rh = a & 1;
+      const int j = 32 * u + mt * 16 + rh * 8 + r;
+      uint32_t w = 0;
+#pragma unroll
+      for (int kt = 0; kt < 8; ++kt)
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+          const int d = kt * 16 + ch * 8 + 2 * t + e;
+          w |= (uint32_t)(cS[j * kD + d] & 3) << (16 * e + 2 * kt);
+        }
+      reinterpret_cast<uint32_t*>(blk + NG * 512 + (size_t)u * lv.unit_bytes)[wi] = w;
+    }
+    // ---- extras: header, BF16 pairs, UINT4 high plane
+    for (int i = tid; i < (int)hdr; i += 256) {
+      uint8_t b = 0;
+      if (i < 2 * n16p) b = (i < n16) ? chan16S[i] : 0xFF;
+      else if (i < 2 * n16p + n4p) b = (i - 2 * n16p < n4) ? chan4S[i - 2 * n16p] : 0xFF;
+      ex[i] = (char)b;
+    }
+    for (int i = tid; i < U * n16p * 32; i += 256) {
+      const int u = i / (n16p * 32), rem = i % (n16p * 32), p = rem >> 5, jj = rem & 31;
+      const int j = 32 * u + jj;
+      uint32_t w = kS[j * kD + chan16S[2 * p]];
+      if (2 * p + 1 < n16) w |= (uint32_t)kS[j * kD + chan16S[2 * p + 1]] << 16;
+      reinterpret_cast<uint32_t*>(ex + hdr + (size_t)u * exunit)[rem] = w;
+    }
+    for (int i = tid; i < U * (n4p / 2) * 4; i += 256) {
+      const int u = i / (n4p * 2), rem = i % (n4p * 2), p = rem >> 2, wj = rem & 3;
+      uint32_t w = 0;
+      for (int e = 0; e < 2; ++e) {
+        if (2 * p + e >= n4) continue;
+        const int d = chan4S[2 * p + e];
+        for (int rhi = 0; rhi < 2; ++rhi)
+          for (int mt = 0; mt < 2; ++mt)
+            for (int rh = 0; rh < 2; ++rh) {
+              const int j = 32 * u + mt * 16 + rh * 8 + wj + 4 * rhi;
+              w |= (uint32_t)(cS[j * kD + d] >> 2) << (16 * e + 8 * rhi + 2 * (2 * mt + rh));
+            }
+      }
+      reinterpret_cast<uint32_t*>(ex + hdr + (size_t)u * exunit + 128 * n16p)[rem] = w;
+    }
   }
   __syncthreads();
 
@@ -150,28 +187,43 @@ flush_kernel(LayerView lv) {
     for (int c = vg * G; c < (vg + 1) * G; ++c)
       cS[j * kD + c] = (uint8_t)quant_code(bf16_bits_to_float(resv[(size_t)c * R + j]), gmn, sc, 3);
     const int u = j >> 5, jj = j & 31;
-    reinterpret_cast<uint32_t*>(blk + NG * 512 + (size_t)u * lv.unit_bytes + 2048)[jj * VG + vg] =
-        float_to_bf16_bits_exact(sc) | (float_to_bf16_bits_exact(gmn) << 16);
+    uint32_t* vmeta = lv.tile ? reinterpret_cast<uint32_t*>(blk + NG * 512 + 8192) + j * VG
+                              : reinterpret_cast<uint32_t*>(blk + NG * 512 + (size_t)u * lv.unit_bytes + 2048) + jj * VG;
+    vmeta[vg] = float_to_bf16_bits_exact(sc) | (float_to_bf16_bits_exact(gmn) << 16);
   }
   __syncthreads();
-  for (int i = tid; i < U * 256; i += 256) {
-    const int u = i >> 8, wi = i & 255;
-    const int ct = (wi >> 7) * 4 + (wi & 3), lane = (wi >> 2) & 31;
-    const int r = lane >> 2, t = lane & 3;
-    uint32_t w = 0;
+  if (lv.tile) {
+    // a channel's value codes over the 128 tokens are 32 contiguous bytes (two 16-byte halves)
+    char* vplane = blk + NG * 512 + 4096;
+    for (int i = tid; i < 128 * 8; i += 256) {
+      const int c = i & 127, W = i >> 7;
+      uint32_t w = 0;
 #pragma unroll
-    for (int rh = 0; rh < 2; ++rh)
+      for (int f = 0; f < 8; ++f)
 #pragma unroll
-      for (int ks = 0; ks < 2; ++ks)
+        for (int e = 0; e < 2; ++e) w |= (uint32_t)cS[(16 * W + 2 * f + e) * kD + c] << (16 * e + 2 * f);
+      *reinterpret_cast<uint32_t*>(vplane + (W >> 2) * 2048 + c * 16 + (W & 3) * 4) = w;
+    }
+  } else {
+    for (int i = tid; i < U * 256; i += 256) {
+      const int u = i >> 8, wi = i & 255;
+      const int ct = (wi >> 7) * 4 + (wi & 3), lane = (wi >> 2) & 31;
+      const int r = lane >> 2, t = lane & 3;
+      uint32_t w = 0;
 #pragma unroll
-        for (int ch = 0; ch < 2; ++ch)
+      for (int rh = 0; rh < 2; ++rh)
 #pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const int c = ct * 16 + rh * 8 + r;
-            const int j = 32 * u + ks * 16 + ch * 8 + 2 * t + e;
-            w |= (uint32_t)cS[j * kD + c] << (16 * e + 2 * (4 * rh + 2 * ks + ch));
-          }
-    reinterpret_cast<uint32_t*>(blk + NG * 512 + (size_t)u * lv.unit_bytes + 1024)[wi] = w;
+        for (int ks = 0; ks < 2; ++ks)
+#pragma unroll
+          for (int ch = 0; ch < 2; ++ch)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              const int c = ct * 16 + rh * 8 + r;
+              const int j = 32 * u + ks * 16 + ch * 8 + 2 * t + e;
+              w |= (uint32_t)cS[j * kD + c] << (16 * e + 2 * (4 * rh + 2 * ks + ch));
+            }
+      reinterpret_cast<uint32_t*>(blk + NG * 512 + (size_t)u * lv.unit_bytes + 1024)[wi] = w;
+    }
   }
 
   // ---- window importance: the accumulator restarts with the next window (Section 4.2)

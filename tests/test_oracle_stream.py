@@ -154,6 +154,50 @@ def test_fragment_order_of_key_codes():
             assert d == (bit % 16) // 2 * 16 + ch * 8 + 2 * t + bit // 16
 
 
+@pytest.mark.parametrize("G", [32, 64, 128])
+def test_tile_layout_roundtrip_and_content(rng, G):
+    st, k, v = _flushed(rng, 128, G)
+    blk = st.blocks[0]
+    chan16 = [d for d in range(128) if blk.tiers[d] == 2]
+    chan4 = [d for d in range(128) if blk.tiers[d] == 1]
+    n16, n4 = len(chan16), len(chan4)
+    assert n16 >= 3 and n4 >= 5
+    base = O.pack_base_tile(blk, G)
+    assert len(base) == (128 // G) * 512 + 8192 + 512 * (128 // G) == O.tile_base_bytes(G)
+    klow, ks, kz, vc, vs, vz = O.unpack_base_tile(base, G)
+    quant = blk.tiers != O.TIER_BF16
+    assert np.array_equal(klow[:, quant], blk.kcodes[:, quant] & 3)
+    assert not klow[:, ~quant].any() and not ks[:, ~quant].any() and not kz[:, ~quant].any()
+    assert np.array_equal(ks[:, quant], blk.ks[:, quant]) and np.array_equal(kz[:, quant], blk.kz[:, quant])
+    assert np.array_equal(vc, blk.vcodes) and np.array_equal(vs, blk.vs) and np.array_equal(vz, blk.vz)
+    # by hand: token 77's key codes are the 32 bytes at {0, 2048} + 77*16 of the key plane, channel d in
+    # word (d % 64) // 16 of half d // 64, field (d % 16) // 2 of 16-bit half d % 2
+    kplane = np.frombuffer(base[(128 // G) * 512:(128 // G) * 512 + 4096], "<u2")
+    for d in [0, 1, 17, 63, 64, 100, 127]:
+        if quant[d]:
+            half = kplane[((d // 64) * 2048 + 77 * 16 + ((d % 64) // 16) * 4) // 2 + d % 2]
+            assert (int(half) >> (2 * ((d % 16) // 2))) & 3 == blk.kcodes[77, d] & 3
+    vplane = np.frombuffer(base[(128 // G) * 512 + 4096:(128 // G) * 512 + 8192], "<u2")
+    for t in [0, 15, 16, 64, 99, 127]:
+        half = vplane[((t // 64) * 2048 + 5 * 16 + ((t % 64) // 16) * 4) // 2 + t % 2]
+        assert (int(half) >> (2 * ((t % 16) // 2))) & 3 == blk.vcodes[t, 5]
+    ex, a, b = O.pack_extras_tile(blk)
+    n16p, n4w = (n16 + 1) // 2, (n4 + 15) // 16
+    assert (a, b) == (n16, n4) and len(ex) == 16 * ((2 * n16p + 16 * n4w + 15) // 16) + 512 * (n16p + n4w)
+    hdr = len(ex) - 512 * (n16p + n4w)
+    assert list(ex[:n16]) == chan16 and list(ex[2 * n16p:2 * n16p + n4]) == chan4
+    assert all(x in (0, 0xFF) for x in ex[2 * n16p + n4:hdr])
+    words = np.frombuffer(ex[hdr:], "<u4")
+    raw = O.bf16_to_u16(k[:128])
+    for (j, i) in [(0, 0), (37, 1), (127, n16p - 1)]:
+        w = int(words[i * 128 + j])
+        assert (w & 0xFFFF) == raw[j, chan16[2 * i]]
+        assert (w >> 16) == (raw[j, chan16[2 * i + 1]] if 2 * i + 1 < n16 else 0)
+    for (j, idx) in [(0, 0), (45, 1), (100, n4 - 1)]:
+        w = int(words[(n16p + idx // 16) * 128 + j])
+        assert (w >> (16 * (idx % 2) + 2 * ((idx % 16) // 2))) & 3 == blk.kcodes[j, chan4[idx]] >> 2
+
+
 def test_stream_regions(rng):
     k, v, q = _tokens(rng, 3 * 128 + 5, 2)
     st = O.OracleStream(g=2, tau_bf16=6.0, tau_u4=3.0)
@@ -165,7 +209,7 @@ def test_stream_regions(rng):
         e = p["table"][8 * i:8 * i + 8]
         assert int.from_bytes(e[:4], "little") == off
         assert e[4] == (blk.tiers == 2).sum() and e[5] == (blk.tiers == 1).sum() and e[6:] == b"\0\0"
-        off += len(O.pack_extras(blk, 128)[0]) // 16
+        off += len(O.pack_extras_tile(blk)[0]) // 16
     assert int.from_bytes(p["state"][1028:1032], "little") == off
     assert len(p["resK"]) == 5 * 256 and len(p["resV_T"]) == 5 * 256
     assert np.array_equal(np.frombuffer(p["resV_T"], "<u2").reshape(128, 5), O.bf16_to_u16(v[-5:]).T)

@@ -136,7 +136,7 @@ int mixkvq_decode_attention(mixkvq_cache* cache, int layer, const void* q_dev, f
  * not call cudaMalloc (or any allocating library routine) once the engine has started, or a host
  * program written in a language binding that exposes no device allocator.  The split partials go to a
  * scratch array that is compiled into the library (static device storage of
- * (1184 + MIXKVQ_NOALLOC_MAX_STREAMS) * 4160 bytes, about 5.7 MiB, which every GPU that loads the
+ * (1184 + 2 * MIXKVQ_NOALLOC_MAX_STREAMS) * 4160 bytes, about 6.7 MiB, which every GPU that loads the
  * library holds until the process exits).  The call allocates and frees nothing.
  *   - batch * n_kv_heads of the cache must be <= MIXKVQ_NOALLOC_MAX_STREAMS, else
  *     MIXKVQ_E_BUILTIN_SCRATCH is returned and nothing is launched.

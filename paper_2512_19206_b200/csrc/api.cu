@@ -79,7 +79,7 @@ uint64_t plan(const mixkvq_config* c, mixkvq_cache* h) {
   return kHeaderBytes + h->layer_stride * (uint64_t)c->n_layers;
 }
 
-size_t workspace_bytes(int S) { return (size_t)(kMaxCtas + S) * kPartialFloats * sizeof(float); }
+size_t workspace_bytes(int S) { return (size_t)(kMaxCtas + 2 * S) * kPartialFloats * sizeof(float); }
 
 LayerView view(const mixkvq_cache* h, int layer) {
   LayerView v{};
@@ -167,7 +167,7 @@ int mixkvq_cache_init(const mixkvq_config* cfg, void* cache_dev, size_t bytes, v
   if (cudaMemsetAsync(h->mem, 0, kHeaderBytes, st) != cudaSuccess) { delete h; return MIXKVQ_E_CUDA; }
   for (int l = 0; l < cfg->n_layers; ++l)
     if (zero_layer_state(h, l, st) != MIXKVQ_OK) { delete h; return MIXKVQ_E_CUDA; }
-  if (attention_mma_setup() != cudaSuccess) { delete h; return MIXKVQ_E_CUDA; }
+  if (attention_mma_setup() != cudaSuccess || attention_tc_setup() != cudaSuccess) { delete h; return MIXKVQ_E_CUDA; }
   *out = h;
   return MIXKVQ_OK;
 }
@@ -249,7 +249,7 @@ int mixkvq_decode_attention(mixkvq_cache* cache, int layer, const void* q_dev, f
 // ---- decode attention with the split partials in storage compiled into the library (no allocation)
 namespace {
 constexpr size_t kBuiltinScratchBytes =
-    (size_t)(kMaxCtas + MIXKVQ_NOALLOC_MAX_STREAMS) * kPartialFloats * sizeof(float);
+    (size_t)(kMaxCtas + 2 * MIXKVQ_NOALLOC_MAX_STREAMS) * kPartialFloats * sizeof(float);
 constexpr int kMaxDevices = 64;
 }  // namespace
 // In host code this name is only a handle for cudaGetSymbolAddress, never a device pointer.

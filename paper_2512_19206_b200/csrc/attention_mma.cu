@@ -659,13 +659,19 @@ cudaError_t attention_mma_setup() {
   return cudaFuncSetAttribute(attention_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
 }
 
+// Number of CTAs the split kernel runs for this layer state (also the number of partial-slot owners).
+int attention_mma_grid(const LayerView& lv, int n_sms) {
+  const long long Us = (long long)lv.n_blocks * lv.U + (lv.r + 31) / 32;
+  const long long total = Us * lv.B * lv.Hkv;
+  const int grid = (int)min((long long)min(n_sms * kCtasPerSm, kMaxCtas / 2), total);
+  return grid < 1 ? 1 : grid;
+}
+
 cudaError_t launch_attention_mma(const LayerView& lv, const void* q, float* out, float scale, float* ws, int n_sms,
                                  cudaStream_t stream, int* launches) {
   const int S = lv.B * lv.Hkv;
   const long long Us = (long long)lv.n_blocks * lv.U + (lv.r + 31) / 32;
-  const long long total = Us * S;
-  int grid = (int)min((long long)min(n_sms * kCtasPerSm, kMaxCtas), total);
-  if (grid < 1) grid = 1;
+  const int grid = attention_mma_grid(lv, n_sms);
   cudaError_t e;
   if (lv.G == 32) e = launch_g<32>(lv, q, scale, ws, grid, stream);
   else if (lv.G == 64) e = launch_g<64>(lv, q, scale, ws, grid, stream);

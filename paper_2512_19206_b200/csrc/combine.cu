@@ -43,4 +43,48 @@ cudaError_t launch_combine(const float* ws, float* out, int g, int Hkv, int Hq, 
   return cudaGetLastError();
 }
 
+// Two sets of partials per stream (packed blocks, residual window), each written by a grid that split its
+// S * units work items evenly over n CTAs or groups: member c of set k wrote its part of stream s to slot
+// base_k + c + s.
+__device__ inline void slot_range(int s, int S, int n, long long units, int* first, int* count) {
+  const long long total = units * S;
+  const long long x0 = units * s, x1 = units * (s + 1) - 1;
+  const int c0 = (int)(((x0 + 1) * n - 1) / total), c1 = (int)(((x1 + 1) * n - 1) / total);
+  *first = c0 + s;
+  *count = c1 - c0 + 1;
+}
+
+__global__ void __launch_bounds__(128)
+combine2_kernel(const float* __restrict__ ws, float* __restrict__ out, int g, int Hkv, int Hq, int S, int n1,
+                long long units1, int slot2, int n2, long long units2) {
+  const int s = blockIdx.x / g, h = blockIdx.x % g, c = threadIdx.x;
+  int f1, c1, f2, c2;
+  slot_range(s, S, n1, units1, &f1, &c1);
+  slot_range(s, S, n2, units2, &f2, &c2);
+  f2 += slot2;
+  const int b = s / Hkv, hk = s % Hkv;
+  float M = -INFINITY;
+  for (int i = 0; i < c1 + c2; ++i) {
+    const int slot = i < c1 ? f1 + i : f2 + (i - c1);
+    M = fmaxf(M, ws[(size_t)slot * kPartialFloats + h * 130]);
+  }
+  float l = 0.f, o = 0.f;
+#pragma unroll 4
+  for (int i = 0; i < c1 + c2; ++i) {
+    const int slot = i < c1 ? f1 + i : f2 + (i - c1);
+    const float* p = ws + (size_t)slot * kPartialFloats + h * 130;
+    const float m = p[0];
+    const float f = (m == -INFINITY) ? 0.f : exp2f(m - M);
+    l += f * p[1];
+    o += f * p[2 + c];
+  }
+  out[((size_t)b * Hq + hk * g + h) * kD + c] = o / l;
+}
+
+cudaError_t launch_combine2(const float* ws, float* out, int g, int Hkv, int Hq, int S, int n1, long long units1,
+                            int slot2, int n2, long long units2, cudaStream_t stream) {
+  combine2_kernel<<<S * g, 128, 0, stream>>>(ws, out, g, Hkv, Hq, S, n1, units1, slot2, n2, units2);
+  return cudaGetLastError();
+}
+
 }  // namespace mixkvq

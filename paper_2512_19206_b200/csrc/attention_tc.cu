@@ -48,13 +48,14 @@ struct Geo {
   static constexpr int oBq = oStages + kStages * kStage;
   static constexpr int oPb = oBq + (NQ / 8) * kBqSBO;
   static constexpr int oQh = oPb + (NV / 8) * 2048;     // [8][128] half: query of the current stream
-  static constexpr int oSh = oQh + 2048;                // [NG][128] half: key scales * 2^(4-p)
+  static constexpr int oQt = oQh + 2048;                // [16 chunks][8 heads][8] half: the same query, chunk-major
+  static constexpr int oSh = oQt + 2048;                // [NG][128] half: key scales * 2^(4-p)
   static constexpr int oZh = oSh + NG * 256;            // [NG][128] half: key zero-points
   static constexpr int oZq = oZh + NG * 256;            // [NG][8] float: q . z * scale * log2(e)
   static constexpr int oMred = oZq + 128;               // [4][8] float
   static constexpr int oRed = oMred + 128;              // [4][40] float
   static constexpr int oEnt = oRed + 640;               // [kStages] uint2 table entries, dead flag at +32
-  static constexpr int oBars = oEnt + 64;               // 11 mbarriers
+  static constexpr int oBars = oEnt + 64;               // 12 mbarriers
   static constexpr int kGroup = (oBars + 128 + 127) / 128 * 128;
   static constexpr int kSmem = kWG * kGroup + 128;
 };
@@ -195,8 +196,18 @@ __device__ __forceinline__ void expand4(const uint4 w, uint32_t (&a)[32]) {
 
 struct Bars {   // byte offsets inside the group's barrier area
   static constexpr int full = 0, empty = 8 * kStages, a_ready = 16 * kStages, s_done = a_ready + 8, ctl_ready = a_ready + 16,
-                       p_ready = a_ready + 24, o_done = a_ready + 32;
+                       p_ready = a_ready + 24, o_done = a_ready + 32, max_ready = a_ready + 40;
 };
+__device__ __forceinline__ bool elect_one() {
+  uint32_t p;
+  asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(p));
+  return p != 0;
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 
 template <int G>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -204,7 +215,7 @@ attention_tc_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
   using L = Geo<G>;
   constexpr int NG = L::NG, VG = L::VG;
   extern __shared__ __align__(128) unsigned char smem[];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0), lane = threadIdx.x & 31;   // warp-uniform
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kWG * L::kGroup);
 
   // ---- set-up: tensor memory, barriers
@@ -225,6 +236,7 @@ attention_tc_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
     mbar_init(bars + Bars::ctl_ready, 1);
     mbar_init(bars + Bars::p_ready, 4);
     mbar_init(bars + Bars::o_done, 1);
+    mbar_init(bars + Bars::max_ready, 4);
     *reinterpret_cast<volatile uint32_t*>(gs + L::oEnt + 32) = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -259,6 +271,7 @@ attention_tc_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
     float* mredS = reinterpret_cast<float*>(gs + L::oMred);
     float* redS = reinterpret_cast<float*>(gs + L::oRed);
     const uint2* entS = reinterpret_cast<const uint2*>(gs + L::oEnt);
+    const __half* qhS = reinterpret_cast<const __half*>(gs + L::oQh);
 
     float mref[8], accL[8], accZ[VG][8];
     int cur_s = -1, i = 0;
@@ -327,6 +340,7 @@ attention_tc_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
                                       : reinterpret_cast<const unsigned char*>(lv.extras) + (size_t)s * lv.extras_stride +
                                             (size_t)ent.x * 16;
       const uint32_t* exb = reinterpret_cast<const uint32_t*>(exh + tile_extras_header_bytes(n16, n4));
+      const uint32_t* kmetaS = reinterpret_cast<const uint32_t*>(st);       // [NG][128] {s, z}
 
       // one extra k-step (8 columns): promoted pairs as fp16 * 2^-10, or one word of the UINT4 high plane
       auto extra_step = [&](int e, uint32_t taddr) {
@@ -344,6 +358,54 @@ attention_tc_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
         tmem_st8(taddr, a8);
       };
 
+      // rows of the B operand (q * s, fp16 high and low parts) for extra k-steps [e0, e1), placed from row `row0`:
+      // thread = (chunk of 8 rows, head), all key groups
+      auto build_extra_rows = [&](int e0, int e1, int row0) {
+        const int hq = j & 7;
+        for (int c8 = j >> 3; c8 < 2 * (e1 - e0); c8 += 16) {
+          const int e = e0 + (c8 >> 1), half = c8 & 1;
+          float qv[8], wgt[8];
+          int chn[8];
+#pragma unroll
+          for (int r8 = 0; r8 < 8; ++r8) {
+            const int r16 = 8 * half + r8;                          // row inside the k-step
+            int ch;
+            if (e < KP) {
+              ch = exh[16 * e + r16];                               // promoted: list position 16e + r16
+              wgt[r8] = 0.0009765625f;
+            } else {
+              ch = exh[2 * n16p + 16 * (e - KP) + r16];             // UINT4 high plane: list position 16(e-KP) + r16
+              wgt[r8] = 4.0f * (float)(1 << 4) / (float)(1 << field_pos(r16 >> 1));
+            }
+            const bool ok = (e < KP) ? (16 * e + r16 < 2 * n16p && ch < 128) : (ch < 128);
+            chn[r8] = ok ? ch : -1;
+            qv[r8] = ok ? __half2float(qhS[hq * kD + ch]) : 0.f;
+          }
+#pragma unroll
+          for (int kg = 0; kg < NG; ++kg) {
+            uint32_t hi[4], lo[4];
+#pragma unroll
+            for (int r2 = 0; r2 < 4; ++r2) {
+              float v[2];
+#pragma unroll
+              for (int u = 0; u < 2; ++u) {
+                const int r8 = 2 * r2 + u;
+                float sc = 1.0f;
+                if (e >= KP && chn[r8] >= 0) sc = bf_lo(kmetaS[kg * 128 + chn[r8]]);
+                v[u] = qv[r8] * wgt[r8] * sc;
+              }
+              hi[r2] = pack_half2(v[0], v[1]);
+              const float2 back = __half22float2(*reinterpret_cast<const __half2*>(&hi[r2]));
+              lo[r2] = pack_half2(v[0] - back.x, v[1] - back.y);
+            }
+            *reinterpret_cast<uint4*>(gs + L::oBq + kg * kBqSBO + (row0 / 8 + c8) * 128 + hq * 16) =
+                make_uint4(hi[0], hi[1], hi[2], hi[3]);
+            *reinterpret_cast<uint4*>(gs + L::oBq + (NG + kg) * kBqSBO + (row0 / 8 + c8) * 128 + hq * 16) =
+                make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          }
+        }
+      };
+
       if (i > 0) mbar_wait(bars + Bars::o_done, (uint32_t)(i - 1) & 1u, dead, lv.status);   // A columns free again
       tc_fence_after();
       // ---- keys: row j of the A operand
@@ -358,21 +420,39 @@ attention_tc_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
           }
           const int e1 = min(E, kPass0Extra);
           for (int e = 0; e < e1; ++e) extra_step(e, tA + 64 + 8 * e);
+          // B operand, base rows: q[h][d] * s[kg][d] * 2^(4 - p(d)) as an exact fp16 pair (product, remainder);
+          // thread = (chunk of 8 channels, head), all key groups.  The scale table comes from the control warp.
+          mbar_wait(bars + Bars::ctl_ready, (uint32_t)i & 1u, dead, lv.status);
+          {
+            const int hq = j & 7, kc = j >> 3;
+            const uint4 q8 = *reinterpret_cast<const uint4*>(gs + L::oQt + j * 16);
+#pragma unroll
+            for (int kg = 0; kg < NG; ++kg) {
+              const uint4 s8 = *reinterpret_cast<const uint4*>(gs + L::oSh + (kg * kD + 8 * kc) * 2);
+              const uint4 hi = make_uint4(hmul2_u(q8.x, s8.x), hmul2_u(q8.y, s8.y), hmul2_u(q8.z, s8.z), hmul2_u(q8.w, s8.w));
+              const uint4 lo = make_uint4(hfma2_u(q8.x, s8.x, hi.x ^ 0x80008000u), hfma2_u(q8.y, s8.y, hi.y ^ 0x80008000u),
+                                          hfma2_u(q8.z, s8.z, hi.z ^ 0x80008000u), hfma2_u(q8.w, s8.w, hi.w ^ 0x80008000u));
+              *reinterpret_cast<uint4*>(gs + L::oBq + kg * kBqSBO + kc * 128 + hq * 16) = hi;
+              *reinterpret_cast<uint4*>(gs + L::oBq + (NG + kg) * kBqSBO + kc * 128 + hq * 16) = lo;
+            }
+          }
+          build_extra_rows(0, e1, 128);
         } else {
-          mbar_wait(bars + Bars::s_done, (npass - 1) & 1u, dead, lv.status);
+          mbar_wait(bars + Bars::s_done, (npass - 1) & 1u, dead, lv.status);      // A columns and B rows free again
           tc_fence_after();
           const int e0 = kPass0Extra + kPassSteps * (p - 1), e1 = min(E, e0 + kPassSteps);
           for (int e = e0; e < e1; ++e) extra_step(e, tA + 8 * (e - e0));
+          build_extra_rows(e0, e1, 0);
         }
         tc_wait_st();
         tc_fence_before();
+        fence_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(bars + Bars::a_ready);
         ++npass;
       }
 
       // ---- softmax of row j
-      mbar_wait(bars + Bars::ctl_ready, (uint32_t)i & 1u, dead, lv.status);
       mbar_wait(bars + Bars::s_done, (npass - 1) & 1u, dead, lv.status);
       tc_fence_after();
       float xv[8];
@@ -393,14 +473,30 @@ attention_tc_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
         if (lane == 0) {
           *reinterpret_cast<float4*>(mredS + quad * 8) = make_float4(bm[0], bm[1], bm[2], bm[3]);
           *reinterpret_cast<float4*>(mredS + quad * 8 + 4) = make_float4(bm[4], bm[5], bm[6], bm[7]);
+          mbar_arrive(bars + Bars::max_ready);
         }
-        bar_sync(1 + wg, 128);
+        // values while the other warps' maxima arrive: row j (= channel j) of V~^T (the key rows are consumed)
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+          uint32_t a[32];
+          expand4(*reinterpret_cast<const uint4*>(st + NG * 512 + 4096 + hh * 2048 + j * 16), a);
+          tmem_st32(tA + 32 * hh, a);
+        }
+        mbar_wait(bars + Bars::max_ready, (uint32_t)i & 1u, dead, lv.status);
         bool grow = false;
         float mn[8];
 #pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          const float4 m0 = *reinterpret_cast<const float4*>(mredS + 4 * hf), m1 = *reinterpret_cast<const float4*>(mredS + 8 + 4 * hf);
+          const float4 m2 = *reinterpret_cast<const float4*>(mredS + 16 + 4 * hf), m3 = *reinterpret_cast<const float4*>(mredS + 24 + 4 * hf);
+          mn[4 * hf + 0] = fmaxf(fmaxf(m0.x, m1.x), fmaxf(m2.x, m3.x));
+          mn[4 * hf + 1] = fmaxf(fmaxf(m0.y, m1.y), fmaxf(m2.y, m3.y));
+          mn[4 * hf + 2] = fmaxf(fmaxf(m0.z, m1.z), fmaxf(m2.z, m3.z));
+          mn[4 * hf + 3] = fmaxf(fmaxf(m0.w, m1.w), fmaxf(m2.w, m3.w));
+        }
+#pragma unroll
         for (int h = 0; h < 8; ++h) {
-          const float b = fmaxf(fmaxf(mredS[h], mredS[8 + h]), fmaxf(mredS[16 + h], mredS[24 + h]));
-          mn[h] = fmaxf(mref[h], b);
+          mn[h] = fmaxf(mref[h], mn[h]);
           grow |= mn[h] > mref[h];
         }
         if (grow) {
@@ -408,7 +504,7 @@ attention_tc_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
             float al[8];
 #pragma unroll
             for (int h = 0; h < 8; ++h) {
-              al[h] = exp2f(mref[h] - mn[h]);
+              al[h] = ex2(mref[h] - mn[h]);
               accL[h] *= al[h];
 #pragma unroll
               for (int vg = 0; vg < VG; ++vg) accZ[vg][h] *= al[h];
@@ -428,9 +524,11 @@ attention_tc_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
         float pv[8];
 #pragma unroll
         for (int h = 0; h < 8; ++h) {
-          pv[h] = exp2f(xv[h] - mref[h]);
+          pv[h] = ex2(xv[h] - mref[h]);
           accL[h] += pv[h];
         }
+        const uint32_t ph[4] = {pack_half2(pv[0], pv[1]), pack_half2(pv[2], pv[3]), pack_half2(pv[4], pv[5]),
+                                pack_half2(pv[6], pv[7])};
         const uint32_t* vmeta = reinterpret_cast<const uint32_t*>(st + NG * 512 + 8192) + j * VG;
 #pragma unroll
         for (int vg = 0; vg < VG; ++vg) {
@@ -438,18 +536,10 @@ attention_tc_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
           const float sv = bf_lo(mz), zv = bf_hi(mz);
 #pragma unroll
           for (int h = 0; h < 8; ++h) accZ[vg][h] = fmaf(pv[h], zv, accZ[vg][h]);
-          const float sp = sv * pscale;
+          const uint32_t s2 = pack_half2(sv * pscale, sv * pscale);       // exact: bf16 scale times a power of two
           *reinterpret_cast<uint4*>(gs + L::oPb + vg * 2048 + j * 16) =
-              make_uint4(pack_half2(pv[0] * sp, pv[1] * sp), pack_half2(pv[2] * sp, pv[3] * sp),
-                         pack_half2(pv[4] * sp, pv[5] * sp), pack_half2(pv[6] * sp, pv[7] * sp));
+              make_uint4(hmul2_u(ph[0], s2), hmul2_u(ph[1], s2), hmul2_u(ph[2], s2), hmul2_u(ph[3], s2));
         }
-      }
-      // ---- values: row j (= channel j) of V~^T
-#pragma unroll
-      for (int hh = 0; hh < 2; ++hh) {
-        uint32_t a[32];
-        expand4(*reinterpret_cast<const uint4*>(st + NG * 512 + 4096 + hh * 2048 + j * 16), a);
-        tmem_st32(tA + 32 * hh, a);
       }
       tc_wait_st();
       tc_fence_before();
@@ -505,23 +595,28 @@ attention_tc_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
     int cur_s = -1;
     uint32_t npass = 0;
     bool first = true;
-    const int hq = lane & 7, kcl = lane >> 3;       // B-operand builder: head column, k-chunk phase
+    // table entries are fetched two blocks before the copy that needs them, so their latency is never waited for
+    uint2 ent_refill = make_uint2(0u, 0u);
+    if (lane == 0 && kStages < nb) ent_refill = entry_of(xb + kStages);
     for (int i = 0; i < nb; ++i) {
       const long long x = xb + i;
       const int s = (int)(x / nblk);
       const int stage = i % kStages;
-      uint2 ent_refill = make_uint2(0u, 0u);        // table entry of the block that will refill this stage
-      if (lane == 0 && i + kStages < nb) ent_refill = entry_of(x + kStages);
+      uint2 ent_ahead = make_uint2(0u, 0u);         // table entry of the block that refills the next stage
+      if (lane == 0 && i + 1 + kStages < nb) ent_ahead = entry_of(x + 1 + kStages);
       if (s != cur_s) {
         // query of the new stream as fp16, heads >= g zero.  The previous block's tensor-core reads of the B
         // operand are complete (its softmax ran), and only this warp reads qh.
         cur_s = s;
         first = true;
         const int b = s / lv.Hkv, hk = s % lv.Hkv;
+        __half* qt = reinterpret_cast<__half*>(gs + L::oQt);
         for (int t = lane; t < 8 * kD; t += 32) {
           const int h = t >> 7, d = t & 127;
-          qh[t] = (h < lv.g) ? __float2half_rn(__bfloat162float(q[((size_t)b * lv.Hq + hk * lv.g + h) * kD + d]))
-                             : __float2half_rn(0.f);
+          const __half v = (h < lv.g) ? __float2half_rn(__bfloat162float(q[((size_t)b * lv.Hq + hk * lv.g + h) * kD + d]))
+                                      : __float2half_rn(0.f);
+          qh[t] = v;
+          qt[((d >> 3) * 8 + h) * 8 + (d & 7)] = v;
         }
         __syncwarp();
       }
@@ -530,10 +625,6 @@ attention_tc_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
       const uint2 ent = entS[stage];
       const int n16 = ent.y & 0xFF, n4 = (ent.y >> 8) & 0xFF;
       const int n16p = (n16 + 1) >> 1, n4w = (n4 + 15) >> 4, KP = (n16p + 7) >> 3, E = KP + n4w;
-      const bool fits = (n16p + n4w) <= 4;
-      const unsigned char* exh = fits ? st + L::kBase
-                                      : reinterpret_cast<const unsigned char*>(lv.extras) + (size_t)s * lv.extras_stride +
-                                            (size_t)ent.x * 16;
       const uint32_t* kmeta = reinterpret_cast<const uint32_t*>(st);       // [NG][128] {s, z}
 
       // key scales (times the field weight of the channel's code) and zero-points as fp16 tables
@@ -546,108 +637,41 @@ attention_tc_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
       }
       __syncwarp();
 
-      // rows of the B operand for extra k-steps [e0, e1) placed from row `row0`
-      auto build_extra_rows = [&](int e0, int e1, int row0) {
-        for (int c8 = kcl; c8 < 2 * (e1 - e0); c8 += 4) {          // chunks of 8 rows
-          const int e = e0 + (c8 >> 1), half = c8 & 1;
-          float qv[8], wgt[8];
-          int chn[8];
+      // zero-point term of the logits: zq[kg][h] = sum_d q[h][d] z[kg][d], times scale * log2(e)
+      {
+        float c[4] = {0.f, 0.f, 0.f, 0.f};
+        const int r = lane >> 2, t = lane & 3;
 #pragma unroll
-          for (int r8 = 0; r8 < 8; ++r8) {
-            const int r16 = 8 * half + r8;                          // row inside the k-step
-            int ch;
-            if (e < KP) {
-              ch = exh[2 * (8 * e) + r16];                          // promoted: list position 16e + r16
-              wgt[r8] = 0.0009765625f;
-            } else {
-              ch = exh[2 * n16p + 16 * (e - KP) + r16];             // UINT4 high plane: list position 16(e-KP) + r16
-              wgt[r8] = 4.0f * (float)(1 << 4) / (float)(1 << field_pos(r16 >> 1));
-            }
-            const bool ok = (e < KP) ? (16 * e + r16 < 2 * n16p && ch < 128) : (ch < 128);
-            chn[r8] = ok ? ch : -1;
-            qv[r8] = ok ? __half2float(qh[hq * kD + ch]) : 0.f;
+        for (int kt = 0; kt < 8; ++kt) {
+          uint32_t a0 = 0u, a2 = 0u;
+          if (r < NG) {
+            a0 = *reinterpret_cast<const uint32_t*>(zh + r * kD + 16 * kt + 2 * t);
+            a2 = *reinterpret_cast<const uint32_t*>(zh + r * kD + 16 * kt + 8 + 2 * t);
           }
-#pragma unroll
-          for (int kg = 0; kg < NG; ++kg) {
-            float v[8];
-#pragma unroll
-            for (int r8 = 0; r8 < 8; ++r8) {
-              float sc = 1.0f;
-              if (e >= KP && chn[r8] >= 0) sc = bf_lo(kmeta[kg * 128 + chn[r8]]);
-              v[r8] = qv[r8] * wgt[r8] * sc;
-            }
-            uint32_t hi[4], lo[4];
-#pragma unroll
-            for (int r2 = 0; r2 < 4; ++r2) {
-              hi[r2] = pack_half2(v[2 * r2], v[2 * r2 + 1]);
-              const float2 back = __half22float2(*reinterpret_cast<const __half2*>(&hi[r2]));
-              lo[r2] = pack_half2(v[2 * r2] - back.x, v[2 * r2 + 1] - back.y);
-            }
-            *reinterpret_cast<uint4*>(gs + L::oBq + kg * kBqSBO + (row0 / 8 + c8) * 128 + hq * 16) =
-                make_uint4(hi[0], hi[1], hi[2], hi[3]);
-            *reinterpret_cast<uint4*>(gs + L::oBq + (NG + kg) * kBqSBO + (row0 / 8 + c8) * 128 + hq * 16) =
-                make_uint4(lo[0], lo[1], lo[2], lo[3]);
-          }
+          const uint32_t b0 = *reinterpret_cast<const uint32_t*>(qh + r * kD + 16 * kt + 2 * t);
+          const uint32_t b1 = *reinterpret_cast<const uint32_t*>(qh + r * kD + 16 * kt + 8 + 2 * t);
+          mma_f16(c, a0, 0u, a2, 0u, b0, b1);
         }
-      };
+        if (r < NG) {
+          zqS[r * 8 + 2 * t] = c[0] * scale_log2e;
+          zqS[r * 8 + 2 * t + 1] = c[1] * scale_log2e;
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bars + Bars::ctl_ready);     // tables and zq of this block are in place
 
+      // ---- q . K~^T: one group of tcgen05.mma per pass, issued by one elected lane from warp-uniform operands
       const int P = 1 + (E > kPass0Extra ? (E - kPass0Extra + kPassSteps - 1) / kPassSteps : 0);
+      const uint64_t bq_desc = make_desc(bq_addr, 128, kBqSBO);
       for (int p = 0; p < P; ++p) {
-        int n_steps;
-        if (p == 0) {
-          // base rows: q[h][d] * s[kg][d] * 2^(4 - p(d)), column (kg, h)
-#pragma unroll
-          for (int kc4 = 0; kc4 < 4; ++kc4) {
-            const int kc = kcl + 4 * kc4;                             // chunk of 8 channels
-            const uint4 q8 = *reinterpret_cast<const uint4*>(qh + hq * kD + 8 * kc);
-#pragma unroll
-            for (int kg = 0; kg < NG; ++kg) {
-              // q * s has 16 significant bits: high part = the fp16 product, low part = the exact remainder
-              const uint4 s8 = *reinterpret_cast<const uint4*>(sh + kg * kD + 8 * kc);
-              const uint4 hi = make_uint4(hmul2_u(q8.x, s8.x), hmul2_u(q8.y, s8.y), hmul2_u(q8.z, s8.z), hmul2_u(q8.w, s8.w));
-              const uint4 lo = make_uint4(hfma2_u(q8.x, s8.x, hi.x ^ 0x80008000u), hfma2_u(q8.y, s8.y, hi.y ^ 0x80008000u),
-                                          hfma2_u(q8.z, s8.z, hi.z ^ 0x80008000u), hfma2_u(q8.w, s8.w, hi.w ^ 0x80008000u));
-              *reinterpret_cast<uint4*>(gs + L::oBq + kg * kBqSBO + kc * 128 + hq * 16) = hi;
-              *reinterpret_cast<uint4*>(gs + L::oBq + (NG + kg) * kBqSBO + kc * 128 + hq * 16) = lo;
-            }
-          }
-          const int e1 = min(E, kPass0Extra);
-          build_extra_rows(0, e1, 128);
-          n_steps = 8 + e1;
-          // zero-point term of the logits: zq[kg][h] = sum_d q[h][d] z[kg][d], times scale * log2(e)
-          {
-            float c[4] = {0.f, 0.f, 0.f, 0.f};
-            const int r = lane >> 2, t = lane & 3;
-#pragma unroll
-            for (int kt = 0; kt < 8; ++kt) {
-              uint32_t a0 = 0u, a2 = 0u;
-              if (r < NG) {
-                a0 = *reinterpret_cast<const uint32_t*>(zh + r * kD + 16 * kt + 2 * t);
-                a2 = *reinterpret_cast<const uint32_t*>(zh + r * kD + 16 * kt + 8 + 2 * t);
-              }
-              const uint32_t b0 = *reinterpret_cast<const uint32_t*>(qh + r * kD + 16 * kt + 2 * t);
-              const uint32_t b1 = *reinterpret_cast<const uint32_t*>(qh + r * kD + 16 * kt + 8 + 2 * t);
-              mma_f16(c, a0, 0u, a2, 0u, b0, b1);
-            }
-            if (r < NG) {
-              zqS[r * 8 + 2 * t] = c[0] * scale_log2e;
-              zqS[r * 8 + 2 * t + 1] = c[1] * scale_log2e;
-            }
-          }
-        } else {
-          mbar_wait(bars + Bars::s_done, (npass - 1) & 1u, dead, lv.status);      // B rows free again
-          const int e0 = kPass0Extra + kPassSteps * (p - 1), e1 = min(E, e0 + kPassSteps);
-          build_extra_rows(e0, e1, 0);
-          n_steps = e1 - e0;
-        }
-        fence_async_smem();
-        __syncwarp();
-        if (p == 0 && lane == 0) mbar_arrive(bars + Bars::ctl_ready);
+        const int n_steps = (p == 0) ? 8 + min(E, kPass0Extra)
+                                     : min(E, kPass0Extra + kPassSteps * p) - (kPass0Extra + kPassSteps * (p - 1));
         mbar_wait(bars + Bars::a_ready, npass & 1u, dead, lv.status);
         tc_fence_after();
-        if (lane == 0) {
-          for (int ks = 0; ks < n_steps; ++ks)
-            tc_mma(tW + kColS, tW + 8 * ks, make_desc(bq_addr + ks * 256, 128, kBqSBO), idesc1, (p > 0 || ks > 0) ? 1u : 0u);
+        if (elect_one()) {
+#pragma unroll
+          for (int ks = 0; ks < kPassSteps; ++ks)
+            if (ks < n_steps) tc_mma(tW + kColS, tW + 8 * ks, bq_desc + (uint64_t)(ks * 16), idesc1, (p > 0 || ks > 0) ? 1u : 0u);
           tc_commit(bars + Bars::s_done);
         }
         __syncwarp();
@@ -657,10 +681,11 @@ attention_tc_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
       // ---- P . V~ once the group's P rows and value rows are in place
       mbar_wait(bars + Bars::p_ready, (uint32_t)i & 1u, dead, lv.status);
       tc_fence_after();
-      if (lane == 0) {
+      if (elect_one()) {
+        const uint64_t pb_desc = make_desc(pb_addr, 128, 2048);
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)
-          tc_mma(tW + kColO, tW + 8 * ks, make_desc(pb_addr + ks * 256, 128, 2048), idesc2, (first && ks == 0) ? 0u : 1u);
+          tc_mma(tW + kColO, tW + 8 * ks, pb_desc + (uint64_t)(ks * 16), idesc2, (first && ks == 0) ? 0u : 1u);
         tc_commit(bars + Bars::o_done);
       }
       __syncwarp();
@@ -670,6 +695,7 @@ attention_tc_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
         if (lane == 0) issue(x + kStages, i + kStages, ent_refill);
         __syncwarp();
       }
+      ent_refill = ent_ahead;
     }
     // the group's last commit must have landed before tensor memory is released
     if (nb > 0) mbar_wait(bars + Bars::o_done, (uint32_t)(nb - 1) & 1u, dead, lv.status);

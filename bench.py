@@ -214,7 +214,7 @@ def run_gpu(args, w):
     n_steps = Wm + K + 4
     cfg = binding.make_config(w.n_layers, w.batch, w.n_q_heads, w.n_kv_heads, w.tokens + n_steps + 2 * w.residual_len,
                               residual_len=w.residual_len, group_size=w.group_size, tau_bf16=w.tau_bf16,
-                              tau_u4=w.tau_u4, score_bits=w.score_bits)
+                              tau_u4=w.tau_u4, score_bits=w.score_bits, block_layout=args.layout)
     cache = binding.Cache(cfg, device=dev)
     prefill(cache, w, dev)
     assert cache.status() == 0
@@ -348,7 +348,7 @@ def run_gpu(args, w):
         "tier_mix_mean": {"n16": n16, "n4": n4, "n2": 128 - n16 - n4},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal_8TBs": achieved / 8000.0, "traffic": None, "peak_source": peak_src,
-                     "kernel": "attention_mma_kernel", "kernel_us": kern_ms * 1e3, "algorithmic_bytes": alg},
+                     "kernel": "attention_tc_kernel" if args.layout == 1 else "attention_mma_kernel", "kernel_us": kern_ms * 1e3, "algorithmic_bytes": alg},
         "e2e": {"value": e2e_us, "unit": "us/step", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": n_e2e},
         "gpu_launches": int(launches),
@@ -376,6 +376,8 @@ def main():
     ap.add_argument("--layers", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layout", type=int, default=0, choices=[0, 1],
+                    help="0: fragment layout + mma.sync attention (default), 1: tile layout + tcgen05 attention")
     args = ap.parse_args()
     w = W.CONFIGS[args.config]
     over = {}

@@ -36,7 +36,7 @@ extern "C" {
 enum {
   MIXKVQ_OK = 0,
   MIXKVQ_E_INVALID_ARG = -1,          /* null pointer, bad dimension, layer out of range            */
-  MIXKVQ_E_UNSUPPORTED = -2,          /* head_dim != 128, v_bits != 2, unsupported R or G            */
+  MIXKVQ_E_UNSUPPORTED = -2,          /* head_dim != 128, v_bits != 2, unsupported R, G or layout    */
   MIXKVQ_E_ALIGNMENT = -3,            /* a device pointer is not 16-byte aligned                     */
   MIXKVQ_E_BUFFER_TOO_SMALL = -4,     /* cache memory or attention workspace smaller than required   */
   MIXKVQ_E_CAPACITY = -5,             /* append would exceed max_tokens                              */
@@ -68,7 +68,8 @@ typedef struct mixkvq_config {
   float tau_u4;                       /* tau_u4 < A_d <= tau_bf16   -> UINT4, else UINT2             */
   int32_t importance_mode;            /* 0: |q| accumulated within the current window (Section 4.2);
                                          1: cumulative over the whole history (Appendix D.2)         */
-  int32_t reserved;
+  int32_t block_layout;               /* 0: fragment layout (any R; mma.sync attention kernel), the default;
+                                         1: tile layout (R must be 128; tcgen05 attention kernel)        */
   uint64_t extras_budget_bytes;       /* per stream, for promoted channels; 0 = library default
                                          (1/8 of the bf16 size of max_tokens keys)                   */
 } mixkvq_config;

@@ -284,7 +284,7 @@ def unquantized_attention(q, K, V, scale):
 
 # --------------------------------------------------------------------------------------------
 # byte layout (written from the layout section of the design document, one element at a time)
-# fragment layout: blocks of any R other than 128
+# fragment layout (the default): blocks of any R
 # --------------------------------------------------------------------------------------------
 def base_bytes(R, G):
     return (R // G) * 512 + (R // 32) * (2048 + 128 * (D // G))
@@ -444,11 +444,10 @@ def unpack_base(buf, R, G):
 
 
 # --------------------------------------------------------------------------------------------
-# tile layout (blocks of R = 128 tokens): one thread of the attention kernel owns one token's key codes
+# tile layout (optional, blocks of R = 128 tokens): one thread of the attention kernel owns one token's key codes
 # and one channel's value codes, each a contiguous run of 2-bit fields
 # --------------------------------------------------------------------------------------------
-def uses_tile_layout(R):
-    return R == 128
+LAYOUT_FRAGMENT, LAYOUT_TILE = 0, 1
 
 
 def tile_base_bytes(G):
@@ -552,11 +551,12 @@ def table_entry(extras_off16, n16, n4):
     return int(extras_off16).to_bytes(4, "little") + bytes([n16, n4, 0, 0])
 
 
-def pack_stream(st: OracleStream):
+def pack_stream(st: OracleStream, layout=LAYOUT_FRAGMENT):
     """All bytes the stream would hold in device memory, by region."""
     base, table, extras = [], [], []
     used16 = 0
-    tile = uses_tile_layout(st.R)
+    tile = layout == LAYOUT_TILE
+    assert not tile or st.R == 128
     for blk in st.blocks:
         if tile:
             base.append(pack_base_tile(blk, st.G))

@@ -42,6 +42,8 @@ int check_config(const mixkvq_config* c) {
     return MIXKVQ_E_UNSUPPORTED;
   if (c->score_bits != 2 && c->score_bits != 4) return MIXKVQ_E_UNSUPPORTED;
   if (c->importance_mode != 0 && c->importance_mode != 1) return MIXKVQ_E_INVALID_ARG;
+  if (c->block_layout != 0 && c->block_layout != 1) return MIXKVQ_E_INVALID_ARG;
+  if (c->block_layout == 1 && c->residual_len != 128) return MIXKVQ_E_UNSUPPORTED;
   return MIXKVQ_OK;
 }
 
@@ -57,7 +59,7 @@ uint64_t plan(const mixkvq_config* c, mixkvq_cache* h) {
   h->VG = kD / h->G;
   h->max_blocks = (c->max_tokens + h->R - 1) / h->R;
   h->unit_bytes = 2048u + 128u * h->VG;
-  h->tile = (h->R == 128) ? 1 : 0;
+  h->tile = (c->block_layout == 1) ? 1 : 0;
   h->base_bytes = h->tile ? (uint32_t)h->NG * 512u + 8192u + 512u * (uint32_t)h->VG
                           : (uint32_t)h->NG * 512u + (uint32_t)h->U * h->unit_bytes;
   h->extras_budget = c->extras_budget_bytes ? align_up(c->extras_budget_bytes, 16)

@@ -25,7 +25,7 @@ struct LayerView {
   int R, G, U, NG, VG;        // residual length, group size, units/block, key groups/block, value groups/token
   int max_blocks;
   int n_blocks, r;            // current fill (same for all streams)
-  int tile;                   // 1: tile layout (R == 128), 0: fragment layout
+  int tile;                   // 1: tile layout (R == 128 only), 0: fragment layout
   uint32_t base_bytes, unit_bytes;
   uint64_t extras_budget;     // bytes per stream
   // method parameters

@@ -10,11 +10,11 @@ def f32(t):
     return t.to(torch.float32).cpu().numpy()
 
 
-def make_cache(binding, w, max_tokens=None, importance_mode=0, extras_budget_bytes=0):
+def make_cache(binding, w, max_tokens=None, importance_mode=0, extras_budget_bytes=0, layout=0):
     cfg = binding.make_config(w.n_layers, w.batch, w.n_q_heads, w.n_kv_heads, max_tokens or (w.tokens + 256),
                               residual_len=w.residual_len, group_size=w.group_size, tau_bf16=w.tau_bf16,
                               tau_u4=w.tau_u4, score_bits=w.score_bits, importance_mode=importance_mode,
-                              extras_budget_bytes=extras_budget_bytes)
+                              extras_budget_bytes=extras_budget_bytes, block_layout=layout)
     return binding.Cache(cfg)
 
 
@@ -38,7 +38,7 @@ def compare_regions(cache, layer, w, oracle):
     """Byte equality of every region of every oracle stream with the device cache."""
     for (b, hk), st in oracle.items():
         got = cache.stream_regions(layer, b * w.n_kv_heads + hk)
-        want = O.pack_stream(st)
+        want = O.pack_stream(st, layout=cache.cfg.block_layout)
         for key in ("table", "base", "extras", "state", "resK"):
             assert got[key] == want[key], f"stream {(b, hk)} region {key} differs"
         R = w.residual_len

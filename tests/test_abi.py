@@ -45,6 +45,8 @@ def test_cache_bytes_and_argument_validation(binding):
         c = binding.make_config(2, 2, 8, 2, 1024)
         setattr(c, field, bad)
         assert lib.mixkvq_cache_bytes(C.byref(c), None, None) == code, field
+    c = binding.make_config(1, 1, 1, 1, 256, residual_len=64, group_size=32, block_layout=1)
+    assert lib.mixkvq_cache_bytes(C.byref(c), None, None) == -2          # the tile layout needs R = 128
     c = binding.make_config(1, 1, 1, 1, 256, residual_len=64, group_size=128)
     assert lib.mixkvq_cache_bytes(C.byref(c), None, None) == -2          # R must be a multiple of G
     assert lib.mixkvq_cache_bytes(None, None, None) == -1

@@ -65,12 +65,15 @@ def test_select_channels_of_current_window(binding):
 GEOMS = [(128, 32), (128, 128), (128, 64), (64, 32), (96, 32), (256, 64), (32, 32)]
 
 
-@pytest.mark.parametrize("R,G", GEOMS)
+TILE_GEOMS = [(128, 32, 1), (128, 64, 1), (128, 128, 1)]      # the optional tile layout exists for R = 128 only
+
+
+@pytest.mark.parametrize("R,G,layout", [(r, g, 0) for r, g in GEOMS] + TILE_GEOMS)
 @pytest.mark.parametrize("preset", ["P24", "P27", "P4BASE"])
-def test_packed_cache_is_byte_exact(binding, R, G, preset):
+def test_packed_cache_is_byte_exact(binding, R, G, layout, preset):
     w = small(tokens=2 * R + 41, residual_len=R, group_size=G, **getattr(W, preset))
     k, v, q = W.tokens(w, 0, 0, w.tokens)
-    cache = U.make_cache(binding, w)
+    cache = U.make_cache(binding, w, layout=layout)
     cache.quantize_append(0, k.cuda(), v.cuda(), q.cuda())
     assert cache.status() == 0
     orc = U.oracle_streams(w, 0, k, v, q)
@@ -84,12 +87,13 @@ def test_packed_cache_is_byte_exact(binding, R, G, preset):
         assert all(not (b.tiers == O.TIER_U2).any() for st in orc.values() for b in st.blocks)
 
 
-def test_tiny_config_full_parity(binding):
+@pytest.mark.parametrize("layout", [0, 1])
+def test_tiny_config_full_parity(binding, layout):
     # configuration 1: 1 layer, batch 1, 1 KV head, 1 query head, 1024 cached tokens, then one decode step
     w = W.CONFIGS["tiny"]
     w = dataclasses.replace(w, **W.P27)
     k, v, q = W.tokens(w, 0, 0, 1025)
-    cache = U.make_cache(binding, w)
+    cache = U.make_cache(binding, w, layout=layout)
     cache.quantize_append(0, k[:, :, :1024].cuda(), v[:, :, :1024].cuda(), q[:, :, :1024].cuda())
     orc = U.oracle_streams(w, 0, k[:, :, :1024], v[:, :, :1024], q[:, :, :1024])
     U.compare_regions(cache, 0, w, orc)
@@ -142,16 +146,16 @@ def test_cumulative_importance_mode(binding):
 
 
 # ------------------------------------------------------------------------------------------- attention
-@pytest.mark.parametrize("kind", [0, 1])
+@pytest.mark.parametrize("kind,layout", [(0, 0), (1, 0), (0, 1), (1, 1)])
 @pytest.mark.parametrize("name,tokens,preset", [
     ("qwen7b", 1, "P24"), ("qwen7b", 31, "P24"), ("qwen7b", 128, "P24"), ("qwen7b", 129, "P24"),
     ("qwen7b", 1153, "P27"), ("llama8b", 700, "P27"), ("llama8b", 700, "P4BASE"), ("qwen32b", 1000, "P24"),
     ("tiny", 2500, "P27"),
 ])
-def test_attention_matches_oracle(binding, kind, name, tokens, preset):
+def test_attention_matches_oracle(binding, kind, layout, name, tokens, preset):
     w = small(name, batch=2 if name != "tiny" else 1, tokens=tokens, **getattr(W, preset))
     k, v, q = W.tokens(w, 0, 0, tokens)
-    cache = U.make_cache(binding, w)
+    cache = U.make_cache(binding, w, layout=layout)
     cache.quantize_append(0, k.cuda(), v.cuda(), q.cuda())
     cache.set_attention_kernel(kind)
     orc = U.oracle_streams(w, 0, k, v, q)
@@ -164,11 +168,12 @@ def test_attention_matches_oracle(binding, kind, name, tokens, preset):
 
 
 @pytest.mark.parametrize("kind", [0, 1])
-@pytest.mark.parametrize("R,G", [(128, 128), (64, 32), (256, 64), (32, 32), (96, 32)])
-def test_attention_other_geometries(binding, kind, R, G):
+@pytest.mark.parametrize("R,G,layout", [(128, 128, 0), (64, 32, 0), (256, 64, 0), (32, 32, 0), (96, 32, 0), (128, 128, 1),
+                                        (128, 64, 1)])
+def test_attention_other_geometries(binding, kind, R, G, layout):
     w = small("llama8b", batch=1, tokens=3 * R + 17, residual_len=R, group_size=G, **W.P27)
     k, v, q = W.tokens(w, 0, 0, w.tokens)
-    cache = U.make_cache(binding, w)
+    cache = U.make_cache(binding, w, layout=layout)
     cache.quantize_append(0, k.cuda(), v.cuda(), q.cuda())
     cache.set_attention_kernel(kind)
     orc = U.oracle_streams(w, 0, k, v, q)

@@ -202,7 +202,7 @@ def test_stream_regions(rng):
     k, v, q = _tokens(rng, 3 * 128 + 5, 2)
     st = O.OracleStream(g=2, tau_bf16=6.0, tau_u4=3.0)
     st.append_many(k, v, q)
-    p = O.pack_stream(st)
+    p = O.pack_stream(st, layout=O.LAYOUT_TILE)
     assert len(p["base"]) == 3 * 12288 and len(p["table"]) == 24
     off = 0
     for i, blk in enumerate(st.blocks):

@@ -30,17 +30,17 @@ def binding():
     return b
 
 
-def _filled_cache(binding, name, batch, tokens, preset):
+def _filled_cache(binding, name, batch, tokens, preset, layout=0):
     w = W.small(W.CONFIGS[name], n_layers=1, batch=batch, tokens=tokens, **preset)
     k, v, q = W.tokens(w, 0, 0, tokens)
-    cache = U.make_cache(binding, w)
+    cache = U.make_cache(binding, w, layout=layout)
     cache.quantize_append(0, k.cuda(), v.cuda(), q.cuda())
     return w, cache
 
 
 def test_noalloc_entry_matches_workspace_entry_on_two_calls_in_a_row(binding):
     w1, c1 = _filled_cache(binding, "qwen7b", 3, 5 * 128 + 77, W.P27)
-    w2, c2 = _filled_cache(binding, "llama8b", 2, 128 + 9, W.P24)
+    w2, c2 = _filled_cache(binding, "llama8b", 2, 128 + 9, W.P24, layout=1)
     for step, (w, cache) in enumerate([(w1, c1), (w2, c2)]):
         qd = W.decode_query(w, 0, step).cuda()
         want = cache.decode_attention(0, qd, W.softmax_scale())

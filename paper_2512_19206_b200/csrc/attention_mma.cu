@@ -24,13 +24,13 @@ cudaError_t launch_combine(const float* ws, float* out, int g, int Hkv, int Hq, 
 namespace {
 
 constexpr int kWarps = 4;
-constexpr int kStages = 4;
+constexpr int kStages = 3;
 constexpr int kStageBytes = 3072;            // unit (<= 2560 B) followed by one key-meta group (512 B)
 constexpr int kKeyMetaOff = 2560;
 constexpr int kPrepBytes = 1280;             // kprep 512 | zprep 256 | svp 256 | zvp 256
 constexpr int kSharedTail = 128 + 2048 + 2048 + 128 + 128 + 4096;
 constexpr int kSmemBytes = kWarps * (kStages * kStageBytes + kPrepBytes) + kSharedTail;
-constexpr int kCtasPerSm = 3;
+constexpr int kCtasPerSm = 4;
 constexpr uint32_t kSpinLimit = 1u << 22;    // bounded wait on a staged copy
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -89,6 +89,12 @@ __device__ __forceinline__ uint32_t hmul2_u(uint32_t a, uint32_t b) {
   uint32_t d;
   asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
   return d;
+}
+// 2^x by the special-function unit alone (no range fix-up): inputs here are <= 0 or -inf
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
 __device__ __forceinline__ uint32_t pack_half2(float lo, float hi) {
   __half2 h = __floats2half2_rn(lo, hi);
@@ -439,8 +445,8 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
       uint32_t Pt[2][2];    // P^T B fragments: [k-step][tokens 2t.. / 2t+8..], head r
 #pragma unroll
       for (int mt = 0; mt < 2; ++mt) {
-        const uint32_t plo = pack_half2(exp2f(xs[mt][0] - m0), exp2f(xs[mt][1] - m1));   // token r
-        const uint32_t phi = pack_half2(exp2f(xs[mt][2] - m0), exp2f(xs[mt][3] - m1));   // token r + 8
+        const uint32_t plo = pack_half2(ex2_approx(xs[mt][0] - m0), ex2_approx(xs[mt][1] - m1));   // token r
+        const uint32_t phi = pack_half2(ex2_approx(xs[mt][2] - m0), ex2_approx(xs[mt][3] - m1));   // token r + 8
         Pt[mt][0] = movmatrix_trans(plo);
         Pt[mt][1] = movmatrix_trans(phi);
       }
@@ -650,13 +656,21 @@ cudaError_t launch_g(const LayerView& lv, const void* q, float scale, float* ws,
 
 }  // namespace
 
+template <int G>
+static cudaError_t setup_g() {
+  cudaError_t e = cudaFuncSetAttribute(attention_mma_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  if (e != cudaSuccess) return e;
+  // kCtasPerSm CTAs only fit with the largest shared-memory carve-out; ask for it explicitly
+  return cudaFuncSetAttribute(attention_mma_kernel<G>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                              (int)cudaSharedmemCarveoutMaxShared);
+}
+
 cudaError_t attention_mma_setup() {
-  cudaError_t e;
-  e = cudaFuncSetAttribute(attention_mma_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  cudaError_t e = setup_g<32>();
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(attention_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  e = setup_g<64>();
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(attention_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  return setup_g<128>();
 }
 
 // Number of CTAs the split kernel runs for this layer state (also the number of partial-slot owners).

@@ -26,6 +26,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 from paper_2512_19206_b200 import workloads as W  # noqa: E402
+from paper_2512_19206_b200.replicas import dist_env, max_over_ranks, job_tokens_per_s  # noqa: E402
 
 METRIC = "decode-attn us/step (all layers) over mixed-precision KV"
 PREFILL_CHUNK = 4096
@@ -37,13 +38,6 @@ def measured_peaks():
         d = json.load(open(p))
         return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
     return 6650.0, "fallback (6.65 TB/s, no MEASURED_PEAKS.json)"
-
-
-def dist_env():
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    return rank, world, local
 
 
 # ---------------------------------------------------------------------------------------------- CPU oracle leg
@@ -184,6 +178,21 @@ def tier_mix(cache, w):
     return n16 / nb, n4 / nb
 
 
+def measured_traffic(kernel, source_file, group_size, tokens_packed, streams):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu capture (profiles/dram_traffic.json),
+    scaled by the packed tokens this launch streams; None when there is no capture for this kernel and group size
+    or the kernel's source changed after the counters were taken."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if not os.path.exists(path):
+        return None
+    ent = json.load(open(path)).get(f"{kernel}:G{group_size}")
+    src = os.path.join(ROOT, "paper_2512_19206_b200", "csrc", source_file)
+    if not ent or hashlib.sha256(open(src, "rb").read()).hexdigest() != ent["source_sha256"]:
+        return None
+    return ent["dram_bytes_per_token_per_kv_head"] * tokens_packed * streams
+
+
 def algorithmic_bytes_per_layer(w, n16, n4, r, tokens_packed, n_partials):
     """Bytes the method must move for one decode-attention launch (one layer): packed keys and values with
     their scales/zeros, promoted channels, residual window, q, o and the split partials."""
@@ -214,7 +223,8 @@ def run_gpu(args, w):
     n_steps = Wm + K + 4
     cfg = binding.make_config(w.n_layers, w.batch, w.n_q_heads, w.n_kv_heads, w.tokens + n_steps + 2 * w.residual_len,
                               residual_len=w.residual_len, group_size=w.group_size, tau_bf16=w.tau_bf16,
-                              tau_u4=w.tau_u4, score_bits=w.score_bits, block_layout=args.layout)
+                              tau_u4=w.tau_u4, score_bits=w.score_bits, block_layout=args.layout,
+                              extras_budget_bytes=((w.tokens + n_steps) // w.residual_len + 3) * 8192 if w.score_bits == 4 else 0)
     cache = binding.Cache(cfg, device=dev)
     prefill(cache, w, dev)
     assert cache.status() == 0
@@ -321,10 +331,7 @@ def run_gpu(args, w):
     status = cache.status()
 
     us = ms * 1e3 / K
-    if world > 1:
-        t = torch.tensor([us, e2e_us, kern_ms, graph_us], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        us, e2e_us, kern_ms, graph_us = [float(x) for x in t]
+    us, e2e_us, kern_ms, graph_us = max_over_ranks([us, e2e_us, kern_ms, graph_us], device=dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -340,14 +347,19 @@ def run_gpu(args, w):
     line = {
         "metric": METRIC, "value": us, "unit": "us/step", "n_gpus": world, "steps": K, "warmup": Wm,
         "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
-        "dtype": "u2/u4 codes + bf16, fp16 tensor-core tiles, fp32 accumulate", "data": "synthetic",
+        "dtype": "f16", "data": "synthetic",
+        "arithmetic": "2/4-bit codes and bf16 metadata expanded to fp16 tensor-core operands, fp32 accumulate and softmax",
         "config": workload_config(w),
-        "tokens_per_s": world * w.batch / (us * 1e-6),
+        "tokens_per_s": job_tokens_per_s(w.batch, world, us),
         "attention_graph_us_per_step": graph_us,
         "flushes_in_timed_region": flushes,
         "tier_mix_mean": {"n16": n16, "n4": n4, "n2": 128 - n16 - n4},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "frac_of_nominal_8TBs": achieved / 8000.0, "traffic": None, "peak_source": peak_src,
+                     "frac_of_nominal_8TBs": achieved / 8000.0,
+                     "traffic": measured_traffic(*(("attention_tc_kernel", "attention_tc.cu") if args.layout == 1 else
+                                                   ("attention_mma_kernel", "attention_mma.cu")), w.group_size,
+                                                 tokens_packed, w.batch * w.n_kv_heads),
+                     "peak_source": peak_src,
                      "kernel": "attention_tc_kernel" if args.layout == 1 else "attention_mma_kernel", "kernel_us": kern_ms * 1e3, "algorithmic_bytes": alg},
         "e2e": {"value": e2e_us, "unit": "us/step", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": n_e2e},
@@ -376,6 +388,8 @@ def main():
     ap.add_argument("--layers", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--preset", default=None, choices=["P24", "P27", "P4BASE"],
+                    help="threshold preset: two tiers (default), three tiers, or 4-bit base precision")
     ap.add_argument("--layout", type=int, default=0, choices=[0, 1],
                     help="0: fragment layout + mma.sync attention (default), 1: tile layout + tcgen05 attention")
     args = ap.parse_args()
@@ -387,6 +401,8 @@ def main():
         over["tokens"] = args.tokens
     if args.layers:
         over["n_layers"] = args.layers
+    if args.preset:
+        over.update(getattr(W, args.preset))
     if over:
         w = W.small(w, **over)
     if args.impl == "reference":

@@ -133,7 +133,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
   float* oS = lS + 32;                                          // [8][128]
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < kWarps * kStages; ++i) mbar_init(smem_u32(&bars[i]), 1);
+    for (int i = 0; i < kWarps * kStages + kWarps; ++i) mbar_init(smem_u32(&bars[i]), 1);   // rings + one per warp for the residual window
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -144,6 +144,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
   const long long total = (long long)Us * S;
   const long long cb = split_begin(total, gridDim.x, blockIdx.x), ce = split_begin(total, gridDim.x, blockIdx.x + 1);
 
+  uint32_t res_phase = 0;         // phase of this warp's residual-staging barrier
   uint32_t ring_count = 0;        // packed units this warp has consumed so far (ring position)
   uint32_t ring_issued = 0;       // packed units this warp has issued so far
   bool gave_up = false;
@@ -507,8 +508,24 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
       if (lane == 0) atomicOr(lv.status, (uint32_t)MIXKVQ_DEV_COPY_TIMEOUT);
     }
 
-    // ---- residual (unquantized) tokens of this warp's range: bf16 tiles from global memory
-    for (int x = max(wb, packed_units); x < we; ++x) {
+    // ---- residual (unquantized) tokens of this warp's range: bf16 rows staged through the (now idle) ring.
+    // Keys: 32 token rows of 256 B, one bulk copy per lane, rows 272 B apart (conflict-free fragment loads).
+    // Values: 128 channel rows of 64 B (tokens j0..j0+31), four bulk copies per lane, rows 64 B apart.
+    for (int x = max(wb, packed_units); x < we && !gave_up; ++x) {
+      const uint32_t rbar = smem_u32(&bars[kWarps * kStages + warp]);
+      {
+        const int j0s = (x - packed_units) * 32, nv = min(32, lv.r - j0s);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        if (lane == 0) mbar_expect_tx(rbar, (uint32_t)nv * 256u);
+        __syncwarp();
+        if (lane < nv) bulk_g2s(smem_u32(ring + lane * 272), resk + (size_t)(j0s + lane) * kD, 256u, rbar);
+        if (!mbar_wait_bounded(rbar, res_phase)) {
+          gave_up = true;
+          if (lane == 0) atomicOr(lv.status, (uint32_t)MIXKVQ_DEV_COPY_TIMEOUT);
+          break;
+        }
+        res_phase ^= 1u;
+      }
       if (!o_true_scale) {
 #pragma unroll
         for (int ct = 0; ct < 8; ++ct)
@@ -525,8 +542,8 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt) {
           const int ta = j0 + mt * 16 + r, tb = ta + 8;
-          const uint32_t* ka = reinterpret_cast<const uint32_t*>(resk + (size_t)ta * kD + 16 * kt + 2 * t);
-          const uint32_t* kb = reinterpret_cast<const uint32_t*>(resk + (size_t)tb * kD + 16 * kt + 2 * t);
+          const uint32_t* ka = reinterpret_cast<const uint32_t*>(ring + (mt * 16 + r) * 272 + (16 * kt + 2 * t) * 2);
+          const uint32_t* kb = reinterpret_cast<const uint32_t*>(ring + (mt * 16 + 8 + r) * 272 + (16 * kt + 2 * t) * 2);
           const uint32_t a0 = ta < rt ? ka[0] : 0u, a1 = tb < rt ? kb[0] : 0u;
           const uint32_t a2 = ta < rt ? ka[4] : 0u, a3 = tb < rt ? kb[4] : 0u;
           mma_bf16(Sx[mt], a0, a1, a2, a3, b0, b1);
@@ -568,6 +585,22 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
       const uint32_t ones = (r == 4) ? 0x3C003C00u : 0u;
 #pragma unroll
       for (int ks = 0; ks < 2; ++ks) mma_f16(Zc, ones, 0u, ones, 0u, Pt[ks][0], Pt[ks][1]);
+      // the key rows are consumed: stage the value rows of these 32 tokens over them
+      __syncwarp();
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      if (lane == 0) mbar_expect_tx(rbar, 128u * 64u);
+      __syncwarp();
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int c = lane + 32 * i;
+        bulk_g2s(smem_u32(ring + c * 64), resv + (size_t)c * lv.R + j0, 64u, rbar);
+      }
+      if (!mbar_wait_bounded(rbar, res_phase)) {
+        gave_up = true;
+        if (lane == 0) atomicOr(lv.status, (uint32_t)MIXKVQ_DEV_COPY_TIMEOUT);
+        break;
+      }
+      res_phase ^= 1u;
 #pragma unroll
       for (int ct = 0; ct < 8; ++ct) {
         const int c0 = 16 * ct + r, c1 = c0 + 8;
@@ -576,7 +609,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
           const int ja = j0 + 16 * ks + 2 * t, jb = ja + 8;
           auto load_pair = [&](int c, int j) -> uint32_t {
             if (j >= rt) return 0u;
-            uint32_t w = *reinterpret_cast<const uint32_t*>(resv + (size_t)c * lv.R + j);
+            uint32_t w = *reinterpret_cast<const uint32_t*>(ring + c * 64 + (j - j0) * 2);
             if (j + 1 >= rt) w &= 0xFFFFu;
             return bf16x2_to_f16x2(w);
           };

@@ -225,3 +225,48 @@ def test_extras_arena_exhaustion_sets_status(binding):
     assert cache.status() & binding.DEV_EXTRAS_FULL
     cache.reset()
     assert cache.status() == 0 and cache.describe(0).n_blocks == 0
+
+
+# ------------------------------------------------------------------------------- degenerate cases of the method
+@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("kind", [0, 1])
+def test_all_channels_promoted_is_unquantized_key_attention(binding, kind, layout):
+    # every key channel in the BF16 tier: the logits are those of the raw bf16 keys (library attention on the
+    # oracle's dequantized values), and the promoted-channel store carries all 128 channels of every block
+    w = small("llama8b", batch=1, tokens=2 * 128 + 30, tau_bf16=-1.0, tau_u4=-1.0)
+    k, v, q = W.tokens(w, 0, 0, w.tokens)
+    cache = U.make_cache(binding, w, extras_budget_bytes=4 * 40000, layout=layout)
+    cache.quantize_append(0, k.cuda(), v.cuda(), q.cuda())
+    cache.set_attention_kernel(kind)
+    orc = U.oracle_streams(w, 0, k, v, q)
+    U.compare_regions(cache, 0, w, orc)
+    qd = W.decode_query(w, 0, 0)
+    out = cache.decode_attention(0, qd.cuda(), W.softmax_scale()).cpu()
+    assert cache.status() == 0
+    for (b, hk), st in orc.items():
+        assert all((blk.tiers == O.TIER_BF16).all() for blk in st.blocks)
+        ref = torch.nn.functional.scaled_dot_product_attention(
+            qd[b, hk * w.g:(hk + 1) * w.g].double()[None], k[b, hk].double()[None], torch.from_numpy(st.values())[None],
+            scale=W.softmax_scale())[0]
+        assert float((out[b, hk * w.g:(hk + 1) * w.g].double() - ref).abs().max()) <= ATTN_TOL
+
+
+@pytest.mark.parametrize("layout", [0, 1])
+def test_zero_keys_and_constant_groups(binding, layout):
+    # all keys zero: every scale is 0 (codes 0, dequantized exactly) and the output is the mean of the values;
+    # values constant inside each group of channels: their scale is 0 and the zero-point carries them exactly
+    w = small("qwen7b", batch=1, tokens=3 * 128 + 5, **W.P27)
+    k, v, q = W.tokens(w, 0, 0, w.tokens)
+    k = torch.zeros_like(k)
+    v = v[..., ::32].repeat_interleave(32, dim=-1).contiguous()
+    cache = U.make_cache(binding, w, layout=layout)
+    cache.quantize_append(0, k.cuda(), v.cuda(), q.cuda())
+    orc = U.oracle_streams(w, 0, k, v, q)
+    U.compare_regions(cache, 0, w, orc)
+    qd = W.decode_query(w, 0, 0)
+    out = cache.decode_attention(0, qd.cuda(), W.softmax_scale()).cpu()
+    mean_v = v.float().mean(dim=2)                                           # [B, Hkv, 128]
+    for hk in range(w.n_kv_heads):
+        got = out[0, hk * w.g:(hk + 1) * w.g]
+        assert float((got - mean_v[0, hk][None]).abs().max()) <= 1e-4
+    assert cache.status() == 0

@@ -160,11 +160,14 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
     {
       const int b = s / lv.Hkv, hk = s % lv.Hkv;
       __syncthreads();
-      for (int i = threadIdx.x; i < 8 * kD; i += kWarps * 32) {
-        const int h = i >> 7, d = i & 127;
-        const __nv_bfloat16 v = (h < g) ? q[((size_t)b * lv.Hq + hk * g + h) * kD + d] : __float2bfloat16(0.f);
-        qb16[i] = *reinterpret_cast<const uint16_t*>(&v);
-        qf16[i] = __float2half_rn(__bfloat162float(v));
+      {
+        // one 16-byte load per thread: head h, channels 8c .. 8c+7 (heads >= g are zero rows)
+        const int h = threadIdx.x >> 4, c = threadIdx.x & 15;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (h < g) v = *reinterpret_cast<const uint4*>(q + ((size_t)b * lv.Hq + hk * g + h) * kD + 8 * c);
+        *reinterpret_cast<uint4*>(&qb16[h * kD + 8 * c]) = v;
+        *reinterpret_cast<uint4*>(&qf16[h * kD + 8 * c]) =
+            make_uint4(bf16x2_to_f16x2(v.x), bf16x2_to_f16x2(v.y), bf16x2_to_f16x2(v.z), bf16x2_to_f16x2(v.w));
       }
       __syncthreads();
     }

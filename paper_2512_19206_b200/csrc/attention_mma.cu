@@ -156,6 +156,44 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
     seg += ue - ub;
     const int wb = ub + (int)split_begin(ue - ub, kWarps, warp), we = ub + (int)split_begin(ue - ub, kWarps, warp + 1);
 
+    const char* base = lv.base + (size_t)s * lv.base_stride;
+    const char* extras = lv.extras + (size_t)s * lv.extras_stride;
+    const uint2* table = reinterpret_cast<const uint2*>(lv.table + (size_t)s * lv.table_stride);
+    const uint16_t* resk = reinterpret_cast<const uint16_t*>(lv.resk + (size_t)s * lv.resk_stride);
+    const uint16_t* resv = reinterpret_cast<const uint16_t*>(lv.resv + (size_t)s * lv.resv_stride);
+
+    // ---- the first copies of this segment go out before anything else: they do not depend on the query
+    const int n_pack = max(0, min(we, packed_units) - wb);
+    int issued = 0;
+    auto issue = [&](int x, bool first) {
+      // lane 0 only: stage unit x of this stream
+      const int bi = x / U, u = x - bi * U;
+      const char* blk = base + (size_t)bi * lv.base_bytes;
+      const uint32_t stage = ring_issued % kStages;
+      const uint32_t bar = smem_u32(&bars[warp * kStages + stage]);
+      const uint32_t dst = smem_u32(ring + stage * kStageBytes);
+      const bool meta = first || ((u * 32) % G == 0);
+      mbar_expect_tx(bar, lv.unit_bytes + (meta ? 512u : 0u));
+      bulk_g2s(dst, blk + lv.NG * 512 + (size_t)u * lv.unit_bytes, lv.unit_bytes, bar);
+      if (meta) bulk_g2s(dst + kKeyMetaOff, blk + ((u * 32) / G) * 512, 512u, bar);
+    };
+    for (; !gave_up && issued < min(n_pack, kStages); ++issued) {
+      if (lane == 0) issue(wb + issued, issued == 0);
+      ++ring_issued;
+    }
+
+    // the first block's table entry is requested now as well, long before the first unit arrives
+    int cur_bi = -1, pf_bi = -1;
+    uint2 entry = make_uint2(0, 0), pf_entry = make_uint2(0, 0);
+    if (n_pack > 0) {
+      pf_bi = wb / U;
+      pf_entry = table[pf_bi];
+    }
+    int n16 = 0, n4 = 0, n16p = 0;
+    const char* ex = nullptr;
+    uint32_t ex_hdr = 0, ex_unit = 0;
+
+
     // ---- query of this stream: bf16 and fp16 tables for the gathered paths
     {
       const int b = s / lv.Hkv, hk = s % lv.Hkv;
@@ -183,12 +221,6 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
       }
     }
 
-    const char* base = lv.base + (size_t)s * lv.base_stride;
-    const char* extras = lv.extras + (size_t)s * lv.extras_stride;
-    const uint2* table = reinterpret_cast<const uint2*>(lv.table + (size_t)s * lv.table_stride);
-    const uint16_t* resk = reinterpret_cast<const uint16_t*>(lv.resk + (size_t)s * lv.resk_stride);
-    const uint16_t* resv = reinterpret_cast<const uint16_t*>(lv.resv + (size_t)s * lv.resv_stride);
-
     float O[8][4];       // O^T tiles: [channel tile] x (channels r, r+8) x (heads 2t, 2t+1); packed part scaled 2^-20
     float Zc[4] = {0.f, 0.f, 0.f, 0.f};   // rows 0..VG-1: sum p * z_v per value group; row 4: sum p
     float zc[4] = {0.f, 0.f, 0.f, 0.f};   // key zero-point term of the current key group
@@ -198,31 +230,6 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
 #pragma unroll
       for (int i = 0; i < 4; ++i) O[ct][i] = 0.f;
     bool o_true_scale = false;
-
-    const int n_pack = max(0, min(we, packed_units) - wb);
-    int issued = 0;
-    auto issue = [&](int x, bool first) {
-      // lane 0 only: stage unit x of this stream
-      const int bi = x / U, u = x - bi * U;
-      const char* blk = base + (size_t)bi * lv.base_bytes;
-      const uint32_t stage = ring_issued % kStages;
-      const uint32_t bar = smem_u32(&bars[warp * kStages + stage]);
-      const uint32_t dst = smem_u32(ring + stage * kStageBytes);
-      const bool meta = first || ((u * 32) % G == 0);
-      mbar_expect_tx(bar, lv.unit_bytes + (meta ? 512u : 0u));
-      bulk_g2s(dst, blk + lv.NG * 512 + (size_t)u * lv.unit_bytes, lv.unit_bytes, bar);
-      if (meta) bulk_g2s(dst + kKeyMetaOff, blk + ((u * 32) / G) * 512, 512u, bar);
-    };
-    for (; !gave_up && issued < min(n_pack, kStages); ++issued) {
-      if (lane == 0) issue(wb + issued, issued == 0);
-      ++ring_issued;
-    }
-
-    int cur_bi = -1, pf_bi = -1;
-    uint2 entry = make_uint2(0, 0), pf_entry = make_uint2(0, 0);
-    int n16 = 0, n4 = 0, n16p = 0;
-    const char* ex = nullptr;
-    uint32_t ex_hdr = 0, ex_unit = 0;
 
     for (int i = 0; i < n_pack && !gave_up; ++i) {
       const int x = wb + i;

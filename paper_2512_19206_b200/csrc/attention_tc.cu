@@ -527,8 +527,6 @@ attention_tc_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
           pv[h] = ex2(xv[h] - mref[h]);
           accL[h] += pv[h];
         }
-        const uint32_t ph[4] = {pack_half2(pv[0], pv[1]), pack_half2(pv[2], pv[3]), pack_half2(pv[4], pv[5]),
-                                pack_half2(pv[6], pv[7])};
         const uint32_t* vmeta = reinterpret_cast<const uint32_t*>(st + NG * 512 + 8192) + j * VG;
 #pragma unroll
         for (int vg = 0; vg < VG; ++vg) {
@@ -536,9 +534,10 @@ attention_tc_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
           const float sv = bf_lo(mz), zv = bf_hi(mz);
 #pragma unroll
           for (int h = 0; h < 8; ++h) accZ[vg][h] = fmaf(pv[h], zv, accZ[vg][h]);
-          const uint32_t s2 = pack_half2(sv * pscale, sv * pscale);       // exact: bf16 scale times a power of two
+          const float sp = sv * pscale;                                    // products in fp32, rounded to fp16 once
           *reinterpret_cast<uint4*>(gs + L::oPb + vg * 2048 + j * 16) =
-              make_uint4(hmul2_u(ph[0], s2), hmul2_u(ph[1], s2), hmul2_u(ph[2], s2), hmul2_u(ph[3], s2));
+              make_uint4(pack_half2(pv[0] * sp, pv[1] * sp), pack_half2(pv[2] * sp, pv[3] * sp),
+                         pack_half2(pv[4] * sp, pv[5] * sp), pack_half2(pv[6] * sp, pv[7] * sp));
         }
       }
       tc_wait_st();

@@ -154,14 +154,23 @@ class ClockSampler:
 
 
 def prefill(cache, w, dev):
+    """Fills every layer to the configured context; returns the device time (ms) spent inside the bulk
+    mixkvq_quantize_append calls alone (input generation excluded)."""
+    ms = 0.0
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for layer in range(w.n_layers):
         t = 0
         while t < w.tokens:
             n = min(PREFILL_CHUNK, w.tokens - t)
             k, v, q = W.tokens(w, layer, t, n, device=dev)
+            e0.record()
             cache.quantize_append(layer, k, v, q)
+            e1.record()
+            e1.synchronize()
+            ms += e0.elapsed_time(e1)
             t += n
     torch.cuda.synchronize()
+    return ms
 
 
 def tier_mix(cache, w):
@@ -226,7 +235,7 @@ def run_gpu(args, w):
                               tau_u4=w.tau_u4, score_bits=w.score_bits, block_layout=args.layout,
                               extras_budget_bytes=((w.tokens + n_steps) // w.residual_len + 3) * 8192 if w.score_bits == 4 else 0)
     cache = binding.Cache(cfg, device=dev)
-    prefill(cache, w, dev)
+    prefill_ms = prefill(cache, w, dev)
     assert cache.status() == 0
     scale = W.softmax_scale()
 
@@ -352,6 +361,9 @@ def run_gpu(args, w):
         "config": workload_config(w),
         "tokens_per_s": job_tokens_per_s(w.batch, world, us),
         "attention_graph_us_per_step": graph_us,
+        "prefill_quantize": {"ms": prefill_ms, "tokens_per_s": w.n_layers * w.batch * w.tokens / (prefill_ms * 1e-3),
+                             "input_gb_per_s": w.n_layers * w.batch * w.tokens * 256 * (2 * w.n_kv_heads + w.n_q_heads)
+                             / (prefill_ms * 1e-3) / 1e9},
         "flushes_in_timed_region": flushes,
         "tier_mix_mean": {"n16": n16, "n4": n4, "n2": 128 - n16 - n4},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,

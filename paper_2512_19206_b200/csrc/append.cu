@@ -16,12 +16,30 @@ append_tokens_kernel(LayerView lv, const __nv_bfloat16* __restrict__ k, const __
   __nv_bfloat16* resv = reinterpret_cast<__nv_bfloat16*>(lv.resv + (size_t)s * lv.resv_stride);
   double* acc = reinterpret_cast<double*>(lv.state + (size_t)s * lv.state_stride);
   double a = acc[d];
-  for (int i = 0; i < m; ++i) {
-    resk[(size_t)(r0 + i) * kD + d] = k[kv_base + (size_t)i * kD];
-    resv[(size_t)d * lv.R + (r0 + i)] = v[kv_base + (size_t)i * kD];
-    for (int h = 0; h < lv.g; ++h) {
-      size_t qi = (((size_t)b * lv.Hq + hk * lv.g + h) * n_tokens + t0 + i) * kD + d;
-      a = __dadd_rn(a, (double)fabsf(__bfloat162float(q[qi])));
+  const __nv_bfloat16* qw = q + (((size_t)b * lv.Hq + hk * lv.g) * n_tokens + t0) * kD + d;
+  const size_t head_stride = (size_t)n_tokens * kD;
+  for (int i0 = 0; i0 < m; i0 += 4) {
+    // the loads of up to four tokens go out together; the fp64 additions keep the defined order
+    float mag[4][8];
+    __nv_bfloat16 kk[4], vv[4];
+#pragma unroll
+    for (int ii = 0; ii < 4; ++ii) {
+      const bool on = i0 + ii < m;
+      kk[ii] = on ? k[kv_base + (size_t)(i0 + ii) * kD] : __float2bfloat16(0.f);
+      vv[ii] = on ? v[kv_base + (size_t)(i0 + ii) * kD] : __float2bfloat16(0.f);
+#pragma unroll
+      for (int h = 0; h < 8; ++h)
+        mag[ii][h] = (on && h < lv.g) ? fabsf(__bfloat162float(qw[(size_t)(i0 + ii) * kD + h * head_stride])) : 0.f;
+    }
+#pragma unroll
+    for (int ii = 0; ii < 4; ++ii) {
+      if (i0 + ii < m) {
+        resk[(size_t)(r0 + i0 + ii) * kD + d] = kk[ii];
+        resv[(size_t)d * lv.R + (r0 + i0 + ii)] = vv[ii];
+#pragma unroll
+        for (int h = 0; h < 8; ++h)
+          if (h < lv.g) a = __dadd_rn(a, (double)mag[ii][h]);
+      }
     }
   }
   acc[d] = a;

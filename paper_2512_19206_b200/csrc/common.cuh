@@ -127,6 +127,8 @@ namespace mixkvq {
 cudaError_t launch_append(const LayerView& lv, const void* k, const void* v, const void* q, int n_tokens, int t0,
                           int m, cudaStream_t stream);
 cudaError_t launch_flush(const LayerView& lv, cudaStream_t stream);
+cudaError_t launch_flush_bulk(const LayerView& lv, const void* k, const void* v, const void* q, int n_tokens, int t0,
+                              int nb, cudaStream_t stream);
 cudaError_t launch_select_window(const LayerView& lv, uint8_t* tiers, double* salience, cudaStream_t stream);
 cudaError_t launch_select_raw(const void* q, const void* k, int B, int Hq, int Hkv, int lq, int lk, int score_bits,
                               float tau_bf16, float tau_u4, uint8_t* tiers, double* salience, cudaStream_t stream);

@@ -1,12 +1,56 @@
 // The lazy update of Appendix D.1 for one full residual window: channel statistics, salience and tiers
 // (Section 4.2), per-channel mixed-precision key quantization and per-token 2-bit value quantization
-// (Eq. 2), and bit-packing into the block layout.  One CTA per stream.
+// (Eq. 2), and bit-packing into the block layout.  One CTA per stream and block.
+//
+// Two sources: the residual window of the cache (decode: one block per call), or R-token windows taken straight
+// from the tensors of a bulk append (prefill: grid.y blocks per call, the block's importance computed from its own
+// queries).  The bulk form runs in two passes around a per-stream prefix sum, because a block's place in the
+// promoted-channel arena depends on the tier counts of the blocks before it.
 #include "common.cuh"
 
 namespace mixkvq {
 
+struct BulkSrc {
+  const uint16_t* k;      // [S][n_tokens][128] bf16 bits
+  const uint16_t* v;      // [S][n_tokens][128]
+  const uint16_t* q;      // [B][Hq][n_tokens][128]
+  int n_tokens, t0;       // tokens per stream in the tensors, first token of block 0 of this call
+  int phase;              // 0: residual window; 1: bulk, tier counts only; 2: bulk, quantize and pack
+};
+
+__host__ __device__ inline uint32_t flush_extras_bytes(const LayerView& lv, int n16, int n4) {
+  return lv.tile ? tile_extras_header_bytes(n16, n4) + tile_extras_body_bytes(n16, n4)
+                 : extras_header_bytes(n16, n4) + (uint32_t)lv.U * extras_unit_bytes(n16, n4);
+}
+
+// Bulk append, between the two passes: one thread per stream walks the new blocks in order, gives each its offset in
+// the promoted-channel arena and advances the arena pointer; a block that no longer fits loses its promotions and
+// the status word says so (the same rule as for a single flush).
+__global__ void bulk_prefix_kernel(LayerView lv, int nb) {
+  const int s = blockIdx.x * blockDim.x + threadIdx.x;
+  if (s >= lv.B * lv.Hkv) return;
+  char* state = lv.state + (size_t)s * lv.state_stride;
+  uint32_t* used = reinterpret_cast<uint32_t*>(state + 1028);
+  uint32_t off16 = *used;
+  uint2* table = reinterpret_cast<uint2*>(lv.table + (size_t)s * lv.table_stride) + lv.n_blocks;
+  for (int i = 0; i < nb; ++i) {
+    uint2 e = table[i];
+    const int n16 = e.y & 0xFF, n4 = (e.y >> 8) & 0xFF;
+    const uint32_t need = flush_extras_bytes(lv, n16, n4);
+    e.x = off16;
+    if ((uint64_t)off16 * 16 + need > lv.extras_budget) {
+      atomicOr(lv.status, (uint32_t)MIXKVQ_DEV_EXTRAS_FULL);
+      e.y = 0u;
+    } else {
+      off16 += need / 16;
+    }
+    table[i] = e;
+  }
+  *used = off16;
+}
+
 __global__ void __launch_bounds__(256)
-flush_kernel(LayerView lv) {
+flush_kernel(LayerView lv, BulkSrc src) {
   extern __shared__ __align__(16) unsigned char smem[];
   const int R = lv.R, G = lv.G, U = lv.U, NG = lv.NG, VG = lv.VG;
   uint16_t* kS = reinterpret_cast<uint16_t*>(smem);      // [R][128] residual keys (bf16 bits)
@@ -17,14 +61,28 @@ flush_kernel(LayerView lv) {
   int* misc = reinterpret_cast<int*>(chan4S + 128);       // n16, n4, extras offset (16-byte units)
 
   const int s = blockIdx.x, tid = threadIdx.x;
+  const bool bulk = src.phase != 0;
+  const int block_index = lv.n_blocks + (bulk ? (int)blockIdx.y : 0);
+  const size_t tok0 = (size_t)s * src.n_tokens + src.t0 + (size_t)blockIdx.y * R;     // bulk: first token of the window
   char* state = lv.state + (size_t)s * lv.state_stride;
-  char* blk = lv.base + (size_t)s * lv.base_stride + (size_t)lv.n_blocks * lv.base_bytes;
-  const uint4* resk4 = reinterpret_cast<const uint4*>(lv.resk + (size_t)s * lv.resk_stride);
+  char* blk = lv.base + (size_t)s * lv.base_stride + (size_t)block_index * lv.base_bytes;
+  const uint4* resk4 = bulk ? reinterpret_cast<const uint4*>(src.k + tok0 * kD)
+                            : reinterpret_cast<const uint4*>(lv.resk + (size_t)s * lv.resk_stride);
   const uint16_t* resv = reinterpret_cast<const uint16_t*>(lv.resv + (size_t)s * lv.resv_stride);
+  // value of (channel c, token j of the window): residual store is channel-major, the bulk tensor token-major
+  auto value_at = [&](int c, int j) -> uint16_t {
+    return bulk ? src.v[(tok0 + j) * kD + c] : resv[(size_t)c * R + j];
+  };
+  uint2* table_entry = reinterpret_cast<uint2*>(lv.table + (size_t)s * lv.table_stride + (size_t)block_index * 8);
 
   for (int i = tid; i < R * 16; i += 256) reinterpret_cast<uint4*>(kS)[i] = resk4[i];
   __syncthreads();
 
+  if (src.phase == 2) {
+    // the first pass left the 128 tiers in the first bytes of the block; fetch them before anything is written there
+    if (tid < kD) tierS[tid] = reinterpret_cast<const uint8_t*>(blk)[tid];
+    __syncthreads();
+  }
   // ---- statistics, salience, tier and key codes: one thread per channel
   if (tid < kD) {
     const int d = tid;
@@ -34,12 +92,43 @@ flush_kernel(LayerView lv) {
       wmx = fmaxf(wmx, x);
       wmn = fminf(wmn, x);
     }
-    double acc = reinterpret_cast<const double*>(state)[d];
-    uint32_t cnt = *reinterpret_cast<const uint32_t*>(state + 1024);
-    uint8_t tier = salience_tier(acc, cnt, wmx, wmn, lv.score_bits, lv.tau_bf16, lv.tau_u4, nullptr);
+    uint8_t tier;
+    if (src.phase == 2) {
+      tier = tierS[d];
+    } else {
+      double acc;
+      uint32_t cnt;
+      if (bulk) {
+        // importance of this window from its own queries, added token-major and head-ascending like the running
+        // accumulator; the loads of four tokens are issued together, the additions keep the order
+        const int b = s / lv.Hkv, hk = s % lv.Hkv;
+        const uint16_t* qw = src.q + (((size_t)b * lv.Hq + hk * lv.g) * src.n_tokens + src.t0 + (size_t)blockIdx.y * R) * kD + d;
+        const size_t head_stride = (size_t)src.n_tokens * kD;
+        acc = 0.0;
+        for (int j = 0; j < R; j += 4) {
+          float a[4][8];
+#pragma unroll
+          for (int jj = 0; jj < 4; ++jj)
+#pragma unroll
+            for (int h = 0; h < 8; ++h)
+              a[jj][h] = (h < lv.g) ? fabsf(bf16_bits_to_float(qw[(size_t)(j + jj) * kD + h * head_stride])) : 0.f;
+#pragma unroll
+          for (int jj = 0; jj < 4; ++jj)
+#pragma unroll
+            for (int h = 0; h < 8; ++h)
+              if (h < lv.g) acc = __dadd_rn(acc, (double)a[jj][h]);
+        }
+        cnt = (uint32_t)(R * lv.g);
+      } else {
+        acc = reinterpret_cast<const double*>(state)[d];
+        cnt = *reinterpret_cast<const uint32_t*>(state + 1024);
+      }
+      tier = salience_tier(acc, cnt, wmx, wmn, lv.score_bits, lv.tau_bf16, lv.tau_u4, nullptr);
+      if (src.phase == 1) reinterpret_cast<uint8_t*>(blk)[d] = tier;
+    }
     tierS[d] = tier;
     const int max_code = (tier == kU4) ? 15 : 3;
-    for (int kg = 0; kg < NG; ++kg) {
+    for (int kg = 0; kg < NG && src.phase != 1; ++kg) {
       uint32_t meta = 0;
       if (tier == kBF16) {
         for (int j = kg * G; j < (kg + 1) * G; ++j) cS[j * kD + d] = 0;
@@ -67,25 +156,37 @@ flush_kernel(LayerView lv) {
       if (tierS[d] == kBF16) chan16S[n16++] = (uint8_t)d;
       else if (tierS[d] == kU4) chan4S[n4++] = (uint8_t)d;
     }
-    uint32_t* used = reinterpret_cast<uint32_t*>(state + 1028);
-    uint32_t off16 = *used;
-    uint32_t need = lv.tile ? tile_extras_header_bytes(n16, n4) + tile_extras_body_bytes(n16, n4)
-                            : extras_header_bytes(n16, n4) + (uint32_t)U * extras_unit_bytes(n16, n4);
-    if ((uint64_t)off16 * 16 + need > lv.extras_budget) {
-      atomicOr(lv.status, (uint32_t)MIXKVQ_DEV_EXTRAS_FULL);
-      n16 = 0;
-      n4 = 0;      // nothing is written to the arena; the block is invalid and the status says so
+    uint32_t off16 = 0;
+    if (src.phase == 1) {
+      // bulk, first pass: only the tier counts; the offsets come from the per-stream prefix sum
+      *table_entry = make_uint2(0u, (uint32_t)n16 | ((uint32_t)n4 << 8));
+    } else if (src.phase == 2) {
+      // bulk, second pass: the prefix sum placed the block (and cleared the counts if the arena was full)
+      const uint2 e = *table_entry;
+      off16 = e.x;
+      if ((e.y & 0xFFFFu) == 0u) {
+        n16 = 0;
+        n4 = 0;
+      }
     } else {
-      *used = off16 + need / 16;
+      uint32_t* used = reinterpret_cast<uint32_t*>(state + 1028);
+      off16 = *used;
+      const uint32_t need = flush_extras_bytes(lv, n16, n4);
+      if ((uint64_t)off16 * 16 + need > lv.extras_budget) {
+        atomicOr(lv.status, (uint32_t)MIXKVQ_DEV_EXTRAS_FULL);
+        n16 = 0;
+        n4 = 0;      // nothing is written to the arena; the block is invalid and the status says so
+      } else {
+        *used = off16 + need / 16;
+      }
+      *table_entry = make_uint2(off16, (uint32_t)n16 | ((uint32_t)n4 << 8));
     }
-    uint32_t* entry = reinterpret_cast<uint32_t*>(lv.table + (size_t)s * lv.table_stride + (size_t)lv.n_blocks * 8);
-    entry[0] = off16;
-    entry[1] = (uint32_t)n16 | ((uint32_t)n4 << 8);
     misc[0] = n16;
     misc[1] = n4;
     misc[2] = (int)off16;
   }
   __syncthreads();
+  if (src.phase == 1) return;
   const int n16 = misc[0], n4 = misc[1];
   const int n16p = (n16 + 1) >> 1, n4p = ((n4 + 1) >> 1) << 1;
   char* ex = lv.extras + (size_t)s * lv.extras_stride + (size_t)misc[2] * 16;
@@ -179,13 +280,13 @@ flush_kernel(LayerView lv) {
     const int j = i % R, vg = i / R;
     float gmx = -INFINITY, gmn = INFINITY;
     for (int c = vg * G; c < (vg + 1) * G; ++c) {
-      float x = bf16_bits_to_float(resv[(size_t)c * R + j]);
+      float x = bf16_bits_to_float(value_at(c, j));
       gmx = fmaxf(gmx, x);
       gmn = fminf(gmn, x);
     }
     float sc = stored_scale(gmx, gmn, 3.0f);
     for (int c = vg * G; c < (vg + 1) * G; ++c)
-      cS[j * kD + c] = (uint8_t)quant_code(bf16_bits_to_float(resv[(size_t)c * R + j]), gmn, sc, 3);
+      cS[j * kD + c] = (uint8_t)quant_code(bf16_bits_to_float(value_at(c, j)), gmn, sc, 3);
     const int u = j >> 5, jj = j & 31;
     uint32_t* vmeta = lv.tile ? reinterpret_cast<uint32_t*>(blk + NG * 512 + 8192) + j * VG
                               : reinterpret_cast<uint32_t*>(blk + NG * 512 + (size_t)u * lv.unit_bytes + 2048) + jj * VG;
@@ -227,7 +328,7 @@ flush_kernel(LayerView lv) {
   }
 
   // ---- window importance: the accumulator restarts with the next window (Section 4.2)
-  if (lv.importance_mode == 0) {
+  if (lv.importance_mode == 0 && !bulk) {
     if (tid < kD) reinterpret_cast<double*>(state)[tid] = 0.0;
     if (tid == 0) *reinterpret_cast<uint32_t*>(state + 1024) = 0u;
   }
@@ -239,7 +340,24 @@ cudaError_t launch_flush(const LayerView& lv, cudaStream_t stream) {
   cudaError_t e = cudaFuncSetAttribute(flush_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)flush_smem_bytes(256));
   if (e != cudaSuccess) return e;
-  flush_kernel<<<lv.B * lv.Hkv, 256, flush_smem_bytes(lv.R), stream>>>(lv);
+  flush_kernel<<<lv.B * lv.Hkv, 256, flush_smem_bytes(lv.R), stream>>>(lv, BulkSrc{nullptr, nullptr, nullptr, 0, 0, 0});
+  return cudaGetLastError();
+}
+
+// nb complete R-token windows starting at token t0 of the append's tensors go straight to packed blocks
+// (three launches).  Preconditions (checked by the caller): window importance mode, empty residual window.
+cudaError_t launch_flush_bulk(const LayerView& lv, const void* k, const void* v, const void* q, int n_tokens, int t0,
+                              int nb, cudaStream_t stream) {
+  cudaError_t e = cudaFuncSetAttribute(flush_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)flush_smem_bytes(256));
+  if (e != cudaSuccess) return e;
+  const int S = lv.B * lv.Hkv;
+  BulkSrc src{static_cast<const uint16_t*>(k), static_cast<const uint16_t*>(v), static_cast<const uint16_t*>(q), n_tokens, t0, 1};
+  const dim3 grid(S, nb);
+  flush_kernel<<<grid, 256, flush_smem_bytes(lv.R), stream>>>(lv, src);
+  bulk_prefix_kernel<<<(S + 127) / 128, 128, 0, stream>>>(lv, nb);
+  src.phase = 2;
+  flush_kernel<<<grid, 256, flush_smem_bytes(lv.R), stream>>>(lv, src);
   return cudaGetLastError();
 }
 

@@ -69,10 +69,6 @@ flush_kernel(LayerView lv, BulkSrc src) {
   const uint4* resk4 = bulk ? reinterpret_cast<const uint4*>(src.k + tok0 * kD)
                             : reinterpret_cast<const uint4*>(lv.resk + (size_t)s * lv.resk_stride);
   const uint16_t* resv = reinterpret_cast<const uint16_t*>(lv.resv + (size_t)s * lv.resv_stride);
-  // value of (channel c, token j of the window): residual store is channel-major, the bulk tensor token-major
-  auto value_at = [&](int c, int j) -> uint16_t {
-    return bulk ? src.v[(tok0 + j) * kD + c] : resv[(size_t)c * R + j];
-  };
   uint2* table_entry = reinterpret_cast<uint2*>(lv.table + (size_t)s * lv.table_stride + (size_t)block_index * 8);
 
   for (int i = tid; i < R * 16; i += 256) reinterpret_cast<uint4*>(kS)[i] = resk4[i];
@@ -82,6 +78,28 @@ flush_kernel(LayerView lv, BulkSrc src) {
     // the first pass left the 128 tiers in the first bytes of the block; fetch them before anything is written there
     if (tid < kD) tierS[tid] = reinterpret_cast<const uint8_t*>(blk)[tid];
     __syncthreads();
+  }
+  // ---- bulk, first pass: importance of this window from its own queries.  All threads stage a few tokens of the g
+  // heads at a time (16-byte loads); thread d then adds |q| of channel d token-major and head-ascending, the order of
+  // the running accumulator of the decode path.
+  double bulk_acc = 0.0;
+  if (src.phase == 1) {
+    const int b = s / lv.Hkv, hk = s % lv.Hkv;
+    const uint16_t* qw = src.q + (((size_t)b * lv.Hq + hk * lv.g) * src.n_tokens + src.t0 + (size_t)blockIdx.y * R) * kD;
+    const size_t head_stride = (size_t)src.n_tokens * kD;
+    uint16_t* qS = reinterpret_cast<uint16_t*>(cS);                  // [tc tokens][g heads][128], the code area is idle here
+    const int tc = R / 16;                                           // tokens per chunk: R * 128 bytes hold tc * 8 rows
+    for (int j0 = 0; j0 < R; j0 += tc) {
+      for (int i = tid; i < tc * lv.g * 16; i += 256) {
+        const int row = i >> 4, c16 = i & 15, jj = row / lv.g, h = row - jj * lv.g;
+        reinterpret_cast<uint4*>(qS)[i] = *reinterpret_cast<const uint4*>(qw + (size_t)(j0 + jj) * kD + h * head_stride + 8 * c16);
+      }
+      __syncthreads();
+      if (tid < kD)
+        for (int row = 0; row < tc * lv.g; ++row)
+          bulk_acc = __dadd_rn(bulk_acc, (double)fabsf(bf16_bits_to_float(qS[row * kD + tid])));
+      __syncthreads();
+    }
   }
   // ---- statistics, salience, tier and key codes: one thread per channel
   if (tid < kD) {
@@ -99,25 +117,7 @@ flush_kernel(LayerView lv, BulkSrc src) {
       double acc;
       uint32_t cnt;
       if (bulk) {
-        // importance of this window from its own queries, added token-major and head-ascending like the running
-        // accumulator; the loads of four tokens are issued together, the additions keep the order
-        const int b = s / lv.Hkv, hk = s % lv.Hkv;
-        const uint16_t* qw = src.q + (((size_t)b * lv.Hq + hk * lv.g) * src.n_tokens + src.t0 + (size_t)blockIdx.y * R) * kD + d;
-        const size_t head_stride = (size_t)src.n_tokens * kD;
-        acc = 0.0;
-        for (int j = 0; j < R; j += 4) {
-          float a[4][8];
-#pragma unroll
-          for (int jj = 0; jj < 4; ++jj)
-#pragma unroll
-            for (int h = 0; h < 8; ++h)
-              a[jj][h] = (h < lv.g) ? fabsf(bf16_bits_to_float(qw[(size_t)(j + jj) * kD + h * head_stride])) : 0.f;
-#pragma unroll
-          for (int jj = 0; jj < 4; ++jj)
-#pragma unroll
-            for (int h = 0; h < 8; ++h)
-              if (h < lv.g) acc = __dadd_rn(acc, (double)a[jj][h]);
-        }
+        acc = bulk_acc;
         cnt = (uint32_t)(R * lv.g);
       } else {
         acc = reinterpret_cast<const double*>(state)[d];
@@ -275,22 +275,62 @@ flush_kernel(LayerView lv, BulkSrc src) {
   }
   __syncthreads();
 
-  // ---- values: per token, per group of G channels, 2 bits
-  for (int i = tid; i < R * VG; i += 256) {
-    const int j = i % R, vg = i / R;
-    float gmx = -INFINITY, gmn = INFINITY;
-    for (int c = vg * G; c < (vg + 1) * G; ++c) {
-      float x = bf16_bits_to_float(value_at(c, j));
-      gmx = fmaxf(gmx, x);
-      gmn = fminf(gmn, x);
-    }
-    float sc = stored_scale(gmx, gmn, 3.0f);
-    for (int c = vg * G; c < (vg + 1) * G; ++c)
-      cS[j * kD + c] = (uint8_t)quant_code(bf16_bits_to_float(value_at(c, j)), gmn, sc, 3);
+  // ---- values: per token, per group of G channels, 2 bits.  The key window is no longer needed: the value window
+  // takes its place in shared memory (as stored: channel-major from the residual store, token-major from a tensor).
+  {
+    const uint4* vsrc = bulk ? reinterpret_cast<const uint4*>(src.v + tok0 * kD) : reinterpret_cast<const uint4*>(resv);
+    for (int i = tid; i < R * 16; i += 256) reinterpret_cast<uint4*>(kS)[i] = vsrc[i];
+  }
+  __syncthreads();
+  auto vmeta_of = [&](int j) -> uint32_t* {
     const int u = j >> 5, jj = j & 31;
-    uint32_t* vmeta = lv.tile ? reinterpret_cast<uint32_t*>(blk + NG * 512 + 8192) + j * VG
-                              : reinterpret_cast<uint32_t*>(blk + NG * 512 + (size_t)u * lv.unit_bytes + 2048) + jj * VG;
-    vmeta[vg] = float_to_bf16_bits_exact(sc) | (float_to_bf16_bits_exact(gmn) << 16);
+    return lv.tile ? reinterpret_cast<uint32_t*>(blk + NG * 512 + 8192) + j * VG
+                   : reinterpret_cast<uint32_t*>(blk + NG * 512 + (size_t)u * lv.unit_bytes + 2048) + jj * VG;
+  };
+  if (bulk) {
+    // token-major window: a warp takes a token, lane l the channels l, l+32, l+64, l+96; group extrema by shuffles
+    const int warp = tid >> 5, lane = tid & 31;
+    for (int j = warp; j < R; j += 8) {
+      float x[4], gmx[4], gmn[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) x[k] = gmx[k] = gmn[k] = bf16_bits_to_float(kS[j * kD + lane + 32 * k]);
+      if (G >= 64) {
+        gmx[0] = gmx[1] = fmaxf(x[0], x[1]); gmn[0] = gmn[1] = fminf(x[0], x[1]);
+        gmx[2] = gmx[3] = fmaxf(x[2], x[3]); gmn[2] = gmn[3] = fminf(x[2], x[3]);
+      }
+      if (G == 128) {
+        gmx[0] = gmx[1] = gmx[2] = gmx[3] = fmaxf(gmx[0], gmx[2]);
+        gmn[0] = gmn[1] = gmn[2] = gmn[3] = fminf(gmn[0], gmn[2]);
+      }
+#pragma unroll
+      for (int off = 16; off; off >>= 1)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          gmx[k] = fmaxf(gmx[k], __shfl_xor_sync(0xffffffffu, gmx[k], off));
+          gmn[k] = fminf(gmn[k], __shfl_xor_sync(0xffffffffu, gmn[k], off));
+        }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const float sc = stored_scale(gmx[k], gmn[k], 3.0f);
+        cS[j * kD + lane + 32 * k] = (uint8_t)quant_code(x[k], gmn[k], sc, 3);
+        const int vg = (32 * k) / G;
+        if (lane == 0 && (32 * k) % G == 0) vmeta_of(j)[vg] = float_to_bf16_bits_exact(sc) | (float_to_bf16_bits_exact(gmn[k]) << 16);
+      }
+    }
+  } else {
+    for (int i = tid; i < R * VG; i += 256) {
+      const int j = i % R, vg = i / R;
+      float gmx = -INFINITY, gmn = INFINITY;
+      for (int c = vg * G; c < (vg + 1) * G; ++c) {
+        float x = bf16_bits_to_float(kS[c * R + j]);
+        gmx = fmaxf(gmx, x);
+        gmn = fminf(gmn, x);
+      }
+      float sc = stored_scale(gmx, gmn, 3.0f);
+      for (int c = vg * G; c < (vg + 1) * G; ++c)
+        cS[j * kD + c] = (uint8_t)quant_code(bf16_bits_to_float(kS[c * R + j]), gmn, sc, 3);
+      vmeta_of(j)[vg] = float_to_bf16_bits_exact(sc) | (float_to_bf16_bits_exact(gmn) << 16);
+    }
   }
   __syncthreads();
   if (lv.tile) {

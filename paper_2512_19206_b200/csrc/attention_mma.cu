@@ -190,6 +190,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
       pf_entry = table[pf_bi];
     }
     int n16 = 0, n4 = 0, n16p = 0;
+    uint32_t xb0 = 0u, xb1 = 0u;          // B fragments of the block's first 16 promoted channels
     const char* ex = nullptr;
     uint32_t ex_hdr = 0, ex_unit = 0;
 
@@ -245,6 +246,19 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
         ex = extras + (size_t)entry.x * 16;
         ex_hdr = extras_header_bytes(n16, n4);
         ex_unit = extras_unit_bytes(n16, n4);
+        // the block's promoted channels are the same for its units: gather their query entries once
+        xb0 = xb1 = 0u;
+        if (n16 > 0) {
+          auto gather_q = [&](int p) -> uint32_t {
+            if (p >= n16p) return 0u;
+            const uint32_t ids = *reinterpret_cast<const uint16_t*>(ex + 2 * p);
+            const uint32_t c0 = ids & 0xFF, c1 = (ids >> 8) & 0xFF;
+            const uint32_t lo = (c0 < 128) ? qb16[r * kD + c0] : 0u, hi = (c1 < 128) ? qb16[r * kD + c1] : 0u;
+            return lo | (hi << 16);
+          };
+          xb0 = gather_q(t);
+          xb1 = gather_q(t + 4);
+        }
       }
       const uint32_t stage = ring_count % kStages, parity = (ring_count / kStages) & 1;
       if (!mbar_wait_bounded(smem_u32(&bars[warp * kStages + stage]), parity)) {
@@ -279,11 +293,9 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
       // ---- extras of this unit: issue the global loads early
       const char* exu = ex + ex_hdr + (size_t)u * ex_unit;
       uint32_t xa[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};   // BF16 pairs, first 16 promoted channels
-      uint32_t xid0 = 0xFFFFFFFFu, xid1 = 0xFFFFFFFFu;
       if (n16 > 0) {
         const uint32_t* xw = reinterpret_cast<const uint32_t*>(exu);
         if (t < n16p) {
-          xid0 = *reinterpret_cast<const uint16_t*>(ex + 2 * t);
 #pragma unroll
           for (int mt = 0; mt < 2; ++mt) {
             xa[mt][0] = xw[t * 32 + mt * 16 + r];
@@ -291,7 +303,6 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
           }
         }
         if (t + 4 < n16p) {
-          xid1 = *reinterpret_cast<const uint16_t*>(ex + 2 * (t + 4));
 #pragma unroll
           for (int mt = 0; mt < 2; ++mt) {
             xa[mt][2] = xw[(t + 4) * 32 + mt * 16 + r];
@@ -329,14 +340,11 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
       // ---- promoted channels (raw bf16 keys) with a gathered q
       if (n16 > 0) {
         for (int kk = 0; kk * 8 < n16p; ++kk) {
-          uint32_t a[2][4], id0, id1;
+          uint32_t a[2][4], id0 = 0xFFFFFFFFu, id1 = 0xFFFFFFFFu;
           if (kk == 0) {
 #pragma unroll
-            for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-              for (int j = 0; j < 4; ++j) a[mt][j] = xa[mt][j];
-            id0 = xid0;
-            id1 = xid1;
+            for (int mt = 0; mt < 2; ++mt) mma_bf16(Sx[mt], xa[mt][0], xa[mt][1], xa[mt][2], xa[mt][3], xb0, xb1);
+            continue;
           } else {
             const uint32_t* xw = reinterpret_cast<const uint32_t*>(exu);
             const int p0 = 8 * kk + t, p1 = p0 + 4;

@@ -82,7 +82,7 @@ typedef struct mixkvq_layout_desc {
   uint64_t state_off, state_stride;       /* per stream: acc fp64[128], cnt u32, extras_used16 u32   */
   uint64_t table_off, table_stride;       /* per stream: max_blocks entries of 8 bytes               */
   uint64_t resk_off, resk_stride;         /* per stream: [R][128] bf16                               */
-  uint64_t resv_off, resv_stride;         /* per stream: [128][R] bf16                               */
+  uint64_t resv_off, resv_stride;         /* per stream: [R][128] bf16                               */
   uint64_t base_off, base_stride;         /* per stream: max_blocks blocks of base_bytes             */
   uint64_t extras_off, extras_stride;     /* per stream: extras arena                                */
   uint64_t base_bytes;                    /* size of one block's fixed part                          */

@@ -577,5 +577,5 @@ def pack_stream(st: OracleStream, layout=LAYOUT_FRAGMENT):
         "extras": b"".join(extras),
         "state": bytes(state),
         "resK": bf16_to_u16(st.resK[:st.r]).astype("<u2").tobytes(),
-        "resV_T": bf16_to_u16(np.ascontiguousarray(st.resV[:st.r].T)).astype("<u2").tobytes(),  # [D][r]
+        "resV": bf16_to_u16(st.resV[:st.r]).astype("<u2").tobytes(),
     }

@@ -223,5 +223,5 @@ class Cache:
             "extras": cut(d.extras_off, d.extras_stride, used16 * 16),
             "state": state,
             "resK": resk[: r * 256],
-            "resV_full": resv,      # [128][R] bf16, only the first r tokens of each row are meaningful
+            "resV": resv[: r * 256],
         }

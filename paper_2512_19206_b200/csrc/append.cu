@@ -35,7 +35,7 @@ append_tokens_kernel(LayerView lv, const __nv_bfloat16* __restrict__ k, const __
     for (int ii = 0; ii < 4; ++ii) {
       if (i0 + ii < m) {
         resk[(size_t)(r0 + i0 + ii) * kD + d] = kk[ii];
-        resv[(size_t)d * lv.R + (r0 + i0 + ii)] = vv[ii];
+        resv[(size_t)(r0 + i0 + ii) * kD + d] = vv[ii];
 #pragma unroll
         for (int h = 0; h < 8; ++h)
           if (h < lv.g) a = __dadd_rn(a, (double)mag[ii][h]);

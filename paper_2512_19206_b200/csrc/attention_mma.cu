@@ -526,17 +526,18 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
       if (lane == 0) atomicOr(lv.status, (uint32_t)MIXKVQ_DEV_COPY_TIMEOUT);
     }
 
-    // ---- residual (unquantized) tokens of this warp's range: bf16 rows staged through the (now idle) ring.
-    // Keys: 32 token rows of 256 B, one bulk copy per lane, rows 272 B apart (conflict-free fragment loads).
-    // Values: 128 channel rows of 64 B (tokens j0..j0+31), four bulk copies per lane, rows 64 B apart.
+    // ---- residual (unquantized) tokens of this warp's range: 32 token rows of 256 B staged through the (now idle)
+    // ring with ONE bulk copy, first the keys, then the values over them (small bulk copies are slow: a copy per row
+    // cost tens of microseconds).  Value tiles are transposed on the way to registers with ldmatrix.trans.
     for (int x = max(wb, packed_units); x < we && !gave_up; ++x) {
       const uint32_t rbar = smem_u32(&bars[kWarps * kStages + warp]);
       {
         const int j0s = (x - packed_units) * 32, nv = min(32, lv.r - j0s);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        if (lane == 0) mbar_expect_tx(rbar, (uint32_t)nv * 256u);
-        __syncwarp();
-        if (lane < nv) bulk_g2s(smem_u32(ring + lane * 272), resk + (size_t)(j0s + lane) * kD, 256u, rbar);
+        if (lane == 0) {
+          mbar_expect_tx(rbar, (uint32_t)nv * 256u);
+          bulk_g2s(smem_u32(ring), resk + (size_t)j0s * kD, (uint32_t)nv * 256u, rbar);
+        }
         if (!mbar_wait_bounded(rbar, res_phase)) {
           gave_up = true;
           if (lane == 0) atomicOr(lv.status, (uint32_t)MIXKVQ_DEV_COPY_TIMEOUT);
@@ -560,8 +561,8 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt) {
           const int ta = j0 + mt * 16 + r, tb = ta + 8;
-          const uint32_t* ka = reinterpret_cast<const uint32_t*>(ring + (mt * 16 + r) * 272 + (16 * kt + 2 * t) * 2);
-          const uint32_t* kb = reinterpret_cast<const uint32_t*>(ring + (mt * 16 + 8 + r) * 272 + (16 * kt + 2 * t) * 2);
+          const uint32_t* ka = reinterpret_cast<const uint32_t*>(ring + (mt * 16 + r) * 256 + (16 * kt + 2 * t) * 2);
+          const uint32_t* kb = reinterpret_cast<const uint32_t*>(ring + (mt * 16 + 8 + r) * 256 + (16 * kt + 2 * t) * 2);
           const uint32_t a0 = ta < rt ? ka[0] : 0u, a1 = tb < rt ? kb[0] : 0u;
           const uint32_t a2 = ta < rt ? ka[4] : 0u, a3 = tb < rt ? kb[4] : 0u;
           mma_bf16(Sx[mt], a0, a1, a2, a3, b0, b1);
@@ -606,12 +607,10 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
       // the key rows are consumed: stage the value rows of these 32 tokens over them
       __syncwarp();
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      if (lane == 0) mbar_expect_tx(rbar, 128u * 64u);
-      __syncwarp();
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int c = lane + 32 * i;
-        bulk_g2s(smem_u32(ring + c * 64), resv + (size_t)c * lv.R + j0, 64u, rbar);
+      const int nvv = min(32, rt - j0);
+      if (lane == 0) {
+        mbar_expect_tx(rbar, (uint32_t)nvv * 256u);
+        bulk_g2s(smem_u32(ring), resv + (size_t)j0 * kD, (uint32_t)nvv * 256u, rbar);
       }
       if (!mbar_wait_bounded(rbar, res_phase)) {
         gave_up = true;
@@ -619,20 +618,23 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
         break;
       }
       res_phase ^= 1u;
+      // tile (ct, ks): A = V^T, 16 channels x 16 tokens, from four transposed 8x8 tiles of the token-major rows:
+      // matrix i of the ldmatrix has tokens 16ks + 8(i >> 1) .., channels 16ct + 8(i & 1) ..; lane l gives row l % 8 of matrix l / 8
+      const uint32_t lm_row = smem_u32(ring) + (uint32_t)((8 * (lane >> 4) + (lane & 7)) * 256 + 16 * ((lane >> 3) & 1));
 #pragma unroll
       for (int ct = 0; ct < 8; ++ct) {
-        const int c0 = 16 * ct + r, c1 = c0 + 8;
 #pragma unroll
         for (int ks = 0; ks < 2; ++ks) {
+          uint32_t a0, a1, a2, a3;
+          asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                       : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3)
+                       : "r"(lm_row + (uint32_t)(ks * 16 * 256 + ct * 32)));
+          // tokens of this lane's pairs: 16ks + 2t, +1 (a0, a1) and 16ks + 8 + 2t, +1 (a2, a3); rows past r are stale
           const int ja = j0 + 16 * ks + 2 * t, jb = ja + 8;
-          auto load_pair = [&](int c, int j) -> uint32_t {
-            if (j >= rt) return 0u;
-            uint32_t w = *reinterpret_cast<const uint32_t*>(ring + c * 64 + (j - j0) * 2);
-            if (j + 1 >= rt) w &= 0xFFFFu;
-            return bf16x2_to_f16x2(w);
-          };
-          mma_f16(O[ct], load_pair(c0, ja), load_pair(c1, ja), load_pair(c0, jb), load_pair(c1, jb), Pt[ks][0],
-                  Pt[ks][1]);
+          const uint32_t ma = ja + 1 < rt ? 0xFFFFFFFFu : (ja < rt ? 0x0000FFFFu : 0u);
+          const uint32_t mb = jb + 1 < rt ? 0xFFFFFFFFu : (jb < rt ? 0x0000FFFFu : 0u);
+          mma_f16(O[ct], bf16x2_to_f16x2(a0 & ma), bf16x2_to_f16x2(a1 & ma), bf16x2_to_f16x2(a2 & mb), bf16x2_to_f16x2(a3 & mb),
+                  Pt[ks][0], Pt[ks][1]);
         }
       }
     }

@@ -159,7 +159,7 @@ attention_simt_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float s
       } else {
         const int j = (unit - packed_units) * 32 + jj;
         for (int i = 0; i < 4; ++i)
-          vv[i] = (j < lv.r) ? bf16_bits_to_float(resv[(size_t)(4 * lane + i) * lv.R + j]) : 0.f;
+          vv[i] = (j < lv.r) ? bf16_bits_to_float(resv[(size_t)j * kD + 4 * lane + i]) : 0.f;
       }
       for (int h = 0; h < 8; ++h) {
         const float ph = __shfl_sync(0xffffffffu, p[h], jj);

@@ -276,7 +276,7 @@ flush_kernel(LayerView lv, BulkSrc src) {
   __syncthreads();
 
   // ---- values: per token, per group of G channels, 2 bits.  The key window is no longer needed: the value window
-  // takes its place in shared memory (as stored: channel-major from the residual store, token-major from a tensor).
+  // takes its place in shared memory (token-major in the residual store and in a tensor alike).
   {
     const uint4* vsrc = bulk ? reinterpret_cast<const uint4*>(src.v + tok0 * kD) : reinterpret_cast<const uint4*>(resv);
     for (int i = tid; i < R * 16; i += 256) reinterpret_cast<uint4*>(kS)[i] = vsrc[i];
@@ -287,7 +287,7 @@ flush_kernel(LayerView lv, BulkSrc src) {
     return lv.tile ? reinterpret_cast<uint32_t*>(blk + NG * 512 + 8192) + j * VG
                    : reinterpret_cast<uint32_t*>(blk + NG * 512 + (size_t)u * lv.unit_bytes + 2048) + jj * VG;
   };
-  if (bulk) {
+  {
     // token-major window: a warp takes a token, lane l the channels l, l+32, l+64, l+96; group extrema by shuffles
     const int warp = tid >> 5, lane = tid & 31;
     for (int j = warp; j < R; j += 8) {
@@ -316,20 +316,6 @@ flush_kernel(LayerView lv, BulkSrc src) {
         const int vg = (32 * k) / G;
         if (lane == 0 && (32 * k) % G == 0) vmeta_of(j)[vg] = float_to_bf16_bits_exact(sc) | (float_to_bf16_bits_exact(gmn[k]) << 16);
       }
-    }
-  } else {
-    for (int i = tid; i < R * VG; i += 256) {
-      const int j = i % R, vg = i / R;
-      float gmx = -INFINITY, gmn = INFINITY;
-      for (int c = vg * G; c < (vg + 1) * G; ++c) {
-        float x = bf16_bits_to_float(kS[c * R + j]);
-        gmx = fmaxf(gmx, x);
-        gmn = fminf(gmn, x);
-      }
-      float sc = stored_scale(gmx, gmn, 3.0f);
-      for (int c = vg * G; c < (vg + 1) * G; ++c)
-        cS[j * kD + c] = (uint8_t)quant_code(bf16_bits_to_float(kS[c * R + j]), gmn, sc, 3);
-      vmeta_of(j)[vg] = float_to_bf16_bits_exact(sc) | (float_to_bf16_bits_exact(gmn) << 16);
     }
   }
   __syncthreads();

@@ -130,10 +130,8 @@ def test_streamed_appends_equal_bulk(binding):
     for s in range(w.n_kv_heads):
         a, b, c = bulk.stream_regions(0, s), one.stream_regions(0, s), two.stream_regions(0, s)
         r = bulk.describe(0).residual_tokens
-        for key in ("table", "base", "extras", "state", "resK"):
+        for key in ("table", "base", "extras", "state", "resK", "resV"):
             assert a[key] == b[key] == c[key], key
-        av = np.frombuffer(a["resV_full"], "<u2").reshape(128, -1)[:, :r]
-        assert np.array_equal(av, np.frombuffer(b["resV_full"], "<u2").reshape(128, -1)[:, :r])
     U.compare_regions(bulk, 0, w, U.oracle_streams(w, 0, k, v, q))
 
 

@@ -211,5 +211,5 @@ def test_stream_regions(rng):
         assert e[4] == (blk.tiers == 2).sum() and e[5] == (blk.tiers == 1).sum() and e[6:] == b"\0\0"
         off += len(O.pack_extras_tile(blk)[0]) // 16
     assert int.from_bytes(p["state"][1028:1032], "little") == off
-    assert len(p["resK"]) == 5 * 256 and len(p["resV_T"]) == 5 * 256
-    assert np.array_equal(np.frombuffer(p["resV_T"], "<u2").reshape(128, 5), O.bf16_to_u16(v[-5:]).T)
+    assert len(p["resK"]) == 5 * 256 and len(p["resV"]) == 5 * 256
+    assert np.array_equal(np.frombuffer(p["resV"], "<u2").reshape(5, 128), O.bf16_to_u16(v[-5:]))

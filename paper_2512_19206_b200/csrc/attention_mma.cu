@@ -31,6 +31,7 @@ constexpr int kPrepBytes = 1280;             // kprep 512 | zprep 256 | svp 256 
 constexpr int kSharedTail = 128 + 2048 + 2048 + 128 + 128 + 4096;
 constexpr int kSmemBytes = kWarps * (kStages * kStageBytes + kPrepBytes) + kSharedTail;
 constexpr int kCtasPerSm = 4;
+constexpr int kResidualWeight = 2;           // a 32-token unit of the residual window counts as this many packed units in the split
 constexpr uint32_t kSpinLimit = 1u << 22;    // bounded wait on a staged copy
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -140,7 +141,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
 
   const int S = lv.B * lv.Hkv, U = lv.U, g = lv.g;
   const int packed_units = lv.n_blocks * U;
-  const int Us = packed_units + (lv.r + 31) / 32;
+  const int Us = packed_units + kResidualWeight * ((lv.r + 31) / 32);     // split positions; a residual unit spans several
   const long long total = (long long)Us * S;
   const long long cb = split_begin(total, gridDim.x, blockIdx.x), ce = split_begin(total, gridDim.x, blockIdx.x + 1);
 
@@ -529,7 +530,9 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
     // ---- residual (unquantized) tokens of this warp's range: 32 token rows of 256 B staged through the (now idle)
     // ring with ONE bulk copy, first the keys, then the values over them (small bulk copies are slow: a copy per row
     // cost tens of microseconds).  Value tiles are transposed on the way to registers with ldmatrix.trans.
-    for (int x = max(wb, packed_units); x < we && !gave_up; ++x) {
+    for (int xv = max(wb, packed_units); xv < we && !gave_up; ++xv) {
+      if ((xv - packed_units) % kResidualWeight != 0) continue;       // the warp owning a unit's first position runs it
+      const int x = packed_units + (xv - packed_units) / kResidualWeight;
       const uint32_t rbar = smem_u32(&bars[kWarps * kStages + warp]);
       {
         const int j0s = (x - packed_units) * 32, nv = min(32, lv.r - j0s);
@@ -727,17 +730,26 @@ cudaError_t attention_mma_setup() {
 }
 
 // Number of CTAs the split kernel runs for this layer state (also the number of partial-slot owners).
+// Split positions per stream: packed units plus the weighted units of the residual window.
+long long attention_mma_positions(const LayerView& lv) {
+  return (long long)lv.n_blocks * lv.U + (long long)kResidualWeight * ((lv.r + 31) / 32);
+}
+
+// Number of CTAs the split kernel runs for this layer state (also the number of partial-slot owners).  When there are
+// fewer streams than CTA slots the grid is a multiple of the stream count, so that no CTA straddles two streams
+// (a second segment costs a pipeline drain, a query load and a second partial).
 int attention_mma_grid(const LayerView& lv, int n_sms) {
-  const long long Us = (long long)lv.n_blocks * lv.U + (lv.r + 31) / 32;
-  const long long total = Us * lv.B * lv.Hkv;
-  const int grid = (int)min((long long)min(n_sms * kCtasPerSm, kMaxCtas / 2), total);
+  const int S = lv.B * lv.Hkv;
+  const long long total = attention_mma_positions(lv) * S;
+  int grid = (int)min((long long)min(n_sms * kCtasPerSm, kMaxCtas / 2), total);
+  if (grid > S) grid = grid / S * S;
   return grid < 1 ? 1 : grid;
 }
 
 cudaError_t launch_attention_mma(const LayerView& lv, const void* q, float* out, float scale, float* ws, int n_sms,
                                  cudaStream_t stream, int* launches) {
   const int S = lv.B * lv.Hkv;
-  const long long Us = (long long)lv.n_blocks * lv.U + (lv.r + 31) / 32;
+  const long long Us = attention_mma_positions(lv);
   const int grid = attention_mma_grid(lv, n_sms);
   cudaError_t e;
   if (lv.G == 32) e = launch_g<32>(lv, q, scale, ws, grid, stream);

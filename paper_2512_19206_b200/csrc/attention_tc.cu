@@ -22,6 +22,7 @@ namespace mixkvq {
 cudaError_t launch_combine2(const float* ws, float* out, int g, int Hkv, int Hq, int S, int n1, long long units1,
                             int slot2, int n2, long long units2, cudaStream_t stream);
 int attention_mma_grid(const LayerView& lv, int n_sms);
+long long attention_mma_positions(const LayerView& lv);
 
 namespace {
 
@@ -748,7 +749,7 @@ cudaError_t launch_attention_tc(const LayerView& lv, const void* q, float* out, 
   *launches += l2;
   if (e != cudaSuccess) return e;
   e = launch_combine2(ws, out, lv.g, lv.Hkv, lv.Hq, S, n1, lv.n_blocks, slot2, attention_mma_grid(res, n_sms),
-                      (lv.r + 31) / 32, stream);
+                      attention_mma_positions(res), stream);
   *launches += 1;
   return e;
 }

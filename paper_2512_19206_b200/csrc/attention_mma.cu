@@ -31,6 +31,7 @@ constexpr int kPrepBytes = 1280;             // kprep 512 | zprep 256 | svp 256 
 constexpr int kSharedTail = 128 + 2048 + 2048 + 128 + 128 + 4096;
 constexpr int kSmemBytes = kWarps * (kStages * kStageBytes + kPrepBytes) + kSharedTail;
 constexpr int kCtasPerSm = 4;
+static_assert((kWarps * kStages + kWarps) * 8 <= 128, "the mbarrier area at the start of the shared tail holds 16 barriers");
 constexpr int kResidualWeight = 2;           // a 32-token unit of the residual window counts as this many packed units in the split
 constexpr uint32_t kSpinLimit = 1u << 22;    // bounded wait on a staged copy
 

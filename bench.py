@@ -1,9 +1,8 @@
 #!/usr/bin/env python
 """Benchmark of the MixKVQ decode hot path on B200.
 
-A step is one decode step of the whole path over all layers: for every layer `mixkvq_quantize_append`
-of the new token (which runs the scoring + quantize + pack flush once per R steps) followed by
-`mixkvq_decode_attention`.  The cache is pre-filled to the configured context with seeded synthetic
+A step is one decode step of the whole path over all layers: for every layer `mixkvq_decode_step`, i.e. the
+append of the new token (with the scoring + quantize + pack flush once per R steps) fused with decode attention.  The cache is pre-filled to the configured context with seeded synthetic
 tensors; all timed inputs are resident in HBM.  Prints one JSON line (rank 0).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config qwen7b|llama8b|tiny|...] [--impl reference]
@@ -250,8 +249,7 @@ def run_gpu(args, w):
     def step(i):
         for layer in range(w.n_layers):
             k, v, q = steps_in[layer][i]
-            cache.quantize_append(layer, k, v, q)
-            cache.decode_attention(layer, q.view(w.batch, w.n_q_heads, 128), scale, out=out[layer])
+            cache.decode_step(layer, k, v, q, scale, out=out[layer])
 
     def barrier():
         torch.cuda.synchronize()
@@ -330,8 +328,7 @@ def run_gpu(args, w):
     for i in range(n_e2e):
         dk.copy_(hk[i], non_blocking=True); dv.copy_(hv[i], non_blocking=True); dq.copy_(hq[i], non_blocking=True)
         for layer in range(w.n_layers):
-            cache.quantize_append(layer, dk[layer], dv[layer], dq[layer])
-            cache.decode_attention(layer, dq[layer].view(w.batch, w.n_q_heads, 128), scale, out=out[layer])
+            cache.decode_step(layer, dk[layer], dv[layer], dq[layer], scale, out=out[layer])
         hout.copy_(out, non_blocking=True)
         torch.cuda.synchronize()
     e2e_us = (time.perf_counter() - t0) / n_e2e * 1e6

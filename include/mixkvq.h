@@ -133,6 +133,14 @@ int mixkvq_quantize_append(mixkvq_cache* cache, int layer, const void* k_dev, co
 int mixkvq_decode_attention(mixkvq_cache* cache, int layer, const void* q_dev, float* out_dev, float softmax_scale,
                             void* workspace_dev, size_t workspace_bytes, void* stream);
 
+/* (2) + (3) fused for one decode step of `layer`: appends the step's token (k_dev, v_dev [B, Hkv, 1, 128],
+ * q_dev [B, Hq, 1, 128] bf16, flushing the residual window first if it is full) and attends with the same q_dev.
+ * The cache state and out_dev are exactly those of mixkvq_quantize_append(n_tokens = 1) followed by
+ * mixkvq_decode_attention; the attention kernel stores the token and updates the importance accumulator itself
+ * (Appendix D.1, D.2), which saves a kernel launch per layer. */
+int mixkvq_decode_step(mixkvq_cache* cache, int layer, const void* k_dev, const void* v_dev, const void* q_dev,
+                       float* out_dev, float softmax_scale, void* workspace_dev, size_t workspace_bytes, void* stream);
+
 /* (The paper has no counterpart of this entry point; it exists for integration reasons only.)
  * Same computation and same results as mixkvq_decode_attention, for callers that have no way to hand
  * over a workspace: code that runs inside a serving engine's pre-sized memory pool, a plugin that may

@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libmixkvq.so")
 EXPORTS = [
     "mixkvq_cache_bytes", "mixkvq_cache_init", "mixkvq_cache_destroy", "mixkvq_cache_reset",
     "mixkvq_select_channels", "mixkvq_select_channels_raw", "mixkvq_quantize_append",
-    "mixkvq_decode_attention", "mixkvq_decode_attention_noalloc", "mixkvq_set_attention_kernel", "mixkvq_query_status",
+    "mixkvq_decode_attention", "mixkvq_decode_attention_noalloc", "mixkvq_decode_step", "mixkvq_set_attention_kernel", "mixkvq_query_status",
     "mixkvq_cache_describe", "mixkvq_launch_count", "mixkvq_status_string",
 ]
 
@@ -67,6 +67,7 @@ def lib():
         L.mixkvq_quantize_append.argtypes = [vp, i32, vp, vp, vp, i32, vp]
         L.mixkvq_decode_attention.argtypes = [vp, i32, vp, vp, f32, vp, C.c_size_t, vp]
         L.mixkvq_decode_attention_noalloc.argtypes = [vp, i32, vp, vp, f32, vp]
+        L.mixkvq_decode_step.argtypes = [vp, i32, vp, vp, vp, vp, f32, vp, C.c_size_t, vp]
         L.mixkvq_set_attention_kernel.argtypes = [vp, i32]
         L.mixkvq_query_status.argtypes = [vp, C.POINTER(i32), vp]
         L.mixkvq_cache_describe.argtypes = [vp, i32, C.POINTER(LayoutDesc)]
@@ -165,6 +166,14 @@ class Cache:
         _check(lib().mixkvq_decode_attention(self.handle, layer, _ptr(q), _ptr(out), float(scale),
                                              _ptr(self.workspace), self.workspace.numel(), _stream()),
                "mixkvq_decode_attention")
+        return out
+
+    def decode_step(self, layer, k, v, q, scale, out=None):
+        """One decode step: k, v [B,Hkv,1,128], q [B,Hq,1,128] bf16 -> out [B,Hq,128] float32 (append + attention)."""
+        if out is None:
+            out = torch.empty((q.shape[0], q.shape[1], 128), dtype=torch.float32, device=q.device)
+        _check(lib().mixkvq_decode_step(self.handle, layer, _ptr(k), _ptr(v), _ptr(q), _ptr(out), float(scale),
+                                        _ptr(self.workspace), self.workspace.numel(), _stream()), "mixkvq_decode_step")
         return out
 
     def decode_attention_noalloc(self, layer, q, scale, out=None):

@@ -116,8 +116,11 @@ int zero_layer_state(mixkvq_cache* h, int layer, cudaStream_t st) {
 }
 
 // Picks the decode-attention kernel for the layer's layout and the selected kind, enqueues it and counts its launches.
-int run_attention(mixkvq_cache* h, int layer, const void* q, float* out, float scale, float* ws, cudaStream_t st) {
+int run_attention(mixkvq_cache* h, int layer, const void* q, float* out, float scale, float* ws, cudaStream_t st,
+                  const void* new_k = nullptr, const void* new_v = nullptr) {
   LayerView lv = view(h, layer);
+  lv.new_k = static_cast<const uint16_t*>(new_k);
+  lv.new_v = static_cast<const uint16_t*>(new_v);
   int launches = 0;
   cudaError_t e;
   if (h->attn_kind == 1)
@@ -258,6 +261,34 @@ int mixkvq_decode_attention(mixkvq_cache* cache, int layer, const void* q_dev, f
   if (cache->n_blocks[layer] == 0 && cache->r[layer] == 0) return MIXKVQ_E_EMPTY;
   return run_attention(cache, layer, q_dev, out_dev, softmax_scale, static_cast<float*>(workspace_dev),
                        static_cast<cudaStream_t>(stream));
+}
+
+int mixkvq_decode_step(mixkvq_cache* cache, int layer, const void* k_dev, const void* v_dev, const void* q_dev,
+                       float* out_dev, float softmax_scale, void* workspace_dev, size_t workspace_bytes_given,
+                       void* stream) {
+  if (!cache || !k_dev || !v_dev || !q_dev || !out_dev || !workspace_dev || layer < 0 || layer >= cache->cfg.n_layers)
+    return MIXKVQ_E_INVALID_ARG;
+  if (!aligned16(k_dev) || !aligned16(v_dev) || !aligned16(q_dev) || !aligned16(out_dev) || !aligned16(workspace_dev))
+    return MIXKVQ_E_ALIGNMENT;
+  if (workspace_bytes_given < workspace_bytes(cache->S)) return MIXKVQ_E_BUFFER_TOO_SMALL;
+  const long long have = (long long)cache->n_blocks[layer] * cache->R + cache->r[layer];
+  if (have + 1 > cache->cfg.max_tokens) return MIXKVQ_E_CAPACITY;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cache->attn_kind != 0) {
+    // the comparison kernels do not take the new token themselves: plain append, then attention
+    int rc = mixkvq_quantize_append(cache, layer, k_dev, v_dev, q_dev, 1, stream);
+    if (rc != MIXKVQ_OK) return rc;
+    return run_attention(cache, layer, q_dev, out_dev, softmax_scale, static_cast<float*>(workspace_dev), st);
+  }
+  if (cache->r[layer] == cache->R) {
+    LayerView lv = view(cache, layer);
+    if (launch_flush(lv, st) != cudaSuccess) return MIXKVQ_E_CUDA;
+    cache->launches += 1;
+    cache->n_blocks[layer] += 1;
+    cache->r[layer] = 0;
+  }
+  cache->r[layer] += 1;        // the attention kernel stores the token at slot r - 1 and accumulates |q|
+  return run_attention(cache, layer, q_dev, out_dev, softmax_scale, static_cast<float*>(workspace_dev), st, k_dev, v_dev);
 }
 
 // ---- decode attention with the split partials in storage compiled into the library (no allocation)

@@ -535,19 +535,41 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
       if ((xv - packed_units) % kResidualWeight != 0) continue;       // the warp owning a unit's first position runs it
       const int x = packed_units + (xv - packed_units) / kResidualWeight;
       const uint32_t rbar = smem_u32(&bars[kWarps * kStages + warp]);
+      // fused decode step: the newest token (slot r - 1) is not in the residual store yet; the warp whose unit holds it
+      // takes its rows from the step's tensors (into the staged tile and into the store) and updates the accumulator
+      const int jn = lv.r - 1;
+      const bool holds_new = lv.new_k != nullptr && jn >= (x - packed_units) * 32 && jn < (x - packed_units) * 32 + 32;
       {
-        const int j0s = (x - packed_units) * 32, nv = min(32, lv.r - j0s);
+        const int j0s = (x - packed_units) * 32, nv = min(32, lv.r - j0s) - (holds_new ? 1 : 0);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        if (lane == 0) {
-          mbar_expect_tx(rbar, (uint32_t)nv * 256u);
-          bulk_g2s(smem_u32(ring), resk + (size_t)j0s * kD, (uint32_t)nv * 256u, rbar);
+        if (nv > 0) {
+          if (lane == 0) {
+            mbar_expect_tx(rbar, (uint32_t)nv * 256u);
+            bulk_g2s(smem_u32(ring), resk + (size_t)j0s * kD, (uint32_t)nv * 256u, rbar);
+          }
+          if (!mbar_wait_bounded(rbar, res_phase)) {
+            gave_up = true;
+            if (lane == 0) atomicOr(lv.status, (uint32_t)MIXKVQ_DEV_COPY_TIMEOUT);
+            break;
+          }
+          res_phase ^= 1u;
         }
-        if (!mbar_wait_bounded(rbar, res_phase)) {
-          gave_up = true;
-          if (lane == 0) atomicOr(lv.status, (uint32_t)MIXKVQ_DEV_COPY_TIMEOUT);
-          break;
+        if (holds_new) {
+          const uint2 kn = reinterpret_cast<const uint2*>(lv.new_k + (size_t)s * kD)[lane];
+          reinterpret_cast<uint2*>(ring + (jn - j0s) * 256)[lane] = kn;
+          reinterpret_cast<uint2*>(lv.resk + (size_t)s * lv.resk_stride + (size_t)jn * 256)[lane] = kn;
+          // importance accumulator: channels 4*lane .. 4*lane+3, heads ascending (the order of the plain append)
+          double* acc = reinterpret_cast<double*>(lv.state + (size_t)s * lv.state_stride);
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const int d = 4 * lane + c;
+            double a = acc[d];
+            for (int h = 0; h < g; ++h) a = __dadd_rn(a, (double)fabsf(__uint_as_float((uint32_t)qb16[h * kD + d] << 16)));
+            acc[d] = a;
+          }
+          if (lane == 0) *reinterpret_cast<uint32_t*>(lv.state + (size_t)s * lv.state_stride + 1024) += (uint32_t)g;
+          __syncwarp();
         }
-        res_phase ^= 1u;
       }
       if (!o_true_scale) {
 #pragma unroll
@@ -611,17 +633,25 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
       // the key rows are consumed: stage the value rows of these 32 tokens over them
       __syncwarp();
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      const int nvv = min(32, rt - j0);
-      if (lane == 0) {
-        mbar_expect_tx(rbar, (uint32_t)nvv * 256u);
-        bulk_g2s(smem_u32(ring), resv + (size_t)j0 * kD, (uint32_t)nvv * 256u, rbar);
+      const int nvv = min(32, rt - j0) - (holds_new ? 1 : 0);
+      if (nvv > 0) {
+        if (lane == 0) {
+          mbar_expect_tx(rbar, (uint32_t)nvv * 256u);
+          bulk_g2s(smem_u32(ring), resv + (size_t)j0 * kD, (uint32_t)nvv * 256u, rbar);
+        }
+        if (!mbar_wait_bounded(rbar, res_phase)) {
+          gave_up = true;
+          if (lane == 0) atomicOr(lv.status, (uint32_t)MIXKVQ_DEV_COPY_TIMEOUT);
+          break;
+        }
+        res_phase ^= 1u;
       }
-      if (!mbar_wait_bounded(rbar, res_phase)) {
-        gave_up = true;
-        if (lane == 0) atomicOr(lv.status, (uint32_t)MIXKVQ_DEV_COPY_TIMEOUT);
-        break;
+      if (holds_new) {
+        const uint2 vn = reinterpret_cast<const uint2*>(lv.new_v + (size_t)s * kD)[lane];
+        reinterpret_cast<uint2*>(ring + (jn - j0) * 256)[lane] = vn;
+        reinterpret_cast<uint2*>(lv.resv + (size_t)s * lv.resv_stride + (size_t)jn * 256)[lane] = vn;
+        __syncwarp();
       }
-      res_phase ^= 1u;
       // tile (ct, ks): A = V^T, 16 channels x 16 tokens, from four transposed 8x8 tiles of the token-major rows:
       // matrix i of the ldmatrix has tokens 16ks + 8(i >> 1) .., channels 16ct + 8(i & 1) ..; lane l gives row l % 8 of matrix l / 8
       const uint32_t lm_row = smem_u32(ring) + (uint32_t)((8 * (lane >> 4) + (lane & 7)) * 256 + 16 * ((lane >> 3) & 1));

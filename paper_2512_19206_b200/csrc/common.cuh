@@ -39,6 +39,10 @@ struct LayerView {
   char* base;   uint64_t base_stride;
   char* extras; uint64_t extras_stride;
   uint32_t* status;           // sticky device status word
+  // fused decode step: the new token's key and value rows [S][128] (bf16 bits); null for plain attention.
+  // The attention kernel then stores them at residual slot r - 1 and adds |q| to the importance accumulator itself.
+  const uint16_t* new_k;
+  const uint16_t* new_v;
 };
 
 __host__ __device__ inline uint32_t extras_header_bytes(int n16, int n4) {

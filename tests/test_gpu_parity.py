@@ -268,3 +268,36 @@ def test_zero_keys_and_constant_groups(binding, layout):
         got = out[0, hk * w.g:(hk + 1) * w.g]
         assert float((got - mean_v[0, hk][None]).abs().max()) <= 1e-4
     assert cache.status() == 0
+
+
+# ------------------------------------------------------------------------------------------- fused decode step
+@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("kind", [0, 1])
+def test_decode_step_equals_append_then_attention(binding, kind, layout):
+    # 40 decode steps across a flush (the window fills at step 14): the fused entry point must leave the same bytes
+    # and give the same outputs as quantize_append(1) + decode_attention, and both must match the oracle
+    w = small("qwen7b", batch=2, tokens=2 * 128 + 114, **W.P27)
+    steps = 40
+    k, v, q = W.tokens(w, 0, 0, w.tokens + steps)
+    kc, vc, qc = k.cuda(), v.cuda(), q.cuda()
+    fused = U.make_cache(binding, w, max_tokens=w.tokens + steps + 8, layout=layout)
+    plain = U.make_cache(binding, w, max_tokens=w.tokens + steps + 8, layout=layout)
+    for c in (fused, plain):
+        c.quantize_append(0, kc[:, :, :w.tokens].contiguous(), vc[:, :, :w.tokens].contiguous(), qc[:, :, :w.tokens].contiguous())
+        c.set_attention_kernel(kind)
+    orc = U.oracle_streams(w, 0, k[:, :, :w.tokens], v[:, :, :w.tokens], q[:, :, :w.tokens])
+    for i in range(steps):
+        t = w.tokens + i
+        ks, vs, qs = (x[:, :, t:t + 1].contiguous() for x in (kc, vc, qc))
+        out_f = fused.decode_step(0, ks, vs, qs, W.softmax_scale())
+        plain.quantize_append(0, ks, vs, qs)
+        out_p = plain.decode_attention(0, qs.view(w.batch, w.n_q_heads, 128), W.softmax_scale())
+        assert float((out_f - out_p).abs().max()) <= 1e-6, i
+        for (b, hk), st in orc.items():
+            st.append(U.f32(k[b, hk, t]), U.f32(v[b, hk, t]), U.f32(q[b, hk * w.g:(hk + 1) * w.g, t]))
+        if i in (0, 13, 14, 15, steps - 1):
+            ref = U.oracle_attention(w, orc, q[:, :, t].contiguous())
+            assert U.max_abs_err(w, out_f, ref) <= ATTN_TOL, i
+    U.compare_regions(fused, 0, w, orc)
+    U.compare_regions(plain, 0, w, orc)
+    assert fused.status() == 0 and fused.describe(0).residual_tokens == plain.describe(0).residual_tokens

@@ -295,6 +295,16 @@ def extras_bytes(R, n16, n4):
     return 16 * ((2 * n16p + n4p + 15) // 16) + (R // 32) * (128 * n16p + 8 * n4p)
 
 
+def frag_meta_off(kg, G, unit_bytes):
+    """Fragment layout: byte offset of key-meta group kg inside the base block (directly before the group's first unit)."""
+    return kg * (G // 32) * unit_bytes + 512 * kg
+
+
+def frag_unit_off(u, G, unit_bytes):
+    """Fragment layout: byte offset of 32-token unit u inside the base block."""
+    return u * unit_bytes + 512 * ((u * 32) // G + 1)
+
+
 def _k_code_pos(jj, d):
     mt, row = divmod(jj, 16)
     rh, r = divmod(row, 8)
@@ -359,12 +369,15 @@ def pack_base(blk: Block, R, G):
     # K meta: entry (kg, d) at kg*512 + d*4 = {s, z}
     ks16 = np.where(quant[None, :], bf16_to_u16(blk.ks), 0).astype(np.uint32)
     kz16 = np.where(quant[None, :], bf16_to_u16(blk.kz), 0).astype(np.uint32)
-    words[:NG * 128] = (ks16 | (kz16 << 16)).reshape(NG * 128)
-    unit_words = (2048 + 128 * VG) // 4
+    unit_bytes = 2048 + 128 * VG
+    meta = ks16 | (kz16 << 16)                                   # entry (kg, d) at frag_meta_off(kg) + d*4
+    for kg in range(NG):
+        mo = frag_meta_off(kg, G, unit_bytes) // 4
+        words[mo:mo + 128] = meta[kg]
     vs16, vz16 = bf16_to_u16(blk.vs).astype(np.uint32), bf16_to_u16(blk.vz).astype(np.uint32)
     klow = np.where(quant[None, :], blk.kcodes & 3, 0)
     for u in range(U):
-        ubase = NG * 128 + u * unit_words
+        ubase = frag_unit_off(u, G, unit_bytes) // 4
         sl = slice(32 * u, 32 * u + 32)
         _scatter_codes(words, ubase + kw, kb, klow[sl])
         _scatter_codes(words, ubase + 256 + vw, vb, blk.vcodes[sl])
@@ -418,17 +431,17 @@ def unpack_base(buf, R, G):
     halves = np.frombuffer(buf, dtype="<u2")
     ks = np.zeros((NG, D), np.float32)
     kz = np.zeros((NG, D), np.float32)
+    unit_bytes = 2048 + 128 * VG
     for kg in range(NG):
         for d in range(D):
-            ks[kg, d] = u16_to_bf16(halves[(kg * 512 + d * 4) // 2])
-            kz[kg, d] = u16_to_bf16(halves[(kg * 512 + d * 4) // 2 + 1])
+            ks[kg, d] = u16_to_bf16(halves[(frag_meta_off(kg, G, unit_bytes) + d * 4) // 2])
+            kz[kg, d] = u16_to_bf16(halves[(frag_meta_off(kg, G, unit_bytes) + d * 4) // 2 + 1])
     klow = np.zeros((R, D), np.uint8)
     vcodes = np.zeros((R, D), np.uint8)
     vs = np.zeros((R, VG), np.float32)
     vz = np.zeros((R, VG), np.float32)
-    unit_bytes = 2048 + 128 * VG
     for u in range(U):
-        ubase = NG * 512 + u * unit_bytes
+        ubase = frag_unit_off(u, G, unit_bytes)
         for jj in range(32):
             j = 32 * u + jj
             for d in range(D):

@@ -25,8 +25,9 @@ namespace {
 
 constexpr int kWarps = 4;
 constexpr int kStages = 3;
-constexpr int kStageBytes = 3072;            // unit (<= 2560 B) followed by one key-meta group (512 B)
-constexpr int kKeyMetaOff = 2560;
+constexpr int kStageBytes = 3072;            // one key-meta group (512 B) followed by the unit (<= 2560 B), as in the block
+constexpr int kKeyMetaOff = 0;
+constexpr int kUnitOff = 512;
 constexpr int kPrepBytes = 1280;             // kprep 512 | zprep 256 | svp 256 | zvp 256
 constexpr int kSharedTail = 128 + 2048 + 2048 + 128 + 128 + 4096;
 constexpr int kSmemBytes = kWarps * (kStages * kStageBytes + kPrepBytes) + kSharedTail;
@@ -175,9 +176,14 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
       const uint32_t bar = smem_u32(&bars[warp * kStages + stage]);
       const uint32_t dst = smem_u32(ring + stage * kStageBytes);
       const bool meta = first || ((u * 32) % G == 0);
+      const bool group_start = (u * 32) % G == 0;       // then the group's scales lie directly before the unit: one copy
       mbar_expect_tx(bar, lv.unit_bytes + (meta ? 512u : 0u));
-      bulk_g2s(dst, blk + lv.NG * 512 + (size_t)u * lv.unit_bytes, lv.unit_bytes, bar);
-      if (meta) bulk_g2s(dst + kKeyMetaOff, blk + ((u * 32) / G) * 512, 512u, bar);
+      if (group_start) {
+        bulk_g2s(dst + kKeyMetaOff, blk + frag_meta_off((u * 32) / G, G, lv.unit_bytes), 512u + lv.unit_bytes, bar);
+      } else {
+        bulk_g2s(dst + kUnitOff, blk + frag_unit_off(u, G, lv.unit_bytes), lv.unit_bytes, bar);
+        if (meta) bulk_g2s(dst + kKeyMetaOff, blk + frag_meta_off((u * 32) / G, G, lv.unit_bytes), 512u, bar);
+      }
     };
     for (; !gave_up && issued < min(n_pack, kStages); ++issued) {
       if (lane == 0) issue(wb + issued, issued == 0);
@@ -268,12 +274,13 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
         break;
       }
       ++ring_count;
-      const unsigned char* st = ring + stage * kStageBytes;
+      const unsigned char* stg = ring + stage * kStageBytes;
+      const unsigned char* st = stg + kUnitOff;        // the unit's codes and value scales
       const bool has_meta = (i == 0) || ((u * 32) % G == 0);
 
       // ---- key-group preparation: fp16 scale pairs in fragment order, zero-point tile
       if (has_meta) {
-        const uint4 mz = reinterpret_cast<const uint4*>(st + kKeyMetaOff)[lane];   // channels 4*lane .. 4*lane+3
+        const uint4 mz = reinterpret_cast<const uint4*>(stg + kKeyMetaOff)[lane];   // channels 4*lane .. 4*lane+3
         const int kt = lane >> 2, ch = (lane & 3) >> 1, t0 = 2 * (lane & 1);
         const float zs = 1.0f / (float)(1 << (8 - key_pos(kt)));
         const uint32_t ma = pack_half2(bf_lo(mz.x), bf_lo(mz.y)), mb = pack_half2(bf_lo(mz.z), bf_lo(mz.w));

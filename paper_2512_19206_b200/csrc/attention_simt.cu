@@ -66,8 +66,9 @@ attention_simt_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float s
         __syncwarp();
       }
       const char* blk = base + (size_t)bi * lv.base_bytes;
-      ub_ptr = blk + lv.NG * 512 + (size_t)u * lv.unit_bytes;
-      const uint32_t* kmeta = reinterpret_cast<const uint32_t*>(blk + ((u * 32) / lv.G) * 512);
+      ub_ptr = blk + frag_unit_off(u, lv.G, lv.unit_bytes);
+      const uint32_t* kmeta = reinterpret_cast<const uint32_t*>(
+          blk + (lv.tile ? (uint32_t)((u * 32) / lv.G) * 512u : frag_meta_off((u * 32) / lv.G, lv.G, lv.unit_bytes)));
       const uint32_t* kcodes = reinterpret_cast<const uint32_t*>(ub_ptr);
       const char* exu = ex + extras_header_bytes(n16, n4) + (size_t)u * extras_unit_bytes(n16, n4);
       const int n16p = (n16 + 1) >> 1;

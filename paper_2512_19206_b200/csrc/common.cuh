@@ -54,6 +54,15 @@ __host__ __device__ inline uint32_t extras_unit_bytes(int n16, int n4) {
   return 128u * n16p + 8u * n4p;
 }
 
+// fragment layout: the key-meta group of G tokens sits directly before the first 32-token unit of those tokens, so a
+// unit and its group's scales are one contiguous piece
+__host__ __device__ inline uint32_t frag_meta_off(int kg, int G, uint32_t unit_bytes) {
+  return (uint32_t)(kg * (G / 32)) * unit_bytes + 512u * (uint32_t)kg;
+}
+__host__ __device__ inline uint32_t frag_unit_off(int u, int G, uint32_t unit_bytes) {
+  return (uint32_t)u * unit_bytes + 512u * (uint32_t)((u * 32) / G + 1);
+}
+
 // tile layout (R == 128): header [chan16: 2*n16p][chan4: 16*n4w][pad to 16], body (n16p + n4w) x 128 words
 __host__ __device__ inline uint32_t tile_extras_header_bytes(int n16, int n4) {
   int n16p = (n16 + 1) >> 1, n4w = (n4 + 15) >> 4;

@@ -144,7 +144,7 @@ flush_kernel(LayerView lv, BulkSrc src) {
           cS[j * kD + d] = (uint8_t)quant_code(bf16_bits_to_float(kS[j * kD + d]), gmn, sc, max_code);
         meta = float_to_bf16_bits_exact(sc) | (float_to_bf16_bits_exact(gmn) << 16);
       }
-      reinterpret_cast<uint32_t*>(blk + kg * 512)[d] = meta;
+      reinterpret_cast<uint32_t*>(blk + (lv.tile ? (uint32_t)kg * 512u : frag_meta_off(kg, G, lv.unit_bytes)))[d] = meta;
     }
   }
   __syncthreads();
@@ -241,7 +241,7 @@ flush_kernel(LayerView lv, BulkSrc src) {
           const int d = kt * 16 + ch * 8 + 2 * t + e;
           w |= (uint32_t)(cS[j * kD + d] & 3) << (16 * e + 2 * kt);
         }
-      reinterpret_cast<uint32_t*>(blk + NG * 512 + (size_t)u * lv.unit_bytes)[wi] = w;
+      reinterpret_cast<uint32_t*>(blk + frag_unit_off(u, G, lv.unit_bytes))[wi] = w;
     }
     // ---- extras: header, BF16 pairs, UINT4 high plane
     for (int i = tid; i < (int)hdr; i += 256) {
@@ -285,7 +285,7 @@ flush_kernel(LayerView lv, BulkSrc src) {
   auto vmeta_of = [&](int j) -> uint32_t* {
     const int u = j >> 5, jj = j & 31;
     return lv.tile ? reinterpret_cast<uint32_t*>(blk + NG * 512 + 8192) + j * VG
-                   : reinterpret_cast<uint32_t*>(blk + NG * 512 + (size_t)u * lv.unit_bytes + 2048) + jj * VG;
+                   : reinterpret_cast<uint32_t*>(blk + frag_unit_off(u, G, lv.unit_bytes) + 2048) + jj * VG;
   };
   {
     // token-major window: a warp takes a token, lane l the channels l, l+32, l+64, l+96; group extrema by shuffles
@@ -349,7 +349,7 @@ flush_kernel(LayerView lv, BulkSrc src) {
               const int j = 32 * u + ks * 16 + ch * 8 + 2 * t + e;
               w |= (uint32_t)cS[j * kD + c] << (16 * e + 2 * (4 * rh + 2 * ks + ch));
             }
-      reinterpret_cast<uint32_t*>(blk + NG * 512 + (size_t)u * lv.unit_bytes + 1024)[wi] = w;
+      reinterpret_cast<uint32_t*>(blk + frag_unit_off(u, G, lv.unit_bytes) + 1024)[wi] = w;
     }
   }
 

@@ -213,3 +213,17 @@ def test_stream_regions(rng):
     assert int.from_bytes(p["state"][1028:1032], "little") == off
     assert len(p["resK"]) == 5 * 256 and len(p["resV"]) == 5 * 256
     assert np.array_equal(np.frombuffer(p["resV"], "<u2").reshape(5, 128), O.bf16_to_u16(v[-5:]))
+
+
+def test_fragment_layout_places_each_scale_group_before_its_first_unit():
+    # G = 32: [meta 0][unit 0][meta 1][unit 1]...; G = 128: [meta 0][unit 0][unit 1][unit 2][unit 3]
+    assert [O.frag_meta_off(kg, 32, 2560) for kg in range(4)] == [0, 3072, 6144, 9216]
+    assert [O.frag_unit_off(u, 32, 2560) for u in range(4)] == [512, 3584, 6656, 9728]
+    assert O.frag_meta_off(0, 128, 2176) == 0 and [O.frag_unit_off(u, 128, 2176) for u in range(4)] == [512, 2688, 4864, 7040]
+    # R = 256, G = 64: a group covers two units
+    assert [O.frag_meta_off(kg, 64, 2304) for kg in range(4)] == [0, 5120, 10240, 15360]
+    assert [O.frag_unit_off(u, 64, 2304) for u in range(8)] == [512, 2816, 5632, 7936, 10752, 13056, 15872, 18176]
+    for G, ub, U in ((32, 2560, 4), (64, 2304, 8), (128, 2176, 4)):
+        spans = sorted([(O.frag_meta_off(kg, G, ub), 512) for kg in range(U * 32 // G)] + [(O.frag_unit_off(u, G, ub), ub) for u in range(U)])
+        assert spans[0][0] == 0 and all(a + n == b for (a, n), (b, _) in zip(spans, spans[1:]))      # a partition of the block
+        assert spans[-1][0] + spans[-1][1] == O.base_bytes(U * 32, G)

@@ -124,7 +124,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+                                          "-lms", "50", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
         except Exception:
             self.proc = None
 
@@ -377,7 +377,7 @@ def run_gpu(args, w):
         "clocks": clocks,
     }
     if world == 1 and not args.no_cpu_baseline:
-        sec, desc = oracle_sample(w, n_streams=2, reps=3)
+        sec, desc = oracle_sample(w, n_streams=8, reps=5)
         n_streams = w.n_layers * w.batch * w.n_kv_heads
         line["cpu_baseline"] = {"value": sec * n_streams * 1e6, "unit": "us/step", "cores": oracle_threads(),
                                 "kind": "oracle", "sample": desc}

@@ -1,7 +1,8 @@
 """CPU oracle for the MixKVQ decode hot path.  TEST INFRASTRUCTURE ONLY.
 
 A plain, slow, obviously-correct numpy restatement of what the method computes, written from the
-paper (arxiv 2512.19206) and from the byte layout text of this repository's design document.  It
+paper (arxiv 2512.19206) and from the written definition of the byte layouts (every position function below
+states its formula).  It
 shares no code with the CUDA path and must never be imported by the product package; only the
 tests, the smoke check and the CPU-baseline leg of the benchmark may call it.
 
@@ -283,7 +284,7 @@ def unquantized_attention(q, K, V, scale):
 
 
 # --------------------------------------------------------------------------------------------
-# byte layout (written from the layout section of the design document, one element at a time)
+# byte layout (one element at a time, from the stated position formulas)
 # fragment layout (the default): blocks of any R
 # --------------------------------------------------------------------------------------------
 def base_bytes(R, G):

@@ -106,7 +106,8 @@ __device__ inline uint8_t salience_tier(double acc, uint32_t cnt, float mx, floa
   return kU2;
 }
 
-// ---- layout: positions inside a unit (see the layout description in the repository's design notes)
+// ---- fragment layout: positions inside a 32-token unit.  The codes are ordered so that one 16-byte load per lane
+// yields the four A-operand registers of an m16n8k16 tile for all eight 16-channel k-tiles.
 // K low-plane code of (token jj in unit, channel d): 32-bit word index inside the unit's K codes, bit offset.
 __host__ __device__ inline void k_code_pos(int jj, int d, int* word, int* bit) {
   int mt = jj >> 4, row = jj & 15, r = row & 7, rh = row >> 3;

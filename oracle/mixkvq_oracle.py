@@ -291,9 +291,16 @@ def base_bytes(R, G):
     return (R // G) * 512 + (R // 32) * (2048 + 128 * (D // G))
 
 
-def extras_bytes(R, n16, n4):
+def dense_high_plane(tau_u4):
+    """4-bit base precision (tau_u4 < 0: no channel stays at 2 bits): the high plane of every block is a full
+    1024-byte plane per unit in the low plane's bit order instead of 16 bytes per UINT4 channel pair."""
+    return tau_u4 < 0
+
+
+def extras_bytes(R, n16, n4, dense=False):
     n16p, n4p = (n16 + 1) // 2, 2 * ((n4 + 1) // 2)
-    return 16 * ((2 * n16p + n4p + 15) // 16) + (R // 32) * (128 * n16p + 8 * n4p)
+    hi = 1024 if dense else 8 * n4p
+    return 16 * ((2 * n16p + n4p + 15) // 16) + (R // 32) * (128 * n16p + hi)
 
 
 def frag_meta_off(kg, G, unit_bytes):
@@ -392,13 +399,13 @@ def channel_lists(tiers):
     return chan16, chan4
 
 
-def pack_extras(blk: Block, R):
+def pack_extras(blk: Block, R, dense=False):
     U = R // 32
     _, _, _, _, hw, hb = _tables()
     chan16, chan4 = channel_lists(blk.tiers)
     n16, n4 = len(chan16), len(chan4)
     n16p, n4p = (n16 + 1) // 2, 2 * ((n4 + 1) // 2)
-    total = extras_bytes(R, n16, n4)
+    total = extras_bytes(R, n16, n4, dense)
     hdr = 16 * ((2 * n16p + n4p + 15) // 16)
     head = bytearray(hdr)
     l16 = chan16 + [0xFF] * (2 * n16p - n16)
@@ -406,7 +413,9 @@ def pack_extras(blk: Block, R):
     head[0:2 * n16p] = bytes(l16)
     head[2 * n16p:2 * n16p + n4p] = bytes(l4)
     words = np.zeros((total - hdr) // 4, np.uint32)
-    unit_words = (128 * n16p + 8 * n4p) // 4
+    unit_words = (128 * n16p + (1024 if dense else 8 * n4p)) // 4
+    kw, kb = _tables()[0], _tables()[1]
+    khigh = np.where((blk.tiers == TIER_U4)[None, :], blk.kcodes >> 2, 0)
     raw16 = bf16_to_u16(blk.kraw).astype(np.uint32)
     for u in range(U):
         ubase = u * unit_words
@@ -416,6 +425,9 @@ def pack_extras(blk: Block, R):
             hi = raw16[sl, l16[2 * i + 1]] if l16[2 * i + 1] != 0xFF else np.zeros(32, np.uint32)
             words[ubase + i * 32:ubase + i * 32 + 32] = lo | (hi << 16)       # word (i*32 + jj)
         hbase = ubase + 32 * n16p
+        if dense:                                   # the low plane's positions, code >> 2 of UINT4 channels, 0 elsewhere
+            _scatter_codes(words, hbase + kw, kb, khigh[sl])
+            continue
         for i in range(n4p // 2):
             for e in range(2):
                 ch = l4[2 * i + e]
@@ -577,7 +589,7 @@ def pack_stream(st: OracleStream, layout=LAYOUT_FRAGMENT):
             ex, n16, n4 = pack_extras_tile(blk)
         else:
             base.append(pack_base(blk, st.R, st.G))
-            ex, n16, n4 = pack_extras(blk, st.R)
+            ex, n16, n4 = pack_extras(blk, st.R, dense_high_plane(st.tau_u4))
         table.append(table_entry(used16, n16, n4))
         extras.append(ex)
         used16 += len(ex) // 16

@@ -90,6 +90,7 @@ LayerView view(const mixkvq_cache* h, int layer) {
   v.max_blocks = h->max_blocks;
   v.n_blocks = h->n_blocks[layer]; v.r = h->r[layer];
   v.tile = h->tile;
+  v.dense_hi = (h->cfg.tau_u4 < 0.0f) ? 1 : 0;
   v.base_bytes = h->base_bytes; v.unit_bytes = h->unit_bytes;
   v.extras_budget = h->extras_budget;
   v.score_bits = h->cfg.score_bits; v.importance_mode = h->cfg.importance_mode;

@@ -113,7 +113,7 @@ __device__ __forceinline__ constexpr int key_pos(int kt) { return (0x86486464u >
 // k-tiles 0,1 are read from (w << 4), 2..4 from w, 5..7 from (w >> 6)
 __device__ __forceinline__ uint32_t key_shift(uint32_t w, int kt) { return kt < 2 ? (w << 4) : (kt < 5 ? w : (w >> 6)); }
 
-template <int G>
+template <int G, bool kDenseHi>
 __global__ void __launch_bounds__(kWarps * 32, kCtasPerSm)
 attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float scale_log2e, float* __restrict__ ws) {
   constexpr int VG = kD / G;              // value groups per token
@@ -253,7 +253,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
         n16p = (n16 + 1) >> 1;
         ex = extras + (size_t)entry.x * 16;
         ex_hdr = extras_header_bytes(n16, n4);
-        ex_unit = extras_unit_bytes(n16, n4);
+        ex_unit = extras_unit_bytes(n16, n4, kDenseHi);
         // the block's promoted channels are the same for its units: gather their query entries once
         xb0 = xb1 = 0u;
         if (n16 > 0) {
@@ -346,6 +346,30 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
           }
         }
       }
+      // ---- dense UINT4 high plane: the same tiles with codes c >> 2 and four times the scale
+      if constexpr (kDenseHi) {
+        // laid out like the low plane: two 16-byte loads per lane
+        const uint4* hp = reinterpret_cast<const uint4*>(exu + 128 * n16p);
+        const uint4 hw0 = hp[lane], hw1 = hp[32 + lane];
+        const uint32_t kw[2][4] = {{hw0.x, hw0.y, hw0.z, hw0.w}, {hw1.x, hw1.y, hw1.z, hw1.w}};
+#pragma unroll
+        for (int kt = 0; kt < 8; ++kt) {
+          const uint4 kp = *reinterpret_cast<const uint4*>(&kprep[(kt * 4 + t) * 4]);
+          const uint32_t m0 = hmul2_u(kp.x, 0x44004400u), o0 = hmul2_u(kp.y, 0x44004400u);
+          const uint32_t m1 = hmul2_u(kp.z, 0x44004400u), o1 = hmul2_u(kp.w, 0x44004400u);
+          const uint32_t mask = 0x00030003u << key_pos(kt);
+#pragma unroll
+          for (int mt = 0; mt < 2; ++mt) {
+            uint32_t a[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const uint32_t code = (key_shift(kw[mt][j], kt) & mask) | 0x44004400u;
+              a[j] = hfma2_u(code, j < 2 ? m0 : m1, j < 2 ? o0 : o1);
+            }
+            mma_f16(Sx[mt], a[0], a[1], a[2], a[3], bq[kt][0], bq[kt][1]);
+          }
+        }
+      }
       // ---- promoted channels (raw bf16 keys) with a gathered q
       if (n16 > 0) {
         for (int kk = 0; kk * 8 < n16p; ++kk) {
@@ -388,7 +412,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
         }
       }
       // ---- UINT4 high plane: c_hi * 4s, gathered q in fp16
-      if (n4 > 0) {
+      if (!kDenseHi && n4 > 0) {
         const int n4pairs = (n4 + 1) >> 1;
         const uint32_t* hw = reinterpret_cast<const uint32_t*>(exu + 128 * n16p);
         const unsigned char* ids4 = reinterpret_cast<const unsigned char*>(ex) + 2 * n16p;
@@ -743,20 +767,30 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
 
 template <int G>
 cudaError_t launch_g(const LayerView& lv, const void* q, float scale, float* ws, int grid, cudaStream_t stream) {
-  attention_mma_kernel<G><<<grid, kWarps * 32, kSmemBytes, stream>>>(lv, static_cast<const __nv_bfloat16*>(q),
-                                                                     scale * 1.4426950408889634f, ws);
+  if (lv.dense_hi)
+    attention_mma_kernel<G, true><<<grid, kWarps * 32, kSmemBytes, stream>>>(lv, static_cast<const __nv_bfloat16*>(q),
+                                                                             scale * 1.4426950408889634f, ws);
+  else
+    attention_mma_kernel<G, false><<<grid, kWarps * 32, kSmemBytes, stream>>>(lv, static_cast<const __nv_bfloat16*>(q),
+                                                                              scale * 1.4426950408889634f, ws);
   return cudaGetLastError();
 }
 
 }  // namespace
 
-template <int G>
-static cudaError_t setup_g() {
-  cudaError_t e = cudaFuncSetAttribute(attention_mma_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+template <int G, bool kDenseHi>
+static cudaError_t setup_one() {
+  cudaError_t e = cudaFuncSetAttribute(attention_mma_kernel<G, kDenseHi>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kSmemBytes);
   if (e != cudaSuccess) return e;
   // kCtasPerSm CTAs only fit with the largest shared-memory carve-out; ask for it explicitly
-  return cudaFuncSetAttribute(attention_mma_kernel<G>, cudaFuncAttributePreferredSharedMemoryCarveout,
+  return cudaFuncSetAttribute(attention_mma_kernel<G, kDenseHi>, cudaFuncAttributePreferredSharedMemoryCarveout,
                               (int)cudaSharedmemCarveoutMaxShared);
+}
+template <int G>
+static cudaError_t setup_g() {
+  cudaError_t e = setup_one<G, false>();
+  return e != cudaSuccess ? e : setup_one<G, true>();
 }
 
 cudaError_t attention_mma_setup() {

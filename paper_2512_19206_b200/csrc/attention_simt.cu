@@ -70,7 +70,7 @@ attention_simt_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float s
       const uint32_t* kmeta = reinterpret_cast<const uint32_t*>(
           blk + (lv.tile ? (uint32_t)((u * 32) / lv.G) * 512u : frag_meta_off((u * 32) / lv.G, lv.G, lv.unit_bytes)));
       const uint32_t* kcodes = reinterpret_cast<const uint32_t*>(ub_ptr);
-      const char* exu = ex + extras_header_bytes(n16, n4) + (size_t)u * extras_unit_bytes(n16, n4);
+      const char* exu = ex + extras_header_bytes(n16, n4) + (size_t)u * extras_unit_bytes(n16, n4, lv.dense_hi != 0);
       const int n16p = (n16 + 1) >> 1;
       // tile layout (R == 128): planes of the whole block, token j of the block
       const int jt = 32 * u + lane;
@@ -97,7 +97,9 @@ attention_simt_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float s
             int word, bit;
             k_code_pos(lane, d, &word, &bit);
             code = (kcodes[word] >> bit) & 3;
-            if (s4 != 0xFF) {
+            if (s4 != 0xFF && lv.dense_hi) {
+              code += 4 * ((reinterpret_cast<const uint32_t*>(exu + 128 * n16p)[word] >> bit) & 3);
+            } else if (s4 != 0xFF) {
               int hw, hb;
               hi_plane_pos(lane, s4 & 1, &hw, &hb);
               const uint32_t w = reinterpret_cast<const uint32_t*>(exu + 128 * n16p)[(s4 >> 1) * 4 + hw];

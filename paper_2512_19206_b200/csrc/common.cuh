@@ -26,6 +26,7 @@ struct LayerView {
   int max_blocks;
   int n_blocks, r;            // current fill (same for all streams)
   int tile;                   // 1: tile layout (R == 128 only), 0: fragment layout
+  int dense_hi;               // 1: 4-bit base (tau_u4 < 0): dense UINT4 high plane in the fragment layout
   uint32_t base_bytes, unit_bytes;
   uint64_t extras_budget;     // bytes per stream
   // method parameters
@@ -49,9 +50,13 @@ __host__ __device__ inline uint32_t extras_header_bytes(int n16, int n4) {
   int n16p = (n16 + 1) >> 1, n4p = ((n4 + 1) >> 1) << 1;
   return 16u * ((2 * n16p + n4p + 15) >> 4);
 }
-__host__ __device__ inline uint32_t extras_unit_bytes(int n16, int n4) {
+// With a 4-bit base precision (tau_u4 < 0: every channel that is not promoted is UINT4) the high plane of a block is
+// stored densely: 1024 bytes per unit in the bit order of the low plane (zero where the channel is BF16) instead of
+// 16 bytes per channel pair, so that the attention kernel runs it through the low plane's code path without gathering
+// scales and query entries.  `dense` is a property of the cache's configuration, the same for all its blocks.
+__host__ __device__ inline uint32_t extras_unit_bytes(int n16, int n4, bool dense) {
   int n16p = (n16 + 1) >> 1, n4p = ((n4 + 1) >> 1) << 1;
-  return 128u * n16p + 8u * n4p;
+  return 128u * n16p + (dense ? 1024u : 8u * n4p);
 }
 
 // fragment layout: the key-meta group of G tokens sits directly before the first 32-token unit of those tokens, so a

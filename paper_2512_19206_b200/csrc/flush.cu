@@ -20,7 +20,7 @@ struct BulkSrc {
 
 __host__ __device__ inline uint32_t flush_extras_bytes(const LayerView& lv, int n16, int n4) {
   return lv.tile ? tile_extras_header_bytes(n16, n4) + tile_extras_body_bytes(n16, n4)
-                 : extras_header_bytes(n16, n4) + (uint32_t)lv.U * extras_unit_bytes(n16, n4);
+                 : extras_header_bytes(n16, n4) + (uint32_t)lv.U * extras_unit_bytes(n16, n4, lv.dense_hi != 0);
 }
 
 // Bulk append, between the two passes: one thread per stream walks the new blocks in order, gives each its offset in
@@ -190,7 +190,7 @@ flush_kernel(LayerView lv, BulkSrc src) {
   const int n16 = misc[0], n4 = misc[1];
   const int n16p = (n16 + 1) >> 1, n4p = ((n4 + 1) >> 1) << 1;
   char* ex = lv.extras + (size_t)s * lv.extras_stride + (size_t)misc[2] * 16;
-  const uint32_t hdr = extras_header_bytes(n16, n4), exunit = extras_unit_bytes(n16, n4);
+  const uint32_t hdr = extras_header_bytes(n16, n4), exunit = extras_unit_bytes(n16, n4, lv.dense_hi != 0);
 
   if (lv.tile) {
     // ---- tile layout (R = 128): a token's key codes are 32 contiguous bytes (two 16-byte halves)
@@ -257,7 +257,25 @@ flush_kernel(LayerView lv, BulkSrc src) {
       if (2 * p + 1 < n16) w |= (uint32_t)kS[j * kD + chan16S[2 * p + 1]] << 16;
       reinterpret_cast<uint32_t*>(ex + hdr + (size_t)u * exunit)[rem] = w;
     }
-    for (int i = tid; i < U * (n4p / 2) * 4; i += 256) {
+    if (lv.dense_hi) {
+      // dense high plane: the low plane's fragment order, code >> 2 of UINT4 channels, 0 elsewhere
+      for (int i = tid; i < U * 256; i += 256) {
+        const int u = i >> 8, wi = i & 255;
+        const int mt = wi >> 7, lane = (wi >> 2) & 31, a = wi & 3;
+        const int r = lane >> 2, t = lane & 3, ch = a >> 1, rh = a & 1;
+        const int j = 32 * u + mt * 16 + rh * 8 + r;
+        uint32_t w = 0;
+#pragma unroll
+        for (int kt = 0; kt < 8; ++kt)
+#pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            const int d = kt * 16 + ch * 8 + 2 * t + e;
+            if (tierS[d] == kU4) w |= (uint32_t)(cS[j * kD + d] >> 2) << (16 * e + 2 * kt);
+          }
+        reinterpret_cast<uint32_t*>(ex + hdr + (size_t)u * exunit + 128 * n16p)[wi] = w;
+      }
+    }
+    for (int i = tid; i < (lv.dense_hi ? 0 : U * (n4p / 2) * 4); i += 256) {
       const int u = i / (n4p * 2), rem = i % (n4p * 2), p = rem >> 2, wj = rem & 3;
       uint32_t w = 0;
       for (int e = 0; e < 2; ++e) {

@@ -87,7 +87,7 @@ def _flushed(rng, R, G, tau16=6.0, tau4=3.0):
 
 @pytest.mark.parametrize("R,G", [(128, 32), (128, 64), (128, 128), (64, 32), (256, 128)])
 def test_pack_roundtrip_and_sizes(rng, R, G):
-    st, k, v = _flushed(rng, R, G)
+    st, k, v = _flushed(rng, R, G, tau4=1.0)
     blk = st.blocks[0]
     n16, n4 = int((blk.tiers == 2).sum()), int((blk.tiers == 1).sum())
     assert n16 >= 3 and n4 >= 5
@@ -99,18 +99,34 @@ def test_pack_roundtrip_and_sizes(rng, R, G):
     assert not klow[:, ~quant].any() and not ks[:, ~quant].any() and not kz[:, ~quant].any()
     assert np.array_equal(ks[:, quant], blk.ks[:, quant]) and np.array_equal(kz[:, quant], blk.kz[:, quant])
     assert np.array_equal(vc, blk.vcodes) and np.array_equal(vs, blk.vs) and np.array_equal(vz, blk.vz)
-    ex, a, b = O.pack_extras(blk, R)
+    ex, a, b = O.pack_extras(blk, R, dense=True)                      # the 4-bit-base form of the high plane
     n16p, n4p = (n16 + 1) // 2, 2 * ((n4 + 1) // 2)
-    assert (a, b) == (n16, n4)
-    assert len(ex) == 16 * ((2 * n16p + n4p + 15) // 16) + (R // 32) * (128 * n16p + 8 * n4p)
+    assert (a, b) == (n16, n4) and O.dense_high_plane(-1.0) and not O.dense_high_plane(3.8)
+    assert len(ex) == 16 * ((2 * n16p + n4p + 15) // 16) + (R // 32) * (128 * n16p + 1024)
     assert len(ex) % 16 == 0
+    # dense high plane: code >> 2 of a UINT4 channel sits where the low plane keeps the channel's low bits
+    hdr = 16 * ((2 * n16p + n4p + 15) // 16)
+    words = np.frombuffer(ex[hdr:], "<u4")
+    unit_words = (128 * n16p + 1024) // 4
+    for (j, d) in [(0, 0), (33, 17), (R - 1, 127), (40, 64), (5, 99)]:
+        u, jj = divmod(j, 32)
+        off, bit = O._k_code_pos(jj, d)
+        got = (int(words[u * unit_words + 32 * n16p + off // 4]) >> bit) & 3
+        assert got == (blk.kcodes[j, d] >> 2 if blk.tiers[d] == O.TIER_U4 else 0)
+    st2, _, _ = _flushed(rng, R, G, tau4=4.5)                         # few UINT4 channels: 16 bytes per channel pair
+    blk2 = st2.blocks[0]
+    m16, m4 = int((blk2.tiers == 2).sum()), int((blk2.tiers == 1).sum())
+    assert m4 > 0
+    assert len(O.pack_extras(blk2, R)[0]) == 16 * ((2 * ((m16 + 1) // 2) + 2 * ((m4 + 1) // 2) + 15) // 16) + (R // 32) * (
+        128 * ((m16 + 1) // 2) + 8 * 2 * ((m4 + 1) // 2))
 
 
 def test_extras_content_by_hand(rng):
     R, G = 128, 32
-    st, k, v = _flushed(rng, R, G)
+    st, k, v = _flushed(rng, R, G, tau4=4.5)
     blk = st.blocks[0]
     ex, n16, n4 = O.pack_extras(blk, R)
+    assert 5 <= n4
     chan16 = [d for d in range(128) if blk.tiers[d] == 2]
     chan4 = [d for d in range(128) if blk.tiers[d] == 1]
     n16p, n4p = (n16 + 1) // 2, 2 * ((n4 + 1) // 2)

@@ -113,7 +113,9 @@ __device__ __forceinline__ constexpr int key_pos(int kt) { return (0x86486464u >
 // k-tiles 0,1 are read from (w << 4), 2..4 from w, 5..7 from (w >> 6)
 __device__ __forceinline__ uint32_t key_shift(uint32_t w, int kt) { return kt < 2 ? (w << 4) : (kt < 5 ? w : (w >> 6)); }
 
-template <int G, bool kDenseHi>
+// kU4: how the configuration can use the UINT4 tier: 0 = never (tau_u4 >= tau_bf16), 1 = some channels (high plane stored
+// per channel pair, gathered), 2 = 4-bit base (dense high plane)
+template <int G, int kU4>
 __global__ void __launch_bounds__(kWarps * 32, kCtasPerSm)
 attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float scale_log2e, float* __restrict__ ws) {
   constexpr int VG = kD / G;              // value groups per token
@@ -253,7 +255,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
         n16p = (n16 + 1) >> 1;
         ex = extras + (size_t)entry.x * 16;
         ex_hdr = extras_header_bytes(n16, n4);
-        ex_unit = extras_unit_bytes(n16, n4, kDenseHi);
+        ex_unit = extras_unit_bytes(n16, n4, kU4 == 2);
         // the block's promoted channels are the same for its units: gather their query entries once
         xb0 = xb1 = 0u;
         if (n16 > 0) {
@@ -347,7 +349,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
         }
       }
       // ---- dense UINT4 high plane: the same tiles with codes c >> 2 and four times the scale
-      if constexpr (kDenseHi) {
+      if constexpr (kU4 == 2) {
         // laid out like the low plane: two 16-byte loads per lane
         const uint4* hp = reinterpret_cast<const uint4*>(exu + 128 * n16p);
         const uint4 hw0 = hp[lane], hw1 = hp[32 + lane];
@@ -412,7 +414,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
         }
       }
       // ---- UINT4 high plane: c_hi * 4s, gathered q in fp16
-      if (!kDenseHi && n4 > 0) {
+      if (kU4 == 1 && n4 > 0) {
         const int n4pairs = (n4 + 1) >> 1;
         const uint32_t* hw = reinterpret_cast<const uint32_t*>(exu + 128 * n16p);
         const unsigned char* ids4 = reinterpret_cast<const unsigned char*>(ex) + 2 * n16p;
@@ -767,30 +769,31 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
 
 template <int G>
 cudaError_t launch_g(const LayerView& lv, const void* q, float scale, float* ws, int grid, cudaStream_t stream) {
-  if (lv.dense_hi)
-    attention_mma_kernel<G, true><<<grid, kWarps * 32, kSmemBytes, stream>>>(lv, static_cast<const __nv_bfloat16*>(q),
-                                                                             scale * 1.4426950408889634f, ws);
-  else
-    attention_mma_kernel<G, false><<<grid, kWarps * 32, kSmemBytes, stream>>>(lv, static_cast<const __nv_bfloat16*>(q),
-                                                                              scale * 1.4426950408889634f, ws);
+  const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q);
+  const float sl = scale * 1.4426950408889634f;
+  if (lv.dense_hi) attention_mma_kernel<G, 2><<<grid, kWarps * 32, kSmemBytes, stream>>>(lv, qb, sl, ws);
+  else if (lv.tau_u4 < lv.tau_bf16) attention_mma_kernel<G, 1><<<grid, kWarps * 32, kSmemBytes, stream>>>(lv, qb, sl, ws);
+  else attention_mma_kernel<G, 0><<<grid, kWarps * 32, kSmemBytes, stream>>>(lv, qb, sl, ws);
   return cudaGetLastError();
 }
 
 }  // namespace
 
-template <int G, bool kDenseHi>
+template <int G, int kU4>
 static cudaError_t setup_one() {
-  cudaError_t e = cudaFuncSetAttribute(attention_mma_kernel<G, kDenseHi>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(attention_mma_kernel<G, kU4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        kSmemBytes);
   if (e != cudaSuccess) return e;
   // kCtasPerSm CTAs only fit with the largest shared-memory carve-out; ask for it explicitly
-  return cudaFuncSetAttribute(attention_mma_kernel<G, kDenseHi>, cudaFuncAttributePreferredSharedMemoryCarveout,
+  return cudaFuncSetAttribute(attention_mma_kernel<G, kU4>, cudaFuncAttributePreferredSharedMemoryCarveout,
                               (int)cudaSharedmemCarveoutMaxShared);
 }
 template <int G>
 static cudaError_t setup_g() {
-  cudaError_t e = setup_one<G, false>();
-  return e != cudaSuccess ? e : setup_one<G, true>();
+  cudaError_t e = setup_one<G, 0>();
+  if (e != cudaSuccess) return e;
+  e = setup_one<G, 1>();
+  return e != cudaSuccess ? e : setup_one<G, 2>();
 }
 
 cudaError_t attention_mma_setup() {

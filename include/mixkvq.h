@@ -67,7 +67,8 @@ typedef struct mixkvq_config {
   float tau_bf16;                     /* A_d >  tau_bf16            -> BF16                          */
   float tau_u4;                       /* tau_u4 < A_d <= tau_bf16   -> UINT4, else UINT2             */
   int32_t importance_mode;            /* 0: |q| accumulated within the current window (Section 4.2);
-                                         1: cumulative over the whole history (Appendix D.2)         */
+                                         1: cumulative over the whole history (Appendix D.2);
+                                         2: error-only ablation (Appendix E): I_d = 1, A_d = S_d     */
   int32_t block_layout;               /* 0: fragment layout (any R; mma.sync attention kernel), the default;
                                          1: tile layout (R must be 128; tcgen05 attention kernel)        */
   uint64_t extras_budget_bytes;       /* per stream, for promoted channels; 0 = library default

@@ -201,7 +201,10 @@ class OracleStream:
             t += m
 
     def current_scores(self):
-        return salience(self.acc, self.cnt, self.resK[:self.r], self.score_bits)
+        I, S, A = salience(self.acc, self.cnt, self.resK[:self.r], self.score_bits)
+        if self.importance_mode == 2:          # error-only ablation of the paper: the query term is dropped, A = S
+            return np.ones_like(I), S, S.copy()
+        return I, S, A
 
     def current_tiers(self):
         _, _, A = self.current_scores()
@@ -231,7 +234,7 @@ class OracleStream:
         self.blocks.append(blk)
         self.r = 0
         self.n_flushes += 1
-        if self.importance_mode == 0:
+        if self.importance_mode != 1:
             self.acc = np.zeros(D, np.float64)
             self.cnt = 0
 

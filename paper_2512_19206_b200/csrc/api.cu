@@ -41,7 +41,7 @@ int check_config(const mixkvq_config* c) {
       c->residual_len % c->group_size != 0)
     return MIXKVQ_E_UNSUPPORTED;
   if (c->score_bits != 2 && c->score_bits != 4) return MIXKVQ_E_UNSUPPORTED;
-  if (c->importance_mode != 0 && c->importance_mode != 1) return MIXKVQ_E_INVALID_ARG;
+  if (c->importance_mode < 0 || c->importance_mode > 2) return MIXKVQ_E_INVALID_ARG;
   if (c->block_layout != 0 && c->block_layout != 1) return MIXKVQ_E_INVALID_ARG;
   if (c->block_layout == 1 && c->residual_len != 128) return MIXKVQ_E_UNSUPPORTED;
   return MIXKVQ_OK;
@@ -233,7 +233,7 @@ int mixkvq_quantize_append(mixkvq_cache* cache, int layer, const void* k_dev, co
     }
     // prefill: complete windows go straight from the tensors to packed blocks; the last 1..R tokens stay in the
     // residual window (the running accumulator is only needed in cumulative mode, which keeps the per-block path)
-    if (cache->cfg.importance_mode == 0 && cache->r[layer] == 0 && n_tokens - t > cache->R) {
+    if (cache->cfg.importance_mode != 1 && cache->r[layer] == 0 && n_tokens - t > cache->R) {
       int nb = (n_tokens - t - 1) / cache->R;
       if (nb > 32768) nb = 32768;                  // grid.y limit
       LayerView lv = view(cache, layer);

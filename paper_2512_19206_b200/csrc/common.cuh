@@ -99,11 +99,12 @@ __device__ inline int quant_code(float x, float z, float s, int max_code) {
 }
 
 // Section 4.2: A_d = (acc / cnt) * (range / (2^B - 1)) in fp64; tier by the two thresholds.
+// error_only (the ablation without the query term): I_d = 1, so A_d = S_d.
 __device__ inline uint8_t salience_tier(double acc, uint32_t cnt, float mx, float mn, int score_bits,
-                                        float tau_bf16, float tau_u4, double* a_out) {
+                                        float tau_bf16, float tau_u4, double* a_out, bool error_only = false) {
   double range = (double)mx - (double)mn;
   double S = __ddiv_rn(range, (double)((1 << score_bits) - 1));
-  double I = __ddiv_rn(acc, (double)cnt);
+  double I = error_only ? 1.0 : __ddiv_rn(acc, (double)cnt);
   double A = __dmul_rn(I, S);
   if (a_out) *a_out = A;
   if (A > (double)tau_bf16) return kBF16;

@@ -123,7 +123,7 @@ flush_kernel(LayerView lv, BulkSrc src) {
         acc = reinterpret_cast<const double*>(state)[d];
         cnt = *reinterpret_cast<const uint32_t*>(state + 1024);
       }
-      tier = salience_tier(acc, cnt, wmx, wmn, lv.score_bits, lv.tau_bf16, lv.tau_u4, nullptr);
+      tier = salience_tier(acc, cnt, wmx, wmn, lv.score_bits, lv.tau_bf16, lv.tau_u4, nullptr, lv.importance_mode == 2);
       if (src.phase == 1) reinterpret_cast<uint8_t*>(blk)[d] = tier;
     }
     tierS[d] = tier;
@@ -372,7 +372,7 @@ flush_kernel(LayerView lv, BulkSrc src) {
   }
 
   // ---- window importance: the accumulator restarts with the next window (Section 4.2)
-  if (lv.importance_mode == 0 && !bulk) {
+  if (lv.importance_mode != 1 && !bulk) {
     if (tid < kD) reinterpret_cast<double*>(state)[tid] = 0.0;
     if (tid == 0) *reinterpret_cast<uint32_t*>(state + 1024) = 0u;
   }

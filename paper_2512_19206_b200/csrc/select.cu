@@ -18,7 +18,7 @@ select_window_kernel(LayerView lv, uint8_t* __restrict__ tiers, double* __restri
   double acc = reinterpret_cast<const double*>(st)[d];
   uint32_t cnt = *reinterpret_cast<const uint32_t*>(st + 1024);
   double A;
-  uint8_t t = salience_tier(acc, cnt, mx, mn, lv.score_bits, lv.tau_bf16, lv.tau_u4, &A);
+  uint8_t t = salience_tier(acc, cnt, mx, mn, lv.score_bits, lv.tau_bf16, lv.tau_u4, &A, lv.importance_mode == 2);
   tiers[(size_t)s * kD + d] = t;
   if (salience) salience[(size_t)s * kD + d] = A;
 }

@@ -135,12 +135,22 @@ def test_streamed_appends_equal_bulk(binding):
     U.compare_regions(bulk, 0, w, U.oracle_streams(w, 0, k, v, q))
 
 
-def test_cumulative_importance_mode(binding):
+@pytest.mark.parametrize("mode", [1, 2])
+def test_other_importance_modes(binding, mode):
+    # 1: cumulative |q| accumulator (Appendix D.2); 2: error-only ablation, A = S (Appendix E)
     w = small(batch=1, tokens=2 * 128 + 9, **W.P27)
+    if mode == 2:
+        w = dataclasses.replace(w, tau_bf16=12.0, tau_u4=1.8)
     k, v, q = W.tokens(w, 0, 0, w.tokens)
-    cache = U.make_cache(binding, w, importance_mode=1)
+    cache = U.make_cache(binding, w, importance_mode=mode)
     cache.quantize_append(0, k.cuda(), v.cuda(), q.cuda())
-    U.compare_regions(cache, 0, w, U.oracle_streams(w, 0, k, v, q, importance_mode=1))
+    orc = U.oracle_streams(w, 0, k, v, q, importance_mode=mode)
+    U.compare_regions(cache, 0, w, orc)
+    tiers, sal = cache.select_channels(0)
+    for (b, hk), st in orc.items():
+        t, A = st.current_tiers()
+        assert np.array_equal(tiers[b, hk].cpu().numpy(), t) and np.array_equal(sal[b, hk].cpu().numpy(), A)
+    assert len({int(x) for st in orc.values() for blk in st.blocks for x in blk.tiers}) == 3
 
 
 # ------------------------------------------------------------------------------------------- attention

@@ -137,3 +137,22 @@ def test_memory_figures():
     assert O.fp16_cache_bytes(m["n_layers"], m["n_kv_heads"], m["head_dim"], m["batch"], m["tokens"]) == m["bytes"] == 2 ** 39
     s = GOLD["memory_saving"]
     assert 1 - s["to_bits"] / s["from_bits"] == pytest.approx(s["saving_min"])
+
+
+def test_error_only_mode_ranks_channels_by_sensitivity_alone(rng):
+    # the ablation of Appendix E: A_d = S_d; the queries must not matter, the key ranges decide
+    from conftest import to_bf16
+    k = to_bf16(rng.standard_normal((129, O.D)) * rng.uniform(0.5, 6.0, (1, O.D)))
+    v = to_bf16(rng.standard_normal((129, O.D)))
+    outs = []
+    for scale in (1.0, 7.0):
+        q = to_bf16(rng.standard_normal((2, 129, O.D)) * scale)
+        st = O.OracleStream(g=2, tau_bf16=5.0, tau_u4=3.0, importance_mode=2)
+        st.append_many(k, v, q)
+        outs.append(st.blocks[0])
+    a, b = outs
+    assert np.array_equal(a.tiers, b.tiers) and np.array_equal(a.A, b.A)
+    S = (k[:128].max(0).astype(np.float64) - k[:128].min(0).astype(np.float64)) / 3.0
+    assert np.array_equal(a.A, S)
+    assert np.array_equal(a.tiers, np.where(S > 5.0, O.TIER_BF16, np.where(S > 3.0, O.TIER_U4, O.TIER_U2)))
+    assert len(set(a.tiers.tolist())) == 3

@@ -311,3 +311,48 @@ def test_decode_step_equals_append_then_attention(binding, kind, layout):
     U.compare_regions(fused, 0, w, orc)
     U.compare_regions(plain, 0, w, orc)
     assert fused.status() == 0 and fused.describe(0).residual_tokens == plain.describe(0).residual_tokens
+
+
+# --------------------------------------------------------------------------- guard bands around caller memory
+@pytest.mark.parametrize("layout", [0, 1])
+def test_no_write_outside_the_callers_buffers(binding, layout):
+    # cache memory, workspace and output are carved out of larger tensors filled with a pattern; after a bulk append,
+    # streamed steps across a flush and attention on both kernels, the bytes around them are untouched
+    import ctypes as C
+    w = small("qwen7b", batch=2, tokens=3 * 128 + 120, **W.P27)
+    steps = 12
+    cfg = binding.make_config(1, w.batch, w.n_q_heads, w.n_kv_heads, w.tokens + steps + 4, tau_bf16=w.tau_bf16,
+                              tau_u4=w.tau_u4, block_layout=layout)
+    nbytes, ws_bytes = binding.cache_bytes(cfg)
+    pad = 4096
+    def guarded(n):
+        t = torch.full((n + 2 * pad,), 0xA5, dtype=torch.uint8, device="cuda")
+        return t, t[pad:pad + n]
+    mem_all, mem = guarded(nbytes)
+    ws_all, ws = guarded(ws_bytes)
+    out_all, out_b = guarded(w.batch * w.n_q_heads * 128 * 4)
+    out = out_b.view(torch.float32).view(w.batch, w.n_q_heads, 128)
+    assert mem.data_ptr() % 256 == 0 and ws.data_ptr() % 16 == 0
+    lib, handle = binding.lib(), C.c_void_p()
+    stream = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    assert lib.mixkvq_cache_init(C.byref(cfg), C.c_void_p(mem.data_ptr()), nbytes, stream, C.byref(handle)) == 0
+    k, v, q = (x.cuda() for x in W.tokens(w, 0, 0, w.tokens + steps))
+    p = lambda t: C.c_void_p(t.data_ptr())
+    first = [x[:, :, :w.tokens].contiguous() for x in (k, v, q)]
+    assert lib.mixkvq_quantize_append(handle, 0, p(first[0]), p(first[1]), p(first[2]), w.tokens, stream) == 0
+    for i in range(steps):
+        t = w.tokens + i
+        ks, vs, qs = (x[:, :, t:t + 1].contiguous() for x in (k, v, q))
+        assert lib.mixkvq_decode_step(handle, 0, p(ks), p(vs), p(qs), p(out), C.c_float(W.softmax_scale()), p(ws), ws_bytes,
+                                      stream) == 0
+    for kind in (1, 0):
+        assert lib.mixkvq_set_attention_kernel(handle, kind) == 0
+        qd = q[:, :, -1].contiguous()
+        assert lib.mixkvq_decode_attention(handle, 0, p(qd), p(out), C.c_float(W.softmax_scale()), p(ws), ws_bytes, stream) == 0
+    status = C.c_int(-1)
+    assert lib.mixkvq_query_status(handle, C.byref(status), stream) == 0 and status.value == 0
+    torch.cuda.synchronize()
+    assert torch.isfinite(out).all()
+    for whole, n in ((mem_all, nbytes), (ws_all, ws_bytes), (out_all, out_b.numel())):
+        assert bool((whole[:pad] == 0xA5).all()) and bool((whole[pad + n:] == 0xA5).all())
+    lib.mixkvq_cache_destroy(handle)

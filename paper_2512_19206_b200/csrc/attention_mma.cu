@@ -28,7 +28,7 @@ constexpr int kStages = 3;
 constexpr int kStageBytes = 3072;            // one key-meta group (512 B) followed by the unit (<= 2560 B), as in the block
 constexpr int kKeyMetaOff = 0;
 constexpr int kUnitOff = 512;
-constexpr int kPrepBytes = 1280;             // kprep 512 | zprep 256 | svp 256 | zvp 256
+constexpr int kPrepBytes = 1536;             // kprep 512 | zprep 256 | svp 256 | zvp 512
 constexpr int kSharedTail = 128 + 2048 + 2048 + 128 + 128 + 4096;
 constexpr int kSmemBytes = kWarps * (kStages * kStageBytes + kPrepBytes) + kSharedTail;
 constexpr int kCtasPerSm = 4;
@@ -70,6 +70,13 @@ __device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1,
   asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// d = a * b + c with the accumulator input in other registers than the result
+__device__ __forceinline__ void mma_f16_to(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                           uint32_t b1, float c0, float c1, float c2, float c3) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%12,%13};"
+               : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(c0), "f"(c1), "f"(c2), "f"(c3));
 }
 __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1) {
@@ -128,7 +135,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
   uint32_t* kprep = reinterpret_cast<uint32_t*>(prep);          // [8 kt][4 t]{m2 ch0, o2 ch0, m2 ch1, o2 ch1}
   uint32_t* zprep = reinterpret_cast<uint32_t*>(prep + 512);    // [8 kt][4 t][2 ch] half2 z / mult
   uint32_t* svp = reinterpret_cast<uint32_t*>(prep + 768);      // [2 ks][2 ch][4 t][4 vg] half2 s_v'
-  uint32_t* zvp = reinterpret_cast<uint32_t*>(prep + 1024);     // [2 ks][2 ch][4 vg][4 t] half2 z_v
+  uint32_t* zvp = reinterpret_cast<uint32_t*>(prep + 1024);     // [2 ks][8 rows][4 t][2 ch] half2: rows < VG z_v, row 4 ones
   unsigned char* tail = smem + kWarps * (kStages * kStageBytes + kPrepBytes);
   uint64_t* bars = reinterpret_cast<uint64_t*>(tail);           // [kWarps][kStages]
   uint16_t* qb16 = reinterpret_cast<uint16_t*>(tail + 128);     // [8][128] q, bf16 bits (0 for heads >= g)
@@ -141,7 +148,25 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
     for (int i = 0; i < kWarps * kStages + kWarps; ++i) mbar_init(smem_u32(&bars[i]), 1);   // rings + one per warp for the residual window
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  // constant rows of the zero-point / denominator tile: row 4 is all ones, the other rows >= VG stay zero
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int idx = lane + 32 * i, row = (idx >> 3) & 7;
+    zvp[idx] = (row == 4) ? 0x3C003C00u : 0u;
+  }
   __syncthreads();
+
+  // per-lane constants of the per-unit preparation steps
+  // keys: the lane converts channels 4*lane .. 4*lane+3 (k-tile lane / 4)
+  const float pk_zs = __uint_as_float((119u + (uint32_t)key_pos(lane >> 2)) << 23);        // 2^(pos - 8)
+  const int pk_kp = (((lane >> 2) * 4 + 2 * (lane & 1)) * 4 + ((lane & 3) >> 1) * 2);      // kprep word of the first pair
+  const int pk_zp = (((lane >> 2) * 4 + 2 * (lane & 1)) * 2 + ((lane & 3) >> 1));          // zprep word of the first pair
+  // values: the lane converts the scales and zero-points of token `lane`
+  const float pv_up = __uint_as_float((131u - 2u * (uint32_t)(lane >> 3)) << 23);          // 2^(4 - 2 * (2 ks + ch))
+  const int pv_sv = (((lane >> 3) * 4 + ((lane & 7) >> 1)) * 4 * 2) + (lane & 1);          // svp half index of group 0
+  const int pv_zv = ((((lane >> 4) * 8 * 4 + ((lane & 7) >> 1)) * 2 + ((lane >> 3) & 1)) * 2) + (lane & 1);   // zvp half index of group 0
+  constexpr uint32_t kUnitBytes = 2048u + 128u * (kD / G);   // codes of 32 tokens: keys 1024, values 1024, value scales
+  constexpr int UPG = G / 32;                                 // units per key group
 
   const int S = lv.B * lv.Hkv, U = lv.U, g = lv.g;
   const int packed_units = lv.n_blocks * U;
@@ -150,8 +175,8 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
   const long long cb = split_begin(total, gridDim.x, blockIdx.x), ce = split_begin(total, gridDim.x, blockIdx.x + 1);
 
   uint32_t res_phase = 0;         // phase of this warp's residual-staging barrier
-  uint32_t ring_count = 0;        // packed units this warp has consumed so far (ring position)
-  uint32_t ring_issued = 0;       // packed units this warp has issued so far
+  uint32_t ring_stage = 0;        // ring stage of the next packed unit this warp consumes
+  uint32_t ring_parity = 0;       // phase parity of that stage's barrier
   bool gave_up = false;
 
   for (long long seg = cb; seg < ce;) {
@@ -167,43 +192,57 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
     const uint16_t* resk = reinterpret_cast<const uint16_t*>(lv.resk + (size_t)s * lv.resk_stride);
     const uint16_t* resv = reinterpret_cast<const uint16_t*>(lv.resv + (size_t)s * lv.resv_stride);
 
-    // ---- the first copies of this segment go out before anything else: they do not depend on the query
+    // ---- the first copies of this segment go out before anything else: they do not depend on the query.
+    // The packed units of a stream are one uniform sequence (a group's scales, then its units), whatever the block size,
+    // so the copy source only ever moves forward: `isrc` is the next unit to stage, `ig` its index inside its key group.
     const int n_pack = max(0, min(we, packed_units) - wb);
     int issued = 0;
-    auto issue = [&](int x, bool first) {
-      // lane 0 only: stage unit x of this stream
-      const int bi = x / U, u = x - bi * U;
-      const char* blk = base + (size_t)bi * lv.base_bytes;
-      const uint32_t stage = ring_issued % kStages;
-      const uint32_t bar = smem_u32(&bars[warp * kStages + stage]);
-      const uint32_t dst = smem_u32(ring + stage * kStageBytes);
-      const bool meta = first || ((u * 32) % G == 0);
-      const bool group_start = (u * 32) % G == 0;       // then the group's scales lie directly before the unit: one copy
-      mbar_expect_tx(bar, lv.unit_bytes + (meta ? 512u : 0u));
-      if (group_start) {
-        bulk_g2s(dst + kKeyMetaOff, blk + frag_meta_off((u * 32) / G, G, lv.unit_bytes), 512u + lv.unit_bytes, bar);
+    const char* isrc = base + (size_t)wb * kUnitBytes + 512u * (size_t)(wb / UPG + 1);
+    int ig = wb & (UPG - 1);
+    auto issue = [&](uint32_t dst, uint32_t bar, bool first) {
+      // all lanes keep the position; lane 0 stages the unit at ring offset dst, signalled on bar
+      if (UPG == 1 || ig == 0) {        // the group's scales lie directly before the unit: one copy
+        if (lane == 0) {
+          mbar_expect_tx(bar, kUnitBytes + 512u);
+          bulk_g2s(dst + kKeyMetaOff, isrc - 512, 512u + kUnitBytes, bar);
+        }
+      } else if (lane == 0) {
+        mbar_expect_tx(bar, kUnitBytes + (first ? 512u : 0u));
+        bulk_g2s(dst + kUnitOff, isrc, kUnitBytes, bar);
+        if (first) bulk_g2s(dst + kKeyMetaOff, isrc - (size_t)ig * kUnitBytes - 512, 512u, bar);
+      }
+      isrc += kUnitBytes;
+      if (UPG == 1) {
+        isrc += 512;
       } else {
-        bulk_g2s(dst + kUnitOff, blk + frag_unit_off(u, G, lv.unit_bytes), lv.unit_bytes, bar);
-        if (meta) bulk_g2s(dst + kKeyMetaOff, blk + frag_meta_off((u * 32) / G, G, lv.unit_bytes), 512u, bar);
+        ig = (ig + 1) & (UPG - 1);
+        if (ig == 0) isrc += 512;
       }
     };
-    for (; !gave_up && issued < min(n_pack, kStages); ++issued) {
-      if (lane == 0) issue(wb + issued, issued == 0);
-      ++ring_issued;
+    // the ring continues where the previous segment left it: stage ring_stage, barrier phase parity ring_parity
+    const uint32_t ring_u32 = smem_u32(ring), bar_u32 = smem_u32(&bars[warp * kStages]);
+    if (!gave_up) {
+      uint32_t sg = ring_stage;
+      for (; issued < min(n_pack, kStages); ++issued) {
+        issue(ring_u32 + sg * kStageBytes, bar_u32 + sg * 8u, issued == 0);
+        sg = (sg == kStages - 1) ? 0u : sg + 1u;
+      }
     }
 
     // the first block's table entry is requested now as well, long before the first unit arrives
-    int cur_bi = -1, pf_bi = -1;
-    uint2 entry = make_uint2(0, 0), pf_entry = make_uint2(0, 0);
+    int bi = 0, u = 0;                     // block and unit inside it of the next unit to consume
+    uint2 pf_entry = make_uint2(0, 0);
     if (n_pack > 0) {
-      pf_bi = wb / U;
-      pf_entry = table[pf_bi];
+      bi = wb / U;
+      u = wb - bi * U;
+      pf_entry = table[bi];
     }
+    bool new_block = true;
     int n16 = 0, n4 = 0, n16p = 0;
     uint32_t xb0 = 0u, xb1 = 0u;          // B fragments of the block's first 16 promoted channels
-    const char* ex = nullptr;
-    uint32_t ex_hdr = 0, ex_unit = 0;
-
+    const char* ex = nullptr;             // the block's extras
+    const char* exu = nullptr;            // ... of the current unit
+    uint32_t ex_unit = 0;
 
     // ---- query of this stream: bf16 and fp16 tables for the gathered paths
     {
@@ -234,7 +273,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
 
     float O[8][4];       // O^T tiles: [channel tile] x (channels r, r+8) x (heads 2t, 2t+1); packed part scaled 2^-20
     float Zc[4] = {0.f, 0.f, 0.f, 0.f};   // rows 0..VG-1: sum p * z_v per value group; row 4: sum p
-    float zc[4] = {0.f, 0.f, 0.f, 0.f};   // key zero-point term of the current key group
+    float zc[4] = {0.f, 0.f, 0.f, 0.f};   // key zero-point term q . z of the current key group (equal for all rows)
     float m0 = -INFINITY, m1 = -INFINITY; // running max (log2 domain) of heads 2t, 2t+1
 #pragma unroll
     for (int ct = 0; ct < 8; ++ct)
@@ -242,20 +281,17 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
       for (int i = 0; i < 4; ++i) O[ct][i] = 0.f;
     bool o_true_scale = false;
 
-    for (int i = 0; i < n_pack && !gave_up; ++i) {
-      const int x = wb + i;
-      const int bi = x / U, u = x - bi * U;
-      if (bi != cur_bi) {
-        entry = (pf_bi == bi) ? pf_entry : table[bi];
-        cur_bi = bi;
-        pf_bi = bi + 1;
-        if (pf_bi < lv.n_blocks) pf_entry = table[pf_bi];
+    int consumed = 0;
+    for (; consumed < n_pack && !gave_up; ++consumed) {
+      if (new_block) {
+        const uint2 entry = pf_entry;
+        if (bi + 1 < lv.n_blocks) pf_entry = table[bi + 1];
         n16 = entry.y & 0xFF;
         n4 = (entry.y >> 8) & 0xFF;
         n16p = (n16 + 1) >> 1;
         ex = extras + (size_t)entry.x * 16;
-        ex_hdr = extras_header_bytes(n16, n4);
         ex_unit = extras_unit_bytes(n16, n4, kU4 == 2);
+        exu = ex + extras_header_bytes(n16, n4) + (size_t)u * ex_unit;
         // the block's promoted channels are the same for its units: gather their query entries once
         xb0 = xb1 = 0u;
         if (n16 > 0) {
@@ -269,65 +305,58 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
           xb0 = gather_q(t);
           xb1 = gather_q(t + 4);
         }
+        new_block = false;
       }
-      const uint32_t stage = ring_count % kStages, parity = (ring_count / kStages) & 1;
-      if (!mbar_wait_bounded(smem_u32(&bars[warp * kStages + stage]), parity)) {
+      if (!mbar_wait_bounded(bar_u32 + ring_stage * 8u, ring_parity)) {
         gave_up = true;
         break;
       }
-      ++ring_count;
-      const unsigned char* stg = ring + stage * kStageBytes;
+      const unsigned char* stg = ring + ring_stage * kStageBytes;
       const unsigned char* st = stg + kUnitOff;        // the unit's codes and value scales
-      const bool has_meta = (i == 0) || ((u * 32) % G == 0);
+      const bool has_meta = (UPG == 1) || (consumed == 0) || ((u & (UPG - 1)) == 0);
 
       // ---- key-group preparation: fp16 scale pairs in fragment order, zero-point tile
       if (has_meta) {
         const uint4 mz = reinterpret_cast<const uint4*>(stg + kKeyMetaOff)[lane];   // channels 4*lane .. 4*lane+3
-        const int kt = lane >> 2, ch = (lane & 3) >> 1, t0 = 2 * (lane & 1);
-        const float zs = 1.0f / (float)(1 << (8 - key_pos(kt)));
         const uint32_t ma = pack_half2(bf_lo(mz.x), bf_lo(mz.y)), mb = pack_half2(bf_lo(mz.z), bf_lo(mz.w));
         const uint32_t neg4 = 0xC400C400u;   // half2(-4, -4)
         __syncwarp();
-        *reinterpret_cast<uint2*>(&kprep[(kt * 4 + t0) * 4 + ch * 2]) = make_uint2(ma, hmul2_u(ma, neg4));
-        *reinterpret_cast<uint2*>(&kprep[(kt * 4 + t0 + 1) * 4 + ch * 2]) = make_uint2(mb, hmul2_u(mb, neg4));
-        zprep[(kt * 4 + t0) * 2 + ch] = pack_half2(bf_hi(mz.x) * zs, bf_hi(mz.y) * zs);
-        zprep[(kt * 4 + t0 + 1) * 2 + ch] = pack_half2(bf_hi(mz.z) * zs, bf_hi(mz.w) * zs);
+        *reinterpret_cast<uint2*>(&kprep[pk_kp]) = make_uint2(ma, hmul2_u(ma, neg4));
+        *reinterpret_cast<uint2*>(&kprep[pk_kp + 4]) = make_uint2(mb, hmul2_u(mb, neg4));
+        zprep[pk_zp] = pack_half2(bf_hi(mz.x) * pk_zs, bf_hi(mz.y) * pk_zs);
+        zprep[pk_zp + 2] = pack_half2(bf_hi(mz.z) * pk_zs, bf_hi(mz.w) * pk_zs);
         __syncwarp();
-        zc[0] = zc[1] = zc[2] = zc[3] = 0.f;
+        // the zero-point term q . z of the group: its own accumulator chain, added to the logits after the key tiles
 #pragma unroll
         for (int kt2 = 0; kt2 < 8; ++kt2) {
           const uint2 zz = *reinterpret_cast<const uint2*>(&zprep[(kt2 * 4 + t) * 2]);
-          mma_f16(zc, zz.x, zz.x, zz.y, zz.y, bq[kt2][0], bq[kt2][1]);
+          if (kt2 == 0) mma_f16_to(zc, zz.x, zz.x, zz.y, zz.y, bq[0][0], bq[0][1], 0.f, 0.f, 0.f, 0.f);
+          else mma_f16(zc, zz.x, zz.x, zz.y, zz.y, bq[kt2][0], bq[kt2][1]);
         }
       }
 
-      // ---- extras of this unit: issue the global loads early
-      const char* exu = ex + ex_hdr + (size_t)u * ex_unit;
-      uint32_t xa[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};   // BF16 pairs, first 16 promoted channels
+      // ---- extras of this unit: issue the global loads early (BF16 pairs of the first 16 promoted channels)
+      uint32_t xa[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};
       if (n16 > 0) {
-        const uint32_t* xw = reinterpret_cast<const uint32_t*>(exu);
-        if (t < n16p) {
+        const uint32_t* xw = reinterpret_cast<const uint32_t*>(exu) + (t * 32 + r);
+        const bool p0 = t < n16p;
 #pragma unroll
-          for (int mt = 0; mt < 2; ++mt) {
-            xa[mt][0] = xw[t * 32 + mt * 16 + r];
-            xa[mt][1] = xw[t * 32 + mt * 16 + 8 + r];
-          }
+        for (int mt = 0; mt < 2; ++mt) {
+          xa[mt][0] = p0 ? xw[mt * 16] : 0u;
+          xa[mt][1] = p0 ? xw[mt * 16 + 8] : 0u;
         }
-        if (t + 4 < n16p) {
+        if (n16p > 4) {       // more than 8 promoted channels (uniform over the warp)
+          const bool p1 = t + 4 < n16p;
 #pragma unroll
           for (int mt = 0; mt < 2; ++mt) {
-            xa[mt][2] = xw[(t + 4) * 32 + mt * 16 + r];
-            xa[mt][3] = xw[(t + 4) * 32 + mt * 16 + 8 + r];
+            xa[mt][2] = p1 ? xw[128 + mt * 16] : 0u;
+            xa[mt][3] = p1 ? xw[128 + mt * 16 + 8] : 0u;
           }
         }
       }
 
       // ---- q.K^T on the base (2-bit low plane) tiles
       float Sx[2][4];
-#pragma unroll
-      for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) Sx[mt][j] = zc[j];
       {
         const uint4 kw0 = reinterpret_cast<const uint4*>(st)[lane];
         const uint4 kw1 = reinterpret_cast<const uint4*>(st)[32 + lane];
@@ -344,7 +373,8 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
               const uint32_t code = (key_shift(kw[mt][j], kt) & mask) | 0x44004400u;     // 4 + c * 2^(pos-8)
               a[j] = hfma2_u(code, j < 2 ? kp.x : kp.z, j < 2 ? kp.y : kp.w);            // c * s * 2^(pos-8)
             }
-            mma_f16(Sx[mt], a[0], a[1], a[2], a[3], bq[kt][0], bq[kt][1]);
+            if (kt == 0) mma_f16_to(Sx[mt], a[0], a[1], a[2], a[3], bq[0][0], bq[0][1], 0.f, 0.f, 0.f, 0.f);
+            else mma_f16(Sx[mt], a[0], a[1], a[2], a[3], bq[kt][0], bq[kt][1]);
           }
         }
       }
@@ -459,33 +489,28 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
 
       // ---- value-group preparation (lane = token)
       {
-        const uint32_t* vmeta = reinterpret_cast<const uint32_t*>(st + 2048);
-        const int ks = lane >> 4, ch = (lane >> 3) & 1, tt = (lane & 7) >> 1, e = lane & 1;
-        const float up = (float)(1 << 4) / (float)(1 << (2 * (lane >> 3)));     // 2^(4 - 2*(2ks + ch))
-        __half* svh = reinterpret_cast<__half*>(svp);
-        __half* zvh = reinterpret_cast<__half*>(zvp);
+        const uint32_t* vmeta = reinterpret_cast<const uint32_t*>(st + 2048) + lane * VG;
+        __half* svh = reinterpret_cast<__half*>(svp) + pv_sv;
+        __half* zvh = reinterpret_cast<__half*>(zvp) + pv_zv;
 #pragma unroll
         for (int vg = 0; vg < VG; ++vg) {
-          const uint32_t mz = vmeta[lane * VG + vg];
-          svh[((((ks * 2 + ch) * 4 + tt) * 4 + vg) << 1) + e] = __float2half_rn(bf_lo(mz) * up);
-          zvh[((((ks * 2 + ch) * 4 + vg) * 4 + tt) << 1) + e] = __float2half_rn(bf_hi(mz));
+          const uint32_t mz = vmeta[vg];
+          svh[2 * vg] = __float2half_rn(bf_lo(mz) * pv_up);
+          zvh[16 * vg] = __float2half_rn(bf_hi(mz));
         }
       }
 
-      // ---- online softmax (log2 domain); heads 2t, 2t+1; tokens r, r+8 of each m-tile
-      float xs[2][4];
-#pragma unroll
-      for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) xs[mt][j] = Sx[mt][j] * scale_log2e;
-      float u0 = fmaxf(fmaxf(xs[0][0], xs[0][2]), fmaxf(xs[1][0], xs[1][2]));
-      float u1 = fmaxf(fmaxf(xs[0][1], xs[0][3]), fmaxf(xs[1][1], xs[1][3]));
+      // ---- online softmax (log2 domain); heads 2t, 2t+1; tokens r, r+8 of each m-tile.
+      // logit = (Sx + zc) * scale: the zero-point term zc is the same for every token of the unit
+      const float zl0 = zc[0] * scale_log2e, zl1 = zc[1] * scale_log2e;
+      float u0 = fmaxf(fmaxf(Sx[0][0], Sx[0][2]), fmaxf(Sx[1][0], Sx[1][2]));
+      float u1 = fmaxf(fmaxf(Sx[0][1], Sx[0][3]), fmaxf(Sx[1][1], Sx[1][3]));
 #pragma unroll
       for (int off = 4; off < 32; off <<= 1) {
         u0 = fmaxf(u0, __shfl_xor_sync(0xffffffffu, u0, off));
         u1 = fmaxf(u1, __shfl_xor_sync(0xffffffffu, u1, off));
       }
-      const float n0 = fmaxf(m0, u0), n1 = fmaxf(m1, u1);
+      const float n0 = fmaxf(m0, fmaf(u0, scale_log2e, zl0)), n1 = fmaxf(m1, fmaf(u1, scale_log2e, zl1));
       if (__any_sync(0xffffffffu, (n0 > m0) || (n1 > m1))) {
         const float a0 = exp2f(m0 - n0), a1 = exp2f(m1 - n1);    // exp2(-inf) = 0 on the first unit
 #pragma unroll
@@ -496,27 +521,22 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
         m0 = n0;
         m1 = n1;
       }
+      const float c0 = zl0 - m0, c1 = zl1 - m1;
       uint32_t Pt[2][2];    // P^T B fragments: [k-step][tokens 2t.. / 2t+8..], head r
 #pragma unroll
       for (int mt = 0; mt < 2; ++mt) {
-        const uint32_t plo = pack_half2(ex2_approx(xs[mt][0] - m0), ex2_approx(xs[mt][1] - m1));   // token r
-        const uint32_t phi = pack_half2(ex2_approx(xs[mt][2] - m0), ex2_approx(xs[mt][3] - m1));   // token r + 8
+        const uint32_t plo = pack_half2(ex2_approx(fmaf(Sx[mt][0], scale_log2e, c0)), ex2_approx(fmaf(Sx[mt][1], scale_log2e, c1)));   // token r
+        const uint32_t phi = pack_half2(ex2_approx(fmaf(Sx[mt][2], scale_log2e, c0)), ex2_approx(fmaf(Sx[mt][3], scale_log2e, c1)));   // token r + 8
         Pt[mt][0] = movmatrix_trans(plo);
         Pt[mt][1] = movmatrix_trans(phi);
       }
       __syncwarp();   // svp / zvp written above are read below
 
-      // ---- zero-point and denominator tile: rows 0..VG-1 = z_v of the group, row 4 = ones
+      // ---- zero-point and denominator tile: rows 0..VG-1 = z_v of the group, row 4 = ones, the rest zero
 #pragma unroll
       for (int ks = 0; ks < 2; ++ks) {
-        uint32_t a0 = 0, a2 = 0;
-        if (r < VG) {
-          a0 = zvp[((ks * 2 + 0) * 4 + r) * 4 + t];
-          a2 = zvp[((ks * 2 + 1) * 4 + r) * 4 + t];
-        } else if (r == 4) {
-          a0 = a2 = 0x3C003C00u;
-        }
-        mma_f16(Zc, a0, 0u, a2, 0u, Pt[ks][0], Pt[ks][1]);
+        const uint2 zz = *reinterpret_cast<const uint2*>(&zvp[((ks * 8 + r) * 4 + t) * 2]);
+        mma_f16(Zc, zz.x, 0u, zz.y, 0u, Pt[ks][0], Pt[ks][1]);
       }
       // ---- P.V: codes as fp16 subnormals, scales folded into P
       {
@@ -543,20 +563,31 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
         }
       }
 
-      // ---- release the stage and refill it
+      // ---- release the stage and refill it, then move on to the next unit
       __syncwarp();
       if (issued < n_pack) {
-        if (lane == 0) issue(wb + issued, false);
-        ++ring_issued;
+        issue(ring_u32 + ring_stage * kStageBytes, bar_u32 + ring_stage * 8u, false);
         ++issued;
+      }
+      if (++ring_stage == kStages) {
+        ring_stage = 0;
+        ring_parity ^= 1u;
+      }
+      exu += ex_unit;
+      if (++u == U) {
+        u = 0;
+        ++bi;
+        new_block = true;
       }
     }
     if (gave_up) {
       // drain what is still in flight (bounded); later segments stage nothing but still join the CTA barriers
-      while (ring_count < ring_issued) {
-        const uint32_t stage = ring_count % kStages, parity = (ring_count / kStages) & 1;
-        mbar_wait_bounded(smem_u32(&bars[warp * kStages + stage]), parity);
-        ++ring_count;
+      for (; consumed < issued; ++consumed) {
+        mbar_wait_bounded(bar_u32 + ring_stage * 8u, ring_parity);
+        if (++ring_stage == kStages) {
+          ring_stage = 0;
+          ring_parity ^= 1u;
+        }
       }
       if (lane == 0) atomicOr(lv.status, (uint32_t)MIXKVQ_DEV_COPY_TIMEOUT);
     }

@@ -28,13 +28,14 @@ constexpr int kStages = 3;
 constexpr int kStageBytes = 3072;            // one key-meta group (512 B) followed by the unit (<= 2560 B), as in the block
 constexpr int kKeyMetaOff = 0;
 constexpr int kUnitOff = 512;
-constexpr int kPrepBytes = 1536;             // kprep 512 | zprep 256 | svp 256 | zvp 512
+constexpr int kPrepBytes = 2304;             // kprep 512 | zprep 512 | svp 256 | zvp 1024
 constexpr int kSharedTail = 128 + 2048 + 2048 + 128 + 128 + 4096;
 constexpr int kSmemBytes = kWarps * (kStages * kStageBytes + kPrepBytes) + kSharedTail;
 constexpr int kCtasPerSm = 4;
 static_assert((kWarps * kStages + kWarps) * 8 <= 128, "the mbarrier area at the start of the shared tail holds 16 barriers");
 constexpr int kResidualWeight = 2;           // a 32-token unit of the residual window counts as this many packed units in the split
 constexpr uint32_t kSpinLimit = 1u << 22;    // bounded wait on a staged copy
+constexpr float kMaxSlack = 3.0f;            // a packed unit's probabilities are at most 2^kMaxSlack (log2 domain)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -124,7 +125,8 @@ __device__ __forceinline__ uint32_t key_shift(uint32_t w, int kt) { return kt < 
 // per channel pair, gathered), 2 = 4-bit base (dense high plane)
 template <int G, int kU4>
 __global__ void __launch_bounds__(kWarps * 32, kCtasPerSm)
-attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float scale_log2e, float* __restrict__ ws) {
+attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float scale_log2e, float* __restrict__ ws,
+                     uint32_t four2) {
   constexpr int VG = kD / G;              // value groups per token
   constexpr int TPG = 8 / VG;             // 16-channel tiles per value group
   extern __shared__ __align__(128) unsigned char smem[];
@@ -133,9 +135,10 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
   unsigned char* ring = smem + warp * (kStages * kStageBytes);
   unsigned char* prep = smem + kWarps * kStages * kStageBytes + warp * kPrepBytes;
   uint32_t* kprep = reinterpret_cast<uint32_t*>(prep);          // [8 kt][4 t]{m2 ch0, o2 ch0, m2 ch1, o2 ch1}
-  uint32_t* zprep = reinterpret_cast<uint32_t*>(prep + 512);    // [8 kt][4 t][2 ch] half2 z / mult
-  uint32_t* svp = reinterpret_cast<uint32_t*>(prep + 768);      // [2 ks][2 ch][4 t][4 vg] half2 s_v'
-  uint32_t* zvp = reinterpret_cast<uint32_t*>(prep + 1024);     // [2 ks][8 rows][4 t][2 ch] half2: rows < VG z_v, row 4 ones
+  // the zero-point tiles are stored as whole A fragments (four registers), so one 16-byte load feeds the MMA
+  uint32_t* zprep = reinterpret_cast<uint32_t*>(prep + 512);    // [8 kt][4 t]{z ch0, z ch0, z ch1, z ch1} half2 z / mult
+  uint32_t* svp = reinterpret_cast<uint32_t*>(prep + 1024);     // [4 t][4 vg][2 ks][2 ch] half2 s_v'
+  uint32_t* zvp = reinterpret_cast<uint32_t*>(prep + 1280);     // [2 ks][8 rows][4 t]{ch0, 0, ch1, 0} half2: rows < VG z_v, row 4 ones
   unsigned char* tail = smem + kWarps * (kStages * kStageBytes + kPrepBytes);
   uint64_t* bars = reinterpret_cast<uint64_t*>(tail);           // [kWarps][kStages]
   uint16_t* qb16 = reinterpret_cast<uint16_t*>(tail + 128);     // [8][128] q, bf16 bits (0 for heads >= g)
@@ -150,9 +153,9 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
   }
   // constant rows of the zero-point / denominator tile: row 4 is all ones, the other rows >= VG stay zero
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int idx = lane + 32 * i, row = (idx >> 3) & 7;
-    zvp[idx] = (row == 4) ? 0x3C003C00u : 0u;
+  for (int i = 0; i < 8; ++i) {
+    const int idx = lane + 32 * i, row = (idx >> 4) & 7;
+    zvp[idx] = (row == 4 && (idx & 1) == 0) ? 0x3C003C00u : 0u;
   }
   __syncthreads();
 
@@ -160,11 +163,11 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
   // keys: the lane converts channels 4*lane .. 4*lane+3 (k-tile lane / 4)
   const float pk_zs = __uint_as_float((119u + (uint32_t)key_pos(lane >> 2)) << 23);        // 2^(pos - 8)
   const int pk_kp = (((lane >> 2) * 4 + 2 * (lane & 1)) * 4 + ((lane & 3) >> 1) * 2);      // kprep word of the first pair
-  const int pk_zp = (((lane >> 2) * 4 + 2 * (lane & 1)) * 2 + ((lane & 3) >> 1));          // zprep word of the first pair
+  const int pk_zp = pk_kp;                                                                  // zprep word of the first pair
   // values: the lane converts the scales and zero-points of token `lane`
   const float pv_up = __uint_as_float((131u - 2u * (uint32_t)(lane >> 3)) << 23);          // 2^(4 - 2 * (2 ks + ch))
-  const int pv_sv = (((lane >> 3) * 4 + ((lane & 7) >> 1)) * 4 * 2) + (lane & 1);          // svp half index of group 0
-  const int pv_zv = ((((lane >> 4) * 8 * 4 + ((lane & 7) >> 1)) * 2 + ((lane >> 3) & 1)) * 2) + (lane & 1);   // zvp half index of group 0
+  const int pv_sv = ((((lane & 7) >> 1) * 16 + (lane >> 3)) * 2) + (lane & 1);             // svp half index of group 0
+  const int pv_zv = ((((lane >> 4) * 8 * 4 + ((lane & 7) >> 1)) * 4 + 2 * ((lane >> 3) & 1)) * 2) + (lane & 1);   // zvp half index of group 0
   constexpr uint32_t kUnitBytes = 2048u + 128u * (kD / G);   // codes of 32 tokens: keys 1024, values 1024, value scales
   constexpr int UPG = G / 32;                                 // units per key group
 
@@ -189,8 +192,6 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
     const char* base = lv.base + (size_t)s * lv.base_stride;
     const char* extras = lv.extras + (size_t)s * lv.extras_stride;
     const uint2* table = reinterpret_cast<const uint2*>(lv.table + (size_t)s * lv.table_stride);
-    const uint16_t* resk = reinterpret_cast<const uint16_t*>(lv.resk + (size_t)s * lv.resk_stride);
-    const uint16_t* resv = reinterpret_cast<const uint16_t*>(lv.resv + (size_t)s * lv.resv_stride);
 
     // ---- the first copies of this segment go out before anything else: they do not depend on the query.
     // The packed units of a stream are one uniform sequence (a group's scales, then its units), whatever the block size,
@@ -273,7 +274,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
 
     float O[8][4];       // O^T tiles: [channel tile] x (channels r, r+8) x (heads 2t, 2t+1); packed part scaled 2^-20
     float Zc[4] = {0.f, 0.f, 0.f, 0.f};   // rows 0..VG-1: sum p * z_v per value group; row 4: sum p
-    float zc[4] = {0.f, 0.f, 0.f, 0.f};   // key zero-point term q . z of the current key group (equal for all rows)
+    float zl0 = 0.f, zl1 = 0.f;           // key zero-point term (q . z) * scale of the current key group, heads 2t, 2t+1
     float m0 = -INFINITY, m1 = -INFINITY; // running max (log2 domain) of heads 2t, 2t+1
 #pragma unroll
     for (int ct = 0; ct < 8; ++ct)
@@ -323,16 +324,22 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
         __syncwarp();
         *reinterpret_cast<uint2*>(&kprep[pk_kp]) = make_uint2(ma, hmul2_u(ma, neg4));
         *reinterpret_cast<uint2*>(&kprep[pk_kp + 4]) = make_uint2(mb, hmul2_u(mb, neg4));
-        zprep[pk_zp] = pack_half2(bf_hi(mz.x) * pk_zs, bf_hi(mz.y) * pk_zs);
-        zprep[pk_zp + 2] = pack_half2(bf_hi(mz.z) * pk_zs, bf_hi(mz.w) * pk_zs);
+        const uint32_t za = pack_half2(bf_hi(mz.x) * pk_zs, bf_hi(mz.y) * pk_zs);
+        const uint32_t zb = pack_half2(bf_hi(mz.z) * pk_zs, bf_hi(mz.w) * pk_zs);
+        *reinterpret_cast<uint2*>(&zprep[pk_zp]) = make_uint2(za, za);
+        *reinterpret_cast<uint2*>(&zprep[pk_zp + 4]) = make_uint2(zb, zb);
         __syncwarp();
         // the zero-point term q . z of the group: its own accumulator chain, added to the logits after the key tiles
+        // (the tile's rows are equal, so are the rows of the result)
+        float zc[4];
 #pragma unroll
         for (int kt2 = 0; kt2 < 8; ++kt2) {
-          const uint2 zz = *reinterpret_cast<const uint2*>(&zprep[(kt2 * 4 + t) * 2]);
-          if (kt2 == 0) mma_f16_to(zc, zz.x, zz.x, zz.y, zz.y, bq[0][0], bq[0][1], 0.f, 0.f, 0.f, 0.f);
-          else mma_f16(zc, zz.x, zz.x, zz.y, zz.y, bq[kt2][0], bq[kt2][1]);
+          const uint4 zz = *reinterpret_cast<const uint4*>(&zprep[(kt2 * 4 + t) * 4]);
+          if (kt2 == 0) mma_f16_to(zc, zz.x, zz.y, zz.z, zz.w, bq[0][0], bq[0][1], 0.f, 0.f, 0.f, 0.f);
+          else mma_f16(zc, zz.x, zz.y, zz.z, zz.w, bq[kt2][0], bq[kt2][1]);
         }
+        zl0 = zc[0] * scale_log2e;
+        zl1 = zc[1] * scale_log2e;
       }
 
       // ---- extras of this unit: issue the global loads early (BF16 pairs of the first 16 promoted channels)
@@ -370,7 +377,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
             uint32_t a[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-              const uint32_t code = (key_shift(kw[mt][j], kt) & mask) | 0x44004400u;     // 4 + c * 2^(pos-8)
+              const uint32_t code = (key_shift(kw[mt][j], kt) & mask) | four2;           // 4 + c * 2^(pos-8)
               a[j] = hfma2_u(code, j < 2 ? kp.x : kp.z, j < 2 ? kp.y : kp.w);            // c * s * 2^(pos-8)
             }
             if (kt == 0) mma_f16_to(Sx[mt], a[0], a[1], a[2], a[3], bq[0][0], bq[0][1], 0.f, 0.f, 0.f, 0.f);
@@ -495,23 +502,26 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
 #pragma unroll
         for (int vg = 0; vg < VG; ++vg) {
           const uint32_t mz = vmeta[vg];
-          svh[2 * vg] = __float2half_rn(bf_lo(mz) * pv_up);
-          zvh[16 * vg] = __float2half_rn(bf_hi(mz));
+          svh[8 * vg] = __float2half_rn(bf_lo(mz) * pv_up);
+          zvh[32 * vg] = __float2half_rn(bf_hi(mz));
         }
       }
 
       // ---- online softmax (log2 domain); heads 2t, 2t+1; tokens r, r+8 of each m-tile.
       // logit = (Sx + zc) * scale: the zero-point term zc is the same for every token of the unit
-      const float zl0 = zc[0] * scale_log2e, zl1 = zc[1] * scale_log2e;
       float u0 = fmaxf(fmaxf(Sx[0][0], Sx[0][2]), fmaxf(Sx[1][0], Sx[1][2]));
       float u1 = fmaxf(fmaxf(Sx[0][1], Sx[0][3]), fmaxf(Sx[1][1], Sx[1][3]));
+      u0 = fmaf(u0, scale_log2e, zl0);
+      u1 = fmaf(u1, scale_log2e, zl1);
+      // The reference maximum only has to keep the probabilities inside the fp16 range: it is raised (to the true
+      // maximum so far, with the accumulators rescaled) when a logit of this unit exceeds it by more than kMaxSlack.
+      if (__any_sync(0xffffffffu, (u0 > m0 + kMaxSlack) || (u1 > m1 + kMaxSlack))) {
 #pragma unroll
-      for (int off = 4; off < 32; off <<= 1) {
-        u0 = fmaxf(u0, __shfl_xor_sync(0xffffffffu, u0, off));
-        u1 = fmaxf(u1, __shfl_xor_sync(0xffffffffu, u1, off));
-      }
-      const float n0 = fmaxf(m0, fmaf(u0, scale_log2e, zl0)), n1 = fmaxf(m1, fmaf(u1, scale_log2e, zl1));
-      if (__any_sync(0xffffffffu, (n0 > m0) || (n1 > m1))) {
+        for (int off = 4; off < 32; off <<= 1) {
+          u0 = fmaxf(u0, __shfl_xor_sync(0xffffffffu, u0, off));
+          u1 = fmaxf(u1, __shfl_xor_sync(0xffffffffu, u1, off));
+        }
+        const float n0 = fmaxf(m0, u0), n1 = fmaxf(m1, u1);
         const float a0 = exp2f(m0 - n0), a1 = exp2f(m1 - n1);    // exp2(-inf) = 0 on the first unit
 #pragma unroll
         for (int ct = 0; ct < 8; ++ct) {
@@ -535,8 +545,8 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
       // ---- zero-point and denominator tile: rows 0..VG-1 = z_v of the group, row 4 = ones, the rest zero
 #pragma unroll
       for (int ks = 0; ks < 2; ++ks) {
-        const uint2 zz = *reinterpret_cast<const uint2*>(&zvp[((ks * 8 + r) * 4 + t) * 2]);
-        mma_f16(Zc, zz.x, 0u, zz.y, 0u, Pt[ks][0], Pt[ks][1]);
+        const uint4 zz = *reinterpret_cast<const uint4*>(&zvp[((ks * 8 + r) * 4 + t) * 4]);
+        mma_f16(Zc, zz.x, zz.y, zz.z, zz.w, Pt[ks][0], Pt[ks][1]);
       }
       // ---- P.V: codes as fp16 subnormals, scales folded into P
       {
@@ -545,11 +555,9 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
         const uint32_t vw[8] = {vw0.x, vw0.y, vw0.z, vw0.w, vw1.x, vw1.y, vw1.z, vw1.w};
 #pragma unroll
         for (int vg = 0; vg < VG; ++vg) {
-          uint32_t Bp[2][2];
-#pragma unroll
-          for (int ks = 0; ks < 2; ++ks)
-#pragma unroll
-            for (int ch = 0; ch < 2; ++ch) Bp[ks][ch] = hmul2_u(Pt[ks][ch], svp[((ks * 2 + ch) * 4 + t) * 4 + vg]);
+          const uint4 sv = *reinterpret_cast<const uint4*>(&svp[(t * 4 + vg) * 4]);
+          const uint32_t Bp[2][2] = {{hmul2_u(Pt[0][0], sv.x), hmul2_u(Pt[0][1], sv.y)},
+                                     {hmul2_u(Pt[1][0], sv.z), hmul2_u(Pt[1][1], sv.w)}};
 #pragma unroll
           for (int c = 0; c < TPG; ++c) {
             const int ct = vg * TPG + c;
@@ -599,6 +607,8 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
       if ((xv - packed_units) % kResidualWeight != 0) continue;       // the warp owning a unit's first position runs it
       const int x = packed_units + (xv - packed_units) / kResidualWeight;
       const uint32_t rbar = smem_u32(&bars[kWarps * kStages + warp]);
+      const uint16_t* resk = reinterpret_cast<const uint16_t*>(lv.resk + (size_t)s * lv.resk_stride);
+      const uint16_t* resv = reinterpret_cast<const uint16_t*>(lv.resv + (size_t)s * lv.resv_stride);
       // fused decode step: the newest token (slot r - 1) is not in the residual store yet; the warp whose unit holds it
       // takes its rows from the step's tensors (into the staged tile and into the store) and updates the accumulator
       const int jn = lv.r - 1;
@@ -802,9 +812,9 @@ template <int G>
 cudaError_t launch_g(const LayerView& lv, const void* q, float scale, float* ws, int grid, cudaStream_t stream) {
   const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q);
   const float sl = scale * 1.4426950408889634f;
-  if (lv.dense_hi) attention_mma_kernel<G, 2><<<grid, kWarps * 32, kSmemBytes, stream>>>(lv, qb, sl, ws);
-  else if (lv.tau_u4 < lv.tau_bf16) attention_mma_kernel<G, 1><<<grid, kWarps * 32, kSmemBytes, stream>>>(lv, qb, sl, ws);
-  else attention_mma_kernel<G, 0><<<grid, kWarps * 32, kSmemBytes, stream>>>(lv, qb, sl, ws);
+  if (lv.dense_hi) attention_mma_kernel<G, 2><<<grid, kWarps * 32, kSmemBytes, stream>>>(lv, qb, sl, ws, 0x44004400u);
+  else if (lv.tau_u4 < lv.tau_bf16) attention_mma_kernel<G, 1><<<grid, kWarps * 32, kSmemBytes, stream>>>(lv, qb, sl, ws, 0x44004400u);
+  else attention_mma_kernel<G, 0><<<grid, kWarps * 32, kSmemBytes, stream>>>(lv, qb, sl, ws, 0x44004400u);
   return cudaGetLastError();
 }
 

@@ -28,7 +28,7 @@ constexpr int kStages = 3;
 constexpr int kStageBytes = 3072;            // one key-meta group (512 B) followed by the unit (<= 2560 B), as in the block
 constexpr int kKeyMetaOff = 0;
 constexpr int kUnitOff = 512;
-constexpr int kPrepBytes = 2304;             // kprep 512 | zprep 512 | svp 256 | zvp 1024
+constexpr int kPrepBytes = 2432;             // kprep 576 | zprep 576 | svp 256 | zvp 1024
 constexpr int kSharedTail = 128 + 2048 + 2048 + 128 + 128 + 4096;
 constexpr int kSmemBytes = kWarps * (kStages * kStageBytes + kPrepBytes) + kSharedTail;
 constexpr int kCtasPerSm = 4;
@@ -68,27 +68,27 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
 
 __device__ __forceinline__ void mma_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                         uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 // d = a * b + c with the accumulator input in other registers than the result
 __device__ __forceinline__ void mma_f16_to(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                            uint32_t b1, float c0, float c1, float c2, float c3) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%12,%13};"
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%12,%13};"
                : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(c0), "f"(c1), "f"(c2), "f"(c3));
 }
 __device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1) {
-  asm volatile(
+  asm(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
   uint32_t y;
-  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+  asm("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
   return y;
 }
 __device__ __forceinline__ uint32_t hfma2_u(uint32_t a, uint32_t b, uint32_t c) {
@@ -116,6 +116,9 @@ __device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 
 // two bf16 in one word -> two fp16 in one word (exact inside the fp16 range)
 __device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t w) { return pack_half2(bf_lo(w), bf_hi(w)); }
 
+// First 32-bit word of k-tile kt in the per-warp scale and zero-point tables (16 words per k-tile; the extra four words
+// every second k-tile keep the stores of the preparation step free of bank conflicts).
+__device__ __forceinline__ constexpr int prep_word(int kt) { return 16 * kt + 4 * (kt >> 1); }
 // Bit position (inside each 16-bit half, after the shift below) of k-tile kt's 2-bit field.
 __device__ __forceinline__ constexpr int key_pos(int kt) { return (0x86486464u >> (4 * kt)) & 0xF; }
 // k-tiles 0,1 are read from (w << 4), 2..4 from w, 5..7 from (w >> 6)
@@ -134,11 +137,11 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
 
   unsigned char* ring = smem + warp * (kStages * kStageBytes);
   unsigned char* prep = smem + kWarps * kStages * kStageBytes + warp * kPrepBytes;
-  uint32_t* kprep = reinterpret_cast<uint32_t*>(prep);          // [8 kt][4 t]{m2 ch0, o2 ch0, m2 ch1, o2 ch1}
+  uint32_t* kprep = reinterpret_cast<uint32_t*>(prep);          // [8 kt: prep_word][4 t]{m2 ch0, o2 ch0, m2 ch1, o2 ch1}
   // the zero-point tiles are stored as whole A fragments (four registers), so one 16-byte load feeds the MMA
-  uint32_t* zprep = reinterpret_cast<uint32_t*>(prep + 512);    // [8 kt][4 t]{z ch0, z ch0, z ch1, z ch1} half2 z / mult
-  uint32_t* svp = reinterpret_cast<uint32_t*>(prep + 1024);     // [4 t][4 vg][2 ks][2 ch] half2 s_v'
-  uint32_t* zvp = reinterpret_cast<uint32_t*>(prep + 1280);     // [2 ks][8 rows][4 t]{ch0, 0, ch1, 0} half2: rows < VG z_v, row 4 ones
+  uint32_t* zprep = reinterpret_cast<uint32_t*>(prep + 576);    // [8 kt][4 t]{z ch0, z ch0, z ch1, z ch1} half2 z / mult
+  uint32_t* svp = reinterpret_cast<uint32_t*>(prep + 1152);     // [4 t][4 vg][2 ks][2 ch] half2 s_v'
+  uint32_t* zvp = reinterpret_cast<uint32_t*>(prep + 1408);     // [2 ks][8 rows][4 t]{ch0, 0, ch1, 0} half2: rows < VG z_v, row 4 ones
   unsigned char* tail = smem + kWarps * (kStages * kStageBytes + kPrepBytes);
   uint64_t* bars = reinterpret_cast<uint64_t*>(tail);           // [kWarps][kStages]
   uint16_t* qb16 = reinterpret_cast<uint16_t*>(tail + 128);     // [8][128] q, bf16 bits (0 for heads >= g)
@@ -162,7 +165,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
   // per-lane constants of the per-unit preparation steps
   // keys: the lane converts channels 4*lane .. 4*lane+3 (k-tile lane / 4)
   const float pk_zs = __uint_as_float((119u + (uint32_t)key_pos(lane >> 2)) << 23);        // 2^(pos - 8)
-  const int pk_kp = (((lane >> 2) * 4 + 2 * (lane & 1)) * 4 + ((lane & 3) >> 1) * 2);      // kprep word of the first pair
+  const int pk_kp = prep_word(lane >> 2) + 8 * (lane & 1) + ((lane & 3) >> 1) * 2;         // kprep word of the first pair
   const int pk_zp = pk_kp;                                                                  // zprep word of the first pair
   // values: the lane converts the scales and zero-points of token `lane`
   const float pv_up = __uint_as_float((131u - 2u * (uint32_t)(lane >> 3)) << 23);          // 2^(4 - 2 * (2 ks + ch))
@@ -316,32 +319,6 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
       const unsigned char* st = stg + kUnitOff;        // the unit's codes and value scales
       const bool has_meta = (UPG == 1) || (consumed == 0) || ((u & (UPG - 1)) == 0);
 
-      // ---- key-group preparation: fp16 scale pairs in fragment order, zero-point tile
-      if (has_meta) {
-        const uint4 mz = reinterpret_cast<const uint4*>(stg + kKeyMetaOff)[lane];   // channels 4*lane .. 4*lane+3
-        const uint32_t ma = pack_half2(bf_lo(mz.x), bf_lo(mz.y)), mb = pack_half2(bf_lo(mz.z), bf_lo(mz.w));
-        const uint32_t neg4 = 0xC400C400u;   // half2(-4, -4)
-        __syncwarp();
-        *reinterpret_cast<uint2*>(&kprep[pk_kp]) = make_uint2(ma, hmul2_u(ma, neg4));
-        *reinterpret_cast<uint2*>(&kprep[pk_kp + 4]) = make_uint2(mb, hmul2_u(mb, neg4));
-        const uint32_t za = pack_half2(bf_hi(mz.x) * pk_zs, bf_hi(mz.y) * pk_zs);
-        const uint32_t zb = pack_half2(bf_hi(mz.z) * pk_zs, bf_hi(mz.w) * pk_zs);
-        *reinterpret_cast<uint2*>(&zprep[pk_zp]) = make_uint2(za, za);
-        *reinterpret_cast<uint2*>(&zprep[pk_zp + 4]) = make_uint2(zb, zb);
-        __syncwarp();
-        // the zero-point term q . z of the group: its own accumulator chain, added to the logits after the key tiles
-        // (the tile's rows are equal, so are the rows of the result)
-        float zc[4];
-#pragma unroll
-        for (int kt2 = 0; kt2 < 8; ++kt2) {
-          const uint4 zz = *reinterpret_cast<const uint4*>(&zprep[(kt2 * 4 + t) * 4]);
-          if (kt2 == 0) mma_f16_to(zc, zz.x, zz.y, zz.z, zz.w, bq[0][0], bq[0][1], 0.f, 0.f, 0.f, 0.f);
-          else mma_f16(zc, zz.x, zz.y, zz.z, zz.w, bq[kt2][0], bq[kt2][1]);
-        }
-        zl0 = zc[0] * scale_log2e;
-        zl1 = zc[1] * scale_log2e;
-      }
-
       // ---- extras of this unit: issue the global loads early (BF16 pairs of the first 16 promoted channels)
       uint32_t xa[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};
       if (n16 > 0) {
@@ -362,15 +339,58 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
         }
       }
 
+      // the key codes: two 16-byte loads per lane are the A fragments of all sixteen key tiles
+      const uint4 kw0 = reinterpret_cast<const uint4*>(st)[lane];
+      const uint4 kw1 = reinterpret_cast<const uint4*>(st)[32 + lane];
+
+      // ---- value-group preparation (lane = token).  The tables of the previous unit were last read before the
+      // warp barrier that closed it, so they can be overwritten right away.
+      {
+        const uint32_t* vmeta = reinterpret_cast<const uint32_t*>(st + 2048) + lane * VG;
+        __half* svh = reinterpret_cast<__half*>(svp) + pv_sv;
+        __half* zvh = reinterpret_cast<__half*>(zvp) + pv_zv;
+#pragma unroll
+        for (int vg = 0; vg < VG; ++vg) {
+          const uint32_t mz = vmeta[vg];
+          svh[8 * vg] = __float2half_rn(bf_lo(mz) * pv_up);
+          zvh[32 * vg] = __float2half_rn(bf_hi(mz));
+        }
+      }
+
+      // ---- key-group preparation: fp16 scale pairs in fragment order, zero-point tile
+      if (has_meta) {
+        const uint4 mz = reinterpret_cast<const uint4*>(stg + kKeyMetaOff)[lane];   // channels 4*lane .. 4*lane+3
+        const uint32_t ma = pack_half2(bf_lo(mz.x), bf_lo(mz.y)), mb = pack_half2(bf_lo(mz.z), bf_lo(mz.w));
+        const uint32_t neg4 = 0xC400C400u;   // half2(-4, -4)
+        *reinterpret_cast<uint2*>(&kprep[pk_kp]) = make_uint2(ma, hmul2_u(ma, neg4));
+        *reinterpret_cast<uint2*>(&kprep[pk_kp + 4]) = make_uint2(mb, hmul2_u(mb, neg4));
+        const uint32_t za = pack_half2(bf_hi(mz.x) * pk_zs, bf_hi(mz.y) * pk_zs);
+        const uint32_t zb = pack_half2(bf_hi(mz.z) * pk_zs, bf_hi(mz.w) * pk_zs);
+        *reinterpret_cast<uint2*>(&zprep[pk_zp]) = make_uint2(za, za);
+        *reinterpret_cast<uint2*>(&zprep[pk_zp + 4]) = make_uint2(zb, zb);
+      }
+      __syncwarp();      // the tables written above are read by other lanes below
+      if (has_meta) {
+        // the zero-point term q . z of the group: its own accumulator chain, added to the logits after the key tiles
+        // (the tile's rows are equal, so are the rows of the result)
+        float zc[4];
+#pragma unroll
+        for (int kt2 = 0; kt2 < 8; ++kt2) {
+          const uint4 zz = *reinterpret_cast<const uint4*>(&zprep[prep_word(kt2) + 4 * t]);
+          if (kt2 == 0) mma_f16_to(zc, zz.x, zz.y, zz.z, zz.w, bq[0][0], bq[0][1], 0.f, 0.f, 0.f, 0.f);
+          else mma_f16(zc, zz.x, zz.y, zz.z, zz.w, bq[kt2][0], bq[kt2][1]);
+        }
+        zl0 = zc[0] * scale_log2e;
+        zl1 = zc[1] * scale_log2e;
+      }
+
       // ---- q.K^T on the base (2-bit low plane) tiles
       float Sx[2][4];
       {
-        const uint4 kw0 = reinterpret_cast<const uint4*>(st)[lane];
-        const uint4 kw1 = reinterpret_cast<const uint4*>(st)[32 + lane];
         const uint32_t kw[2][4] = {{kw0.x, kw0.y, kw0.z, kw0.w}, {kw1.x, kw1.y, kw1.z, kw1.w}};
 #pragma unroll
         for (int kt = 0; kt < 8; ++kt) {
-          const uint4 kp = *reinterpret_cast<const uint4*>(&kprep[(kt * 4 + t) * 4]);
+          const uint4 kp = *reinterpret_cast<const uint4*>(&kprep[prep_word(kt) + 4 * t]);
           const uint32_t mask = 0x00030003u << key_pos(kt);
 #pragma unroll
           for (int mt = 0; mt < 2; ++mt) {
@@ -393,7 +413,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
         const uint32_t kw[2][4] = {{hw0.x, hw0.y, hw0.z, hw0.w}, {hw1.x, hw1.y, hw1.z, hw1.w}};
 #pragma unroll
         for (int kt = 0; kt < 8; ++kt) {
-          const uint4 kp = *reinterpret_cast<const uint4*>(&kprep[(kt * 4 + t) * 4]);
+          const uint4 kp = *reinterpret_cast<const uint4*>(&kprep[prep_word(kt) + 4 * t]);
           const uint32_t m0 = hmul2_u(kp.x, 0x44004400u), o0 = hmul2_u(kp.y, 0x44004400u);
           const uint32_t m1 = hmul2_u(kp.z, 0x44004400u), o1 = hmul2_u(kp.w, 0x44004400u);
           const uint32_t mask = 0x00030003u << key_pos(kt);
@@ -469,7 +489,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
               auto scale_of = [&](uint32_t c) -> __half {
                 // fp16 scale of channel c in kprep: [(kt*4 + t')*4 + ch*2] half2, element e
                 const int kt = c >> 4, col = c & 15;
-                return kph[(((kt * 4 + ((col & 7) >> 1)) * 4 + (col >> 3) * 2) << 1) + (col & 1)];
+                return kph[((prep_word(kt) + ((col & 7) >> 1) * 4 + (col >> 3) * 2) << 1) + (col & 1)];
               };
               const __half zero = __float2half_rn(0.f);
               const __half s0 = (c0 < 128) ? scale_of(c0) : zero, s1 = (c1 < 128) ? scale_of(c1) : zero;
@@ -491,19 +511,6 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
           }
 #pragma unroll
           for (int mt = 0; mt < 2; ++mt) mma_f16(Sx[mt], a[mt][0], a[mt][1], a[mt][2], a[mt][3], b[0], b[1]);
-        }
-      }
-
-      // ---- value-group preparation (lane = token)
-      {
-        const uint32_t* vmeta = reinterpret_cast<const uint32_t*>(st + 2048) + lane * VG;
-        __half* svh = reinterpret_cast<__half*>(svp) + pv_sv;
-        __half* zvh = reinterpret_cast<__half*>(zvp) + pv_zv;
-#pragma unroll
-        for (int vg = 0; vg < VG; ++vg) {
-          const uint32_t mz = vmeta[vg];
-          svh[8 * vg] = __float2half_rn(bf_lo(mz) * pv_up);
-          zvh[32 * vg] = __float2half_rn(bf_hi(mz));
         }
       }
 
@@ -540,7 +547,6 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
         Pt[mt][0] = movmatrix_trans(plo);
         Pt[mt][1] = movmatrix_trans(phi);
       }
-      __syncwarp();   // svp / zvp written above are read below
 
       // ---- zero-point and denominator tile: rows 0..VG-1 = z_v of the group, row 4 = ones, the rest zero
 #pragma unroll

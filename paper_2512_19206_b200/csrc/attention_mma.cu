@@ -14,6 +14,8 @@
 //           and the softmax denominator through one extra tile (rows = value groups and a row of ones).
 //   promoted (BF16) key channels and the UINT4 high plane come from the block's extras with a gathered q.
 //   residual (unquantized) tokens use bf16 tiles straight from global memory.
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace mixkvq {
@@ -29,12 +31,14 @@ constexpr int kStageBytes = 3072;            // one key-meta group (512 B) follo
 constexpr int kKeyMetaOff = 0;
 constexpr int kUnitOff = 512;
 constexpr int kPrepBytes = 2432;             // kprep 576 | zprep 576 | svp 256 | zvp 1024
-constexpr int kSharedTail = 128 + 2048 + 2048 + 128 + 128 + 4096;
+constexpr int kSharedTail = 128 + 2048 + 2048 + 128 + 128;
 constexpr int kSmemBytes = kWarps * (kStages * kStageBytes + kPrepBytes) + kSharedTail;
 constexpr int kCtasPerSm = 4;
+constexpr int kCtasPerSmDense = 3;           // with a 4-bit base two key planes are in flight: more registers per thread, fewer CTAs
 static_assert((kWarps * kStages + kWarps) * 8 <= 128, "the mbarrier area at the start of the shared tail holds 16 barriers");
 constexpr int kResidualWeight = 2;           // a 32-token unit of the residual window counts as this many packed units in the split
 constexpr uint32_t kSpinLimit = 1u << 22;    // bounded wait on a staged copy
+constexpr int kMergeStride = 132;            // floats per head row of a warp's output in the merge (bank-conflict-free stores)
 constexpr float kMaxSlack = 3.0f;            // a packed unit's probabilities are at most 2^kMaxSlack (log2 domain)
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -127,7 +131,7 @@ __device__ __forceinline__ uint32_t key_shift(uint32_t w, int kt) { return kt < 
 // kU4: how the configuration can use the UINT4 tier: 0 = never (tau_u4 >= tau_bf16), 1 = some channels (high plane stored
 // per channel pair, gathered), 2 = 4-bit base (dense high plane)
 template <int G, int kU4>
-__global__ void __launch_bounds__(kWarps * 32, kCtasPerSm)
+__global__ void __launch_bounds__(kWarps * 32, kU4 == 2 ? kCtasPerSmDense : kCtasPerSm)
 attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float scale_log2e, float* __restrict__ ws,
                      uint32_t four2) {
   constexpr int VG = kD / G;              // value groups per token
@@ -148,7 +152,6 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
   __half* qf16 = reinterpret_cast<__half*>(tail + 128 + 2048);  // [8][128] q, fp16
   float* mS = reinterpret_cast<float*>(tail + 128 + 4096);      // [4][8]
   float* lS = mS + 32;                                          // [4][8]
-  float* oS = lS + 32;                                          // [8][128]
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < kWarps * kStages + kWarps; ++i) mbar_init(smem_u32(&bars[i]), 1);   // rings + one per warp for the residual window
@@ -285,6 +288,26 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
       for (int i = 0; i < 4; ++i) O[ct][i] = 0.f;
     bool o_true_scale = false;
 
+    // A fragments of the first 16 promoted channels of a unit: lane (r, t) holds channel pairs t and t + 4 for tokens
+    // r, r + 8 of both m-tiles.  Pairs past the block's count read an existing pair instead (their query entries are 0).
+    uint32_t xa[2][4];
+    bool xa_loaded = false;
+    auto load_xa = [&](const char* e) {
+      const uint32_t* xw = reinterpret_cast<const uint32_t*>(e) + (min(t, n16p - 1) * 32 + r);
+#pragma unroll
+      for (int mt = 0; mt < 2; ++mt) {
+        xa[mt][0] = xw[mt * 16];
+        xa[mt][1] = xw[mt * 16 + 8];
+      }
+      if (n16p > 4) {       // more than 8 promoted channels (uniform over the warp)
+        const uint32_t* xv = reinterpret_cast<const uint32_t*>(e) + (min(t + 4, n16p - 1) * 32 + r);
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+          xa[mt][2] = xv[mt * 16];
+          xa[mt][3] = xv[mt * 16 + 8];
+        }
+      }
+    };
     int consumed = 0;
     for (; consumed < n_pack && !gave_up; ++consumed) {
       if (new_block) {
@@ -310,6 +333,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
           xb1 = gather_q(t + 4);
         }
         new_block = false;
+        xa_loaded = false;
       }
       if (!mbar_wait_bounded(bar_u32 + ring_stage * 8u, ring_parity)) {
         gave_up = true;
@@ -319,29 +343,13 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
       const unsigned char* st = stg + kUnitOff;        // the unit's codes and value scales
       const bool has_meta = (UPG == 1) || (consumed == 0) || ((u & (UPG - 1)) == 0);
 
-      // ---- extras of this unit: issue the global loads early (BF16 pairs of the first 16 promoted channels)
-      uint32_t xa[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};
-      if (n16 > 0) {
-        const uint32_t* xw = reinterpret_cast<const uint32_t*>(exu) + (t * 32 + r);
-        const bool p0 = t < n16p;
-#pragma unroll
-        for (int mt = 0; mt < 2; ++mt) {
-          xa[mt][0] = p0 ? xw[mt * 16] : 0u;
-          xa[mt][1] = p0 ? xw[mt * 16 + 8] : 0u;
-        }
-        if (n16p > 4) {       // more than 8 promoted channels (uniform over the warp)
-          const bool p1 = t + 4 < n16p;
-#pragma unroll
-          for (int mt = 0; mt < 2; ++mt) {
-            xa[mt][2] = p1 ? xw[128 + mt * 16] : 0u;
-            xa[mt][3] = p1 ? xw[128 + mt * 16 + 8] : 0u;
-          }
-        }
-      }
-
-      // the key codes: two 16-byte loads per lane are the A fragments of all sixteen key tiles
-      const uint4 kw0 = reinterpret_cast<const uint4*>(st)[lane];
-      const uint4 kw1 = reinterpret_cast<const uint4*>(st)[32 + lane];
+      // ---- extras of this unit (BF16 pairs of the first 16 promoted channels), unless the previous unit already
+      // requested them
+      if (n16 > 0 && !xa_loaded) load_xa(exu);
+      // the key codes: two 16-byte loads per lane are the A fragments of all sixteen key tiles (with a 4-bit base the
+      // first plane to run is the high plane, which lies with the block's extras in global memory)
+      const uint4* kplane = (kU4 == 2) ? reinterpret_cast<const uint4*>(exu + 128 * n16p) : reinterpret_cast<const uint4*>(st);
+      const uint4 hw0 = kplane[lane], hw1 = kplane[32 + lane];
 
       // ---- value-group preparation (lane = token).  The tables of the previous unit were last read before the
       // warp barrier that closed it, so they can be overwritten right away.
@@ -384,13 +392,16 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
         zl1 = zc[1] * scale_log2e;
       }
 
-      // ---- q.K^T on the base (2-bit low plane) tiles
+      // ---- q.K^T on the key tiles.  One pass over a plane of 2-bit codes: the base (low) plane with the scales s, and,
+      // with a 4-bit base, first the dense high plane (codes c >> 2, laid out like the low plane) with the scales 4s.
       float Sx[2][4];
-      {
-        const uint32_t kw[2][4] = {{kw0.x, kw0.y, kw0.z, kw0.w}, {kw1.x, kw1.y, kw1.z, kw1.w}};
+      auto key_pass = [&](const uint4& w0, const uint4& w1, auto first_tag, auto high_tag) {
+        constexpr bool first = decltype(first_tag)::value, high = decltype(high_tag)::value;
+        const uint32_t kw[2][4] = {{w0.x, w0.y, w0.z, w0.w}, {w1.x, w1.y, w1.z, w1.w}};
 #pragma unroll
         for (int kt = 0; kt < 8; ++kt) {
-          const uint4 kp = *reinterpret_cast<const uint4*>(&kprep[prep_word(kt) + 4 * t]);
+          uint4 kp = *reinterpret_cast<const uint4*>(&kprep[prep_word(kt) + 4 * t]);
+          if (high) kp = make_uint4(hmul2_u(kp.x, four2), hmul2_u(kp.y, four2), hmul2_u(kp.z, four2), hmul2_u(kp.w, four2));
           const uint32_t mask = 0x00030003u << key_pos(kt);
 #pragma unroll
           for (int mt = 0; mt < 2; ++mt) {
@@ -400,64 +411,51 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
               const uint32_t code = (key_shift(kw[mt][j], kt) & mask) | four2;           // 4 + c * 2^(pos-8)
               a[j] = hfma2_u(code, j < 2 ? kp.x : kp.z, j < 2 ? kp.y : kp.w);            // c * s * 2^(pos-8)
             }
-            if (kt == 0) mma_f16_to(Sx[mt], a[0], a[1], a[2], a[3], bq[0][0], bq[0][1], 0.f, 0.f, 0.f, 0.f);
+            if (first && kt == 0) mma_f16_to(Sx[mt], a[0], a[1], a[2], a[3], bq[0][0], bq[0][1], 0.f, 0.f, 0.f, 0.f);
             else mma_f16(Sx[mt], a[0], a[1], a[2], a[3], bq[kt][0], bq[kt][1]);
           }
         }
-      }
-      // ---- dense UINT4 high plane: the same tiles with codes c >> 2 and four times the scale
+      };
       if constexpr (kU4 == 2) {
-        // laid out like the low plane: two 16-byte loads per lane
-        const uint4* hp = reinterpret_cast<const uint4*>(exu + 128 * n16p);
-        const uint4 hw0 = hp[lane], hw1 = hp[32 + lane];
-        const uint32_t kw[2][4] = {{hw0.x, hw0.y, hw0.z, hw0.w}, {hw1.x, hw1.y, hw1.z, hw1.w}};
-#pragma unroll
-        for (int kt = 0; kt < 8; ++kt) {
-          const uint4 kp = *reinterpret_cast<const uint4*>(&kprep[prep_word(kt) + 4 * t]);
-          const uint32_t m0 = hmul2_u(kp.x, 0x44004400u), o0 = hmul2_u(kp.y, 0x44004400u);
-          const uint32_t m1 = hmul2_u(kp.z, 0x44004400u), o1 = hmul2_u(kp.w, 0x44004400u);
-          const uint32_t mask = 0x00030003u << key_pos(kt);
-#pragma unroll
-          for (int mt = 0; mt < 2; ++mt) {
-            uint32_t a[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const uint32_t code = (key_shift(kw[mt][j], kt) & mask) | 0x44004400u;
-              a[j] = hfma2_u(code, j < 2 ? m0 : m1, j < 2 ? o0 : o1);
-            }
-            mma_f16(Sx[mt], a[0], a[1], a[2], a[3], bq[kt][0], bq[kt][1]);
-          }
-        }
+        key_pass(hw0, hw1, std::true_type{}, std::true_type{});
+        const uint4 kw0 = reinterpret_cast<const uint4*>(st)[lane];
+        const uint4 kw1 = reinterpret_cast<const uint4*>(st)[32 + lane];
+        key_pass(kw0, kw1, std::false_type{}, std::false_type{});
+      } else {
+        key_pass(hw0, hw1, std::true_type{}, std::false_type{});
       }
       // ---- promoted channels (raw bf16 keys) with a gathered q
       if (n16 > 0) {
-        for (int kk = 0; kk * 8 < n16p; ++kk) {
+        if (n16p > 4) {
+#pragma unroll
+          for (int mt = 0; mt < 2; ++mt) mma_bf16(Sx[mt], xa[mt][0], xa[mt][1], xa[mt][2], xa[mt][3], xb0, xb1);
+        } else {
+#pragma unroll
+          for (int mt = 0; mt < 2; ++mt) mma_bf16(Sx[mt], xa[mt][0], xa[mt][1], 0u, 0u, xb0, 0u);
+        }
+        // the registers are free again: request the next unit's pairs now, most of an iteration ahead of their use
+        xa_loaded = (u + 1 < U) && (consumed + 1 < n_pack);
+        if (xa_loaded) load_xa(exu + ex_unit);
+        for (int kk = 1; kk * 8 < n16p; ++kk) {       // more than 16 promoted channels
           uint32_t a[2][4], id0 = 0xFFFFFFFFu, id1 = 0xFFFFFFFFu;
-          if (kk == 0) {
+          const uint32_t* xw = reinterpret_cast<const uint32_t*>(exu);
+          const int p0 = 8 * kk + t, p1 = p0 + 4;
 #pragma unroll
-            for (int mt = 0; mt < 2; ++mt) mma_bf16(Sx[mt], xa[mt][0], xa[mt][1], xa[mt][2], xa[mt][3], xb0, xb1);
-            continue;
-          } else {
-            const uint32_t* xw = reinterpret_cast<const uint32_t*>(exu);
-            const int p0 = 8 * kk + t, p1 = p0 + 4;
-            id0 = id1 = 0xFFFFFFFFu;
+          for (int mt = 0; mt < 2; ++mt) a[mt][0] = a[mt][1] = a[mt][2] = a[mt][3] = 0;
+          if (p0 < n16p) {
+            id0 = *reinterpret_cast<const uint16_t*>(ex + 2 * p0);
 #pragma unroll
-            for (int mt = 0; mt < 2; ++mt) a[mt][0] = a[mt][1] = a[mt][2] = a[mt][3] = 0;
-            if (p0 < n16p) {
-              id0 = *reinterpret_cast<const uint16_t*>(ex + 2 * p0);
-#pragma unroll
-              for (int mt = 0; mt < 2; ++mt) {
-                a[mt][0] = xw[p0 * 32 + mt * 16 + r];
-                a[mt][1] = xw[p0 * 32 + mt * 16 + 8 + r];
-              }
+            for (int mt = 0; mt < 2; ++mt) {
+              a[mt][0] = xw[p0 * 32 + mt * 16 + r];
+              a[mt][1] = xw[p0 * 32 + mt * 16 + 8 + r];
             }
-            if (p1 < n16p) {
-              id1 = *reinterpret_cast<const uint16_t*>(ex + 2 * p1);
+          }
+          if (p1 < n16p) {
+            id1 = *reinterpret_cast<const uint16_t*>(ex + 2 * p1);
 #pragma unroll
-              for (int mt = 0; mt < 2; ++mt) {
-                a[mt][2] = xw[p1 * 32 + mt * 16 + r];
-                a[mt][3] = xw[p1 * 32 + mt * 16 + 8 + r];
-              }
+            for (int mt = 0; mt < 2; ++mt) {
+              a[mt][2] = xw[p1 * 32 + mt * 16 + r];
+              a[mt][3] = xw[p1 * 32 + mt * 16 + 8 + r];
             }
           }
           auto gather_bf16 = [&](uint32_t ids) -> uint32_t {
@@ -768,48 +766,56 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
     }
     const float l0 = __shfl_sync(0xffffffffu, Zc[0], 16 + t), l1 = __shfl_sync(0xffffffffu, Zc[1], 16 + t);
 
-    // ---- merge the warps of the CTA, write the partial of (CTA, stream)
+    // ---- merge the warps of the CTA, write the partial of (CTA, stream).  Every warp leaves its (m, l) and its
+    // unnormalized output in shared memory, the output in its own, now idle, ring as [8 heads][132] floats; then
+    // the 16 threads that own a head add the four warps' rows with the factors 2^(m_w - M).
     if (r == 0) {
       mS[warp * 8 + 2 * t] = m0;
       mS[warp * 8 + 2 * t + 1] = m1;
       lS[warp * 8 + 2 * t] = l0;
       lS[warp * 8 + 2 * t + 1] = l1;
     }
-    for (int i = threadIdx.x; i < 8 * kD; i += kWarps * 32) oS[i] = 0.f;
-    __syncthreads();
     {
-      float M0 = -INFINITY, M1 = -INFINITY;
+      float* mine = reinterpret_cast<float*>(ring);
 #pragma unroll
-      for (int w = 0; w < kWarps; ++w) {
-        M0 = fmaxf(M0, mS[w * 8 + 2 * t]);
-        M1 = fmaxf(M1, mS[w * 8 + 2 * t + 1]);
-      }
-      const float f0 = (m0 == -INFINITY) ? 0.f : exp2f(m0 - M0), f1 = (m1 == -INFINITY) ? 0.f : exp2f(m1 - M1);
-      if (m0 != -INFINITY || m1 != -INFINITY) {
-#pragma unroll
-        for (int ct = 0; ct < 8; ++ct) {
-          atomicAdd(&oS[(2 * t) * kD + 16 * ct + r], f0 * O[ct][0]);
-          atomicAdd(&oS[(2 * t + 1) * kD + 16 * ct + r], f1 * O[ct][1]);
-          atomicAdd(&oS[(2 * t) * kD + 16 * ct + 8 + r], f0 * O[ct][2]);
-          atomicAdd(&oS[(2 * t + 1) * kD + 16 * ct + 8 + r], f1 * O[ct][3]);
-        }
+      for (int ct = 0; ct < 8; ++ct) {
+        mine[(2 * t) * kMergeStride + 16 * ct + r] = O[ct][0];
+        mine[(2 * t + 1) * kMergeStride + 16 * ct + r] = O[ct][1];
+        mine[(2 * t) * kMergeStride + 16 * ct + 8 + r] = O[ct][2];
+        mine[(2 * t + 1) * kMergeStride + 16 * ct + 8 + r] = O[ct][3];
       }
     }
     __syncthreads();
     {
-      float* part = ws + (size_t)(blockIdx.x + s) * kPartialFloats;
-      for (int i = threadIdx.x; i < 8 * kD; i += kWarps * 32) part[(i >> 7) * 130 + 2 + (i & 127)] = oS[i];
-      if (threadIdx.x < 8) {
-        const int h = threadIdx.x;
-        float M = -INFINITY, L = 0.f;
-        for (int w = 0; w < kWarps; ++w) M = fmaxf(M, mS[w * 8 + h]);
-        for (int w = 0; w < kWarps; ++w) {
-          const float mw = mS[w * 8 + h];
-          L += (mw == -INFINITY) ? 0.f : exp2f(mw - M) * lS[w * 8 + h];
-        }
-        part[h * 130] = M;
-        part[h * 130 + 1] = L;
+      const int h = threadIdx.x >> 4, c0 = threadIdx.x & 15;
+      float M = -INFINITY, L = 0.f, f[kWarps];
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) M = fmaxf(M, mS[w * 8 + h]);
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) {
+        const float mw = mS[w * 8 + h];
+        f[w] = (mw == -INFINITY) ? 0.f : exp2f(mw - M);
+        L += f[w] * lS[w * 8 + h];
       }
+      float* part = ws + (size_t)(blockIdx.x + s) * kPartialFloats + h * 130;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const int c = c0 + 16 * k;
+        float acc = 0.f;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w)
+          acc += f[w] * reinterpret_cast<const float*>(smem + w * (kStages * kStageBytes))[h * kMergeStride + c];
+        part[2 + c] = acc;
+      }
+      if (c0 == 0) {
+        part[0] = M;
+        part[1] = L;
+      }
+    }
+    if (seg < ce) {
+      // another segment follows: its copies are staged into the rings that were just read
+      __syncthreads();
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
   }
 }
@@ -863,7 +869,7 @@ long long attention_mma_positions(const LayerView& lv) {
 int attention_mma_grid(const LayerView& lv, int n_sms) {
   const int S = lv.B * lv.Hkv;
   const long long total = attention_mma_positions(lv) * S;
-  int grid = (int)min((long long)min(n_sms * kCtasPerSm, kMaxCtas / 2), total);
+  int grid = (int)min((long long)min(n_sms * (lv.dense_hi ? kCtasPerSmDense : kCtasPerSm), kMaxCtas / 2), total);
   if (grid > S) grid = grid / S * S;
   return grid < 1 ? 1 : grid;
 }

@@ -33,7 +33,7 @@ constexpr int kUnitOff = 512;
 constexpr int kPrepBytes = 2432;             // kprep 576 | zprep 576 | svp 256 | zvp 1024
 constexpr int kSharedTail = 128 + 2048 + 2048 + 128 + 128;
 constexpr int kSmemBytes = kWarps * (kStages * kStageBytes + kPrepBytes) + kSharedTail;
-constexpr int kCtasPerSm = 4;
+constexpr int kCtasPerSm = 3;
 constexpr int kCtasPerSmDense = 3;           // with a 4-bit base two key planes are in flight: more registers per thread, fewer CTAs
 static_assert((kWarps * kStages + kWarps) * 8 <= 128, "the mbarrier area at the start of the shared tail holds 16 barriers");
 constexpr int kResidualWeight = 2;           // a 32-token unit of the residual window counts as this many packed units in the split
@@ -123,6 +123,8 @@ __device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t w) { return pack_ha
 // First 32-bit word of k-tile kt in the per-warp scale and zero-point tables (16 words per k-tile; the extra four words
 // every second k-tile keep the stores of the preparation step free of bank conflicts).
 __device__ __forceinline__ constexpr int prep_word(int kt) { return 16 * kt + 4 * (kt >> 1); }
+// The same for the scale table, which has two words per (k-tile, t): 8 words per k-tile, two extra after the fourth.
+__device__ __forceinline__ constexpr int scale_word(int kt) { return 8 * kt + 2 * (kt >> 2); }
 // Bit position (inside each 16-bit half, after the shift below) of k-tile kt's 2-bit field.
 __device__ __forceinline__ constexpr int key_pos(int kt) { return (0x86486464u >> (4 * kt)) & 0xF; }
 // k-tiles 0,1 are read from (w << 4), 2..4 from w, 5..7 from (w >> 6)
@@ -141,7 +143,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
 
   unsigned char* ring = smem + warp * (kStages * kStageBytes);
   unsigned char* prep = smem + kWarps * kStages * kStageBytes + warp * kPrepBytes;
-  uint32_t* kprep = reinterpret_cast<uint32_t*>(prep);          // [8 kt: prep_word][4 t]{m2 ch0, o2 ch0, m2 ch1, o2 ch1}
+  uint32_t* kprep = reinterpret_cast<uint32_t*>(prep);          // [8 kt: scale_word][4 t]{s ch0, s ch1} half2 (first 288 of 576 bytes)
   // the zero-point tiles are stored as whole A fragments (four registers), so one 16-byte load feeds the MMA
   uint32_t* zprep = reinterpret_cast<uint32_t*>(prep + 576);    // [8 kt][4 t]{z ch0, z ch0, z ch1, z ch1} half2 z / mult
   uint32_t* svp = reinterpret_cast<uint32_t*>(prep + 1152);     // [4 t][4 vg][2 ks][2 ch] half2 s_v'
@@ -168,8 +170,8 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
   // per-lane constants of the per-unit preparation steps
   // keys: the lane converts channels 4*lane .. 4*lane+3 (k-tile lane / 4)
   const float pk_zs = __uint_as_float((119u + (uint32_t)key_pos(lane >> 2)) << 23);        // 2^(pos - 8)
-  const int pk_kp = prep_word(lane >> 2) + 8 * (lane & 1) + ((lane & 3) >> 1) * 2;         // kprep word of the first pair
-  const int pk_zp = pk_kp;                                                                  // zprep word of the first pair
+  const int pk_zp = prep_word(lane >> 2) + 8 * (lane & 1) + ((lane & 3) >> 1) * 2;         // zprep word of the first pair
+  const int pk_kp = scale_word(lane >> 2) + 4 * (lane & 1) + ((lane & 3) >> 1);            // kprep word of the first pair
   // values: the lane converts the scales and zero-points of token `lane`
   const float pv_up = __uint_as_float((131u - 2u * (uint32_t)(lane >> 3)) << 23);          // 2^(4 - 2 * (2 ks + ch))
   const int pv_sv = ((((lane & 7) >> 1) * 16 + (lane >> 3)) * 2) + (lane & 1);             // svp half index of group 0
@@ -369,9 +371,8 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
       if (has_meta) {
         const uint4 mz = reinterpret_cast<const uint4*>(stg + kKeyMetaOff)[lane];   // channels 4*lane .. 4*lane+3
         const uint32_t ma = pack_half2(bf_lo(mz.x), bf_lo(mz.y)), mb = pack_half2(bf_lo(mz.z), bf_lo(mz.w));
-        const uint32_t neg4 = 0xC400C400u;   // half2(-4, -4)
-        *reinterpret_cast<uint2*>(&kprep[pk_kp]) = make_uint2(ma, hmul2_u(ma, neg4));
-        *reinterpret_cast<uint2*>(&kprep[pk_kp + 4]) = make_uint2(mb, hmul2_u(mb, neg4));
+        kprep[pk_kp] = ma;
+        kprep[pk_kp + 2] = mb;
         const uint32_t za = pack_half2(bf_hi(mz.x) * pk_zs, bf_hi(mz.y) * pk_zs);
         const uint32_t zb = pack_half2(bf_hi(mz.z) * pk_zs, bf_hi(mz.w) * pk_zs);
         *reinterpret_cast<uint2*>(&zprep[pk_zp]) = make_uint2(za, za);
@@ -400,7 +401,10 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
         const uint32_t kw[2][4] = {{w0.x, w0.y, w0.z, w0.w}, {w1.x, w1.y, w1.z, w1.w}};
 #pragma unroll
         for (int kt = 0; kt < 8; ++kt) {
-          uint4 kp = *reinterpret_cast<const uint4*>(&kprep[prep_word(kt) + 4 * t]);
+          // scales of the lane's channel pairs (16kt + 2t, +1) and (16kt + 8 + 2t, +1); code bias 4 -> offset -4 s
+          const uint2 sc = *reinterpret_cast<const uint2*>(&kprep[scale_word(kt) + 2 * t]);
+          const uint32_t neg4 = 0xC400C400u;   // half2(-4, -4)
+          uint4 kp = make_uint4(sc.x, hmul2_u(sc.x, neg4), sc.y, hmul2_u(sc.y, neg4));
           if (high) kp = make_uint4(hmul2_u(kp.x, four2), hmul2_u(kp.y, four2), hmul2_u(kp.z, four2), hmul2_u(kp.w, four2));
           const uint32_t mask = 0x00030003u << key_pos(kt);
 #pragma unroll
@@ -487,7 +491,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
               auto scale_of = [&](uint32_t c) -> __half {
                 // fp16 scale of channel c in kprep: [(kt*4 + t')*4 + ch*2] half2, element e
                 const int kt = c >> 4, col = c & 15;
-                return kph[((prep_word(kt) + ((col & 7) >> 1) * 4 + (col >> 3) * 2) << 1) + (col & 1)];
+                return kph[((scale_word(kt) + ((col & 7) >> 1) * 2 + (col >> 3)) << 1) + (col & 1)];
               };
               const __half zero = __float2half_rn(0.f);
               const __half s0 = (c0 < 128) ? scale_of(c0) : zero, s1 = (c1 < 128) ? scale_of(c1) : zero;

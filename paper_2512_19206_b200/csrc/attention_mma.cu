@@ -25,17 +25,18 @@ cudaError_t launch_combine(const float* ws, float* out, int g, int Hkv, int Hq, 
 
 namespace {
 
-constexpr int kWarps = 4;
+constexpr int kWarps = 6;
 constexpr int kStages = 3;
 constexpr int kStageBytes = 3072;            // one key-meta group (512 B) followed by the unit (<= 2560 B), as in the block
 constexpr int kKeyMetaOff = 0;
 constexpr int kUnitOff = 512;
 constexpr int kPrepBytes = 2432;             // kprep 576 | zprep 576 | svp 256 | zvp 1024
-constexpr int kSharedTail = 128 + 2048 + 2048 + 128 + 128;
+constexpr int kBarBytes = 256;                 // mbarriers: a ring per warp and one more per warp for the residual window
+constexpr int kSharedTail = kBarBytes + 2048 + 2048 + 2 * kWarps * 32;
 constexpr int kSmemBytes = kWarps * (kStages * kStageBytes + kPrepBytes) + kSharedTail;
-constexpr int kCtasPerSm = 3;
-constexpr int kCtasPerSmDense = 3;           // with a 4-bit base two key planes are in flight: more registers per thread, fewer CTAs
-static_assert((kWarps * kStages + kWarps) * 8 <= 128, "the mbarrier area at the start of the shared tail holds 16 barriers");
+constexpr int kCtasPerSm = 2;
+constexpr int kCtasPerSmDense = 2;           // with a 4-bit base two key planes are in flight: more registers per thread, fewer CTAs
+static_assert((kWarps * kStages + kWarps) * 8 <= kBarBytes, "the mbarrier area at the start of the shared tail is too small");
 constexpr int kResidualWeight = 2;           // a 32-token unit of the residual window counts as this many packed units in the split
 constexpr uint32_t kSpinLimit = 1u << 22;    // bounded wait on a staged copy
 constexpr int kMergeStride = 132;            // floats per head row of a warp's output in the merge (bank-conflict-free stores)
@@ -150,10 +151,10 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
   uint32_t* zvp = reinterpret_cast<uint32_t*>(prep + 1408);     // [2 ks][8 rows][4 t]{ch0, 0, ch1, 0} half2: rows < VG z_v, row 4 ones
   unsigned char* tail = smem + kWarps * (kStages * kStageBytes + kPrepBytes);
   uint64_t* bars = reinterpret_cast<uint64_t*>(tail);           // [kWarps][kStages]
-  uint16_t* qb16 = reinterpret_cast<uint16_t*>(tail + 128);     // [8][128] q, bf16 bits (0 for heads >= g)
-  __half* qf16 = reinterpret_cast<__half*>(tail + 128 + 2048);  // [8][128] q, fp16
-  float* mS = reinterpret_cast<float*>(tail + 128 + 4096);      // [4][8]
-  float* lS = mS + 32;                                          // [4][8]
+  uint16_t* qb16 = reinterpret_cast<uint16_t*>(tail + kBarBytes);           // [8][128] q, bf16 bits (0 for heads >= g)
+  __half* qf16 = reinterpret_cast<__half*>(tail + kBarBytes + 2048);        // [8][128] q, fp16
+  float* mS = reinterpret_cast<float*>(tail + kBarBytes + 4096);            // [kWarps][8]
+  float* lS = mS + kWarps * 8;                                              // [kWarps][8]
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < kWarps * kStages + kWarps; ++i) mbar_init(smem_u32(&bars[i]), 1);   // rings + one per warp for the residual window
@@ -258,13 +259,15 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
       const int b = s / lv.Hkv, hk = s % lv.Hkv;
       __syncthreads();
       {
-        // one 16-byte load per thread: head h, channels 8c .. 8c+7 (heads >= g are zero rows)
+        // one 16-byte load per thread (the first 128): head h, channels 8c .. 8c+7 (heads >= g are zero rows)
         const int h = threadIdx.x >> 4, c = threadIdx.x & 15;
-        uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (h < g) v = *reinterpret_cast<const uint4*>(q + ((size_t)b * lv.Hq + hk * g + h) * kD + 8 * c);
-        *reinterpret_cast<uint4*>(&qb16[h * kD + 8 * c]) = v;
-        *reinterpret_cast<uint4*>(&qf16[h * kD + 8 * c]) =
-            make_uint4(bf16x2_to_f16x2(v.x), bf16x2_to_f16x2(v.y), bf16x2_to_f16x2(v.z), bf16x2_to_f16x2(v.w));
+        if (h < 8) {
+          uint4 v = make_uint4(0u, 0u, 0u, 0u);
+          if (h < g) v = *reinterpret_cast<const uint4*>(q + ((size_t)b * lv.Hq + hk * g + h) * kD + 8 * c);
+          *reinterpret_cast<uint4*>(&qb16[h * kD + 8 * c]) = v;
+          *reinterpret_cast<uint4*>(&qf16[h * kD + 8 * c]) =
+              make_uint4(bf16x2_to_f16x2(v.x), bf16x2_to_f16x2(v.y), bf16x2_to_f16x2(v.z), bf16x2_to_f16x2(v.w));
+        }
       }
       __syncthreads();
     }
@@ -790,7 +793,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
       }
     }
     __syncthreads();
-    {
+    if (threadIdx.x < 128) {
       const int h = threadIdx.x >> 4, c0 = threadIdx.x & 15;
       float M = -INFINITY, L = 0.f, f[kWarps];
 #pragma unroll

@@ -166,6 +166,11 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
     const int idx = lane + 32 * i, row = (idx >> 4) & 7;
     zvp[idx] = (row == 4 && (idx & 1) == 0) ? 0x3C003C00u : 0u;
   }
+  // Programmatic dependent launch: the grid may have been started while the kernel before it in the stream was still
+  // running.  Nothing above touches global memory; everything below does, so wait here for that kernel's results,
+  // and let the kernel after this one be started early in the same way.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   __syncthreads();
 
   // per-lane constants of the per-unit preparation steps
@@ -827,14 +832,29 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
   }
 }
 
+template <int G, int kU4>
+cudaError_t launch_one(const LayerView& lv, const __nv_bfloat16* qb, float sl, float* ws, int grid, cudaStream_t stream) {
+  // launched with programmatic stream serialization: the kernel itself waits for its predecessor (griddepcontrol.wait)
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(kWarps * 32);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, attention_mma_kernel<G, kU4>, lv, qb, sl, ws, 0x44004400u);
+}
+
 template <int G>
 cudaError_t launch_g(const LayerView& lv, const void* q, float scale, float* ws, int grid, cudaStream_t stream) {
   const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q);
   const float sl = scale * 1.4426950408889634f;
-  if (lv.dense_hi) attention_mma_kernel<G, 2><<<grid, kWarps * 32, kSmemBytes, stream>>>(lv, qb, sl, ws, 0x44004400u);
-  else if (lv.tau_u4 < lv.tau_bf16) attention_mma_kernel<G, 1><<<grid, kWarps * 32, kSmemBytes, stream>>>(lv, qb, sl, ws, 0x44004400u);
-  else attention_mma_kernel<G, 0><<<grid, kWarps * 32, kSmemBytes, stream>>>(lv, qb, sl, ws, 0x44004400u);
-  return cudaGetLastError();
+  if (lv.dense_hi) return launch_one<G, 2>(lv, qb, sl, ws, grid, stream);
+  if (lv.tau_u4 < lv.tau_bf16) return launch_one<G, 1>(lv, qb, sl, ws, grid, stream);
+  return launch_one<G, 0>(lv, qb, sl, ws, grid, stream);
 }
 
 }  // namespace

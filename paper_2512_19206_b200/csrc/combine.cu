@@ -9,6 +9,9 @@ namespace mixkvq {
 __global__ void __launch_bounds__(128)
 combine_kernel(const float* __restrict__ ws, float* __restrict__ out, int g, int Hkv, int Hq, int mode, int n,
                long long units_per_stream, int S) {
+  // started early (programmatic dependent launch): wait for the kernel that wrote the partials
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int s = blockIdx.x / g, h = blockIdx.x % g, c = threadIdx.x;
   int first, count;
   if (mode == 0) {
@@ -39,8 +42,16 @@ combine_kernel(const float* __restrict__ ws, float* __restrict__ out, int g, int
 
 cudaError_t launch_combine(const float* ws, float* out, int g, int Hkv, int Hq, int mode, int n,
                            long long units_per_stream, int S, cudaStream_t stream) {
-  combine_kernel<<<S * g, 128, 0, stream>>>(ws, out, g, Hkv, Hq, mode, n, units_per_stream, S);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(S * g));
+  cfg.blockDim = dim3(128);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, combine_kernel, ws, out, g, Hkv, Hq, mode, n, units_per_stream, S);
 }
 
 // Two sets of partials per stream (packed blocks, residual window), each written by a grid that split its

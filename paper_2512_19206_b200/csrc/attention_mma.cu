@@ -37,7 +37,7 @@ constexpr int kSmemBytes = kWarps * (kStages * kStageBytes + kPrepBytes) + kShar
 constexpr int kCtasPerSm = 2;
 constexpr int kCtasPerSmDense = 2;           // with a 4-bit base two key planes are in flight: more registers per thread, fewer CTAs
 static_assert((kWarps * kStages + kWarps) * 8 <= kBarBytes, "the mbarrier area at the start of the shared tail is too small");
-constexpr int kResidualWeight = 2;           // a 32-token unit of the residual window counts as this many packed units in the split
+constexpr int kResidualWeight = 3;           // a 32-token unit of the residual window counts as this many packed units in the split
 constexpr uint32_t kSpinLimit = 1u << 22;    // bounded wait on a staged copy
 constexpr int kMergeStride = 132;            // floats per head row of a warp's output in the merge (bank-conflict-free stores)
 constexpr float kMaxSlack = 3.0f;            // a packed unit's probabilities are at most 2^kMaxSlack (log2 domain)
@@ -166,11 +166,6 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
     const int idx = lane + 32 * i, row = (idx >> 4) & 7;
     zvp[idx] = (row == 4 && (idx & 1) == 0) ? 0x3C003C00u : 0u;
   }
-  // Programmatic dependent launch: the grid may have been started while the kernel before it in the stream was still
-  // running.  Nothing above touches global memory; everything below does, so wait here for that kernel's results,
-  // and let the kernel after this one be started early in the same way.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   __syncthreads();
 
   // per-lane constants of the per-unit preparation steps
@@ -192,6 +187,12 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
   const long long cb = split_begin(total, gridDim.x, blockIdx.x), ce = split_begin(total, gridDim.x, blockIdx.x + 1);
 
   uint32_t res_phase = 0;         // phase of this warp's residual-staging barrier
+  // Programmatic dependent launch: the grid may have been started while the kernel before it in the stream was still
+  // running.  Nothing above touches global memory; everything below does, so wait here for that kernel's results,
+  // and let the kernel after this one be started early in the same way.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
   uint32_t ring_stage = 0;        // ring stage of the next packed unit this warp consumes
   uint32_t ring_parity = 0;       // phase parity of that stage's barrier
   bool gave_up = false;
@@ -201,7 +202,37 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
     const int ub = (int)(seg - (long long)s * Us);
     const int ue = (int)min((long long)Us, ce - (long long)s * Us);
     seg += ue - ub;
-    const int wb = ub + (int)split_begin(ue - ub, kWarps, warp), we = ub + (int)split_begin(ue - ub, kWarps, warp + 1);
+    // ---- the query of this stream is requested before anything else: the burst of staged copies below would delay it
+    uint4 q_regs = make_uint4(0u, 0u, 0u, 0u);      // thread (h, c) of the first 128: head h, channels 8c .. 8c+7
+    {
+      const int b = s / lv.Hkv, hk = s % lv.Hkv, h = threadIdx.x >> 4, c = threadIdx.x & 15;
+      if (h < g) q_regs = *reinterpret_cast<const uint4*>(q + ((size_t)b * lv.Hq + hk * g + h) * kD + 8 * c);
+    }
+    // ---- this warp's share of the segment.  The residual units of the segment go to different warps (unit i to warp
+    // kWarps - 1 - i % kWarps), so that their copies and their arithmetic run side by side; the packed units are split
+    // in order so that every warp carries about the same weight.
+    const int pk_b = min(ub, packed_units), pk_e = min(ue, packed_units);
+    const int res_b = (max(ub, packed_units) - packed_units + kResidualWeight - 1) / kResidualWeight;
+    const int res_e = ue > packed_units ? (ue - packed_units + kResidualWeight - 1) / kResidualWeight : res_b;
+    const int n_res = res_e - res_b;
+    int wb = pk_b, we = pk_b;
+    {
+      const int weight = (pk_e - pk_b) + kResidualWeight * n_res;
+      int remaining = pk_e - pk_b;
+#pragma unroll
+      for (int w = 0; w < kWarps; ++w) {
+        const int share = weight * (w + 1) / kWarps - weight * w / kWarps;       // weight < 2^24: 32-bit arithmetic
+        const int first_i = kWarps - 1 - w;                                   // residual units first_i, first_i + kWarps, ...
+        const int res_w = n_res > first_i ? (n_res - first_i + kWarps - 1) / kWarps : 0;
+        int p = min(remaining, max(0, share - kResidualWeight * res_w));
+        if (w == kWarps - 1) p = remaining;
+        if (w == warp) {
+          wb = pk_e - remaining;
+          we = wb + p;
+        }
+        remaining -= p;
+      }
+    }
 
     const char* base = lv.base + (size_t)s * lv.base_stride;
     const char* extras = lv.extras + (size_t)s * lv.extras_stride;
@@ -210,7 +241,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
     // ---- the first copies of this segment go out before anything else: they do not depend on the query.
     // The packed units of a stream are one uniform sequence (a group's scales, then its units), whatever the block size,
     // so the copy source only ever moves forward: `isrc` is the next unit to stage, `ig` its index inside its key group.
-    const int n_pack = max(0, min(we, packed_units) - wb);
+    const int n_pack = we - wb;
     int issued = 0;
     const char* isrc = base + (size_t)wb * kUnitBytes + 512u * (size_t)(wb / UPG + 1);
     int ig = wb & (UPG - 1);
@@ -261,14 +292,12 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
 
     // ---- query of this stream: bf16 and fp16 tables for the gathered paths
     {
-      const int b = s / lv.Hkv, hk = s % lv.Hkv;
       __syncthreads();
       {
-        // one 16-byte load per thread (the first 128): head h, channels 8c .. 8c+7 (heads >= g are zero rows)
+        // heads >= g are zero rows
         const int h = threadIdx.x >> 4, c = threadIdx.x & 15;
         if (h < 8) {
-          uint4 v = make_uint4(0u, 0u, 0u, 0u);
-          if (h < g) v = *reinterpret_cast<const uint4*>(q + ((size_t)b * lv.Hq + hk * g + h) * kD + 8 * c);
+          const uint4 v = q_regs;
           *reinterpret_cast<uint4*>(&qb16[h * kD + 8 * c]) = v;
           *reinterpret_cast<uint4*>(&qf16[h * kD + 8 * c]) =
               make_uint4(bf16x2_to_f16x2(v.x), bf16x2_to_f16x2(v.y), bf16x2_to_f16x2(v.z), bf16x2_to_f16x2(v.w));
@@ -619,9 +648,8 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
     // ---- residual (unquantized) tokens of this warp's range: 32 token rows of 256 B staged through the (now idle)
     // ring with ONE bulk copy, first the keys, then the values over them (small bulk copies are slow: a copy per row
     // cost tens of microseconds).  Value tiles are transposed on the way to registers with ldmatrix.trans.
-    for (int xv = max(wb, packed_units); xv < we && !gave_up; ++xv) {
-      if ((xv - packed_units) % kResidualWeight != 0) continue;       // the warp owning a unit's first position runs it
-      const int x = packed_units + (xv - packed_units) / kResidualWeight;
+    for (int ri = kWarps - 1 - warp; ri < n_res && !gave_up; ri += kWarps) {
+      const int x = packed_units + res_b + ri;
       const uint32_t rbar = smem_u32(&bars[kWarps * kStages + warp]);
       const uint16_t* resk = reinterpret_cast<const uint16_t*>(lv.resk + (size_t)s * lv.resk_stride);
       const uint16_t* resv = reinterpret_cast<const uint16_t*>(lv.resv + (size_t)s * lv.resv_stride);

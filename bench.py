@@ -346,7 +346,12 @@ def run_gpu(args, w):
     n16, n4 = tier_mix(cache, w)
     tokens_packed = d0.n_blocks * w.residual_len
     units = (tokens_packed // 32 + (d0.residual_tokens + 31) // 32) * w.batch * w.n_kv_heads
-    n_part = min(148 * 3, units) + w.batch * w.n_kv_heads
+    # partials written per launch = CTAs of the split kernel: two per SM, a multiple of the stream count when there are
+    # fewer streams than CTA slots (the library's grid rule), each CTA one partial per stream it touches
+    streams = w.batch * w.n_kv_heads
+    n_sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    n_part = min(2 * n_sms, units)
+    n_part = n_part // streams * streams if n_part > streams else n_part + streams
     alg = algorithmic_bytes_per_layer(w, n16, n4, d0.residual_tokens, tokens_packed, n_part)
     peak, peak_src = measured_peaks()
     achieved = alg / (kern_ms * 1e-3) / 1e9

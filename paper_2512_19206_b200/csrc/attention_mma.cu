@@ -30,7 +30,7 @@ constexpr int kStages = 3;
 constexpr int kStageBytes = 3072;            // one key-meta group (512 B) followed by the unit (<= 2560 B), as in the block
 constexpr int kKeyMetaOff = 0;
 constexpr int kUnitOff = 512;
-constexpr int kPrepBytes = 2432;             // kprep 576 | zprep 576 | svp 256 | zvp 1024
+constexpr int kPrepBytes = 2560;             // kprep 576 | zprep 576 | svp 320 | zvp 1088
 constexpr int kBarBytes = 256;                 // mbarriers: a ring per warp and one more per warp for the residual window
 constexpr int kSharedTail = kBarBytes + 2048 + 2048 + 2 * kWarps * 32;
 constexpr int kSmemBytes = kWarps * (kStages * kStageBytes + kPrepBytes) + kSharedTail;
@@ -147,8 +147,9 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
   uint32_t* kprep = reinterpret_cast<uint32_t*>(prep);          // [8 kt: scale_word][4 t]{s ch0, s ch1} half2 (first 288 of 576 bytes)
   // the zero-point tiles are stored as whole A fragments (four registers), so one 16-byte load feeds the MMA
   uint32_t* zprep = reinterpret_cast<uint32_t*>(prep + 576);    // [8 kt][4 t]{z ch0, z ch0, z ch1, z ch1} half2 z / mult
-  uint32_t* svp = reinterpret_cast<uint32_t*>(prep + 1152);     // [4 t][4 vg][2 ks][2 ch] half2 s_v'
-  uint32_t* zvp = reinterpret_cast<uint32_t*>(prep + 1408);     // [2 ks][8 rows][4 t]{ch0, 0, ch1, 0} half2: rows < VG z_v, row 4 ones
+  // (20 words per t and 144 per ks instead of 16 and 128: the preparation's 16-bit stores then hit distinct banks)
+  uint32_t* svp = reinterpret_cast<uint32_t*>(prep + 1152);     // [4 t: 20 words][4 vg][2 ks][2 ch] half2 s_v'
+  uint32_t* zvp = reinterpret_cast<uint32_t*>(prep + 1472);     // [2 ks][8 rows][4 t]{ch0, 0, ch1, 0} half2: rows < VG z_v, row 4 ones
   unsigned char* tail = smem + kWarps * (kStages * kStageBytes + kPrepBytes);
   uint64_t* bars = reinterpret_cast<uint64_t*>(tail);           // [kWarps][kStages]
   uint16_t* qb16 = reinterpret_cast<uint16_t*>(tail + kBarBytes);           // [8][128] q, bf16 bits (0 for heads >= g)
@@ -162,9 +163,9 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
   }
   // constant rows of the zero-point / denominator tile: row 4 is all ones, the other rows >= VG stay zero
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int idx = lane + 32 * i, row = (idx >> 4) & 7;
-    zvp[idx] = (row == 4 && (idx & 1) == 0) ? 0x3C003C00u : 0u;
+  for (int i = 0; i < 9; ++i) {
+    const int idx = lane + 32 * i, rem = idx % 144, row = rem >> 4;      // [2 ks: 144 words][8 rows][4 t][4]
+    if (idx < 272) zvp[idx] = (row == 4 && (idx & 1) == 0) ? 0x3C003C00u : 0u;
   }
   __syncthreads();
 
@@ -175,8 +176,8 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
   const int pk_kp = scale_word(lane >> 2) + 4 * (lane & 1) + ((lane & 3) >> 1);            // kprep word of the first pair
   // values: the lane converts the scales and zero-points of token `lane`
   const float pv_up = __uint_as_float((131u - 2u * (uint32_t)(lane >> 3)) << 23);          // 2^(4 - 2 * (2 ks + ch))
-  const int pv_sv = ((((lane & 7) >> 1) * 16 + (lane >> 3)) * 2) + (lane & 1);             // svp half index of group 0
-  const int pv_zv = ((((lane >> 4) * 8 * 4 + ((lane & 7) >> 1)) * 4 + 2 * ((lane >> 3) & 1)) * 2) + (lane & 1);   // zvp half index of group 0
+  const int pv_sv = ((((lane & 7) >> 1) * 20 + (lane >> 3)) * 2) + (lane & 1);             // svp half index of group 0
+  const int pv_zv = (((lane >> 4) * 144 + ((lane & 7) >> 1) * 4 + 2 * ((lane >> 3) & 1)) * 2) + (lane & 1);   // zvp half index of group 0
   constexpr uint32_t kUnitBytes = 2048u + 128u * (kD / G);   // codes of 32 tokens: keys 1024, values 1024, value scales
   constexpr int UPG = G / 32;                                 // units per key group
 
@@ -590,7 +591,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
       // ---- zero-point and denominator tile: rows 0..VG-1 = z_v of the group, row 4 = ones, the rest zero
 #pragma unroll
       for (int ks = 0; ks < 2; ++ks) {
-        const uint4 zz = *reinterpret_cast<const uint4*>(&zvp[((ks * 8 + r) * 4 + t) * 4]);
+        const uint4 zz = *reinterpret_cast<const uint4*>(&zvp[ks * 144 + (r * 4 + t) * 4]);
         mma_f16(Zc, zz.x, zz.y, zz.z, zz.w, Pt[ks][0], Pt[ks][1]);
       }
       // ---- P.V: codes as fp16 subnormals, scales folded into P
@@ -600,7 +601,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
         const uint32_t vw[8] = {vw0.x, vw0.y, vw0.z, vw0.w, vw1.x, vw1.y, vw1.z, vw1.w};
 #pragma unroll
         for (int vg = 0; vg < VG; ++vg) {
-          const uint4 sv = *reinterpret_cast<const uint4*>(&svp[(t * 4 + vg) * 4]);
+          const uint4 sv = *reinterpret_cast<const uint4*>(&svp[t * 20 + vg * 4]);
           const uint32_t Bp[2][2] = {{hmul2_u(Pt[0][0], sv.x), hmul2_u(Pt[0][1], sv.y)},
                                      {hmul2_u(Pt[1][0], sv.z), hmul2_u(Pt[1][1], sv.w)}};
 #pragma unroll

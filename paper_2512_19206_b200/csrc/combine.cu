@@ -9,9 +9,6 @@ namespace mixkvq {
 __global__ void __launch_bounds__(128)
 combine_kernel(const float* __restrict__ ws, float* __restrict__ out, int g, int Hkv, int Hq, int mode, int n,
                long long units_per_stream, int S) {
-  // started early (programmatic dependent launch): wait for the kernel that wrote the partials
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int s = blockIdx.x / g, h = blockIdx.x % g, c = threadIdx.x;
   int first, count;
   if (mode == 0) {
@@ -26,16 +23,36 @@ combine_kernel(const float* __restrict__ ws, float* __restrict__ out, int g, int
   }
   const int b = s / Hkv, hk = s % Hkv;
   const float* base = ws + (size_t)first * kPartialFloats + h * 130;
-  float M = -INFINITY;
-  for (int i = 0; i < count; ++i) M = fmaxf(M, base[(size_t)i * kPartialFloats]);
-  float l = 0.f, o = 0.f;
-#pragma unroll 4
-  for (int i = 0; i < count; ++i) {
-    const float* p = base + (size_t)i * kPartialFloats;
-    const float m = p[0];
-    const float f = (m == -INFINITY) ? 0.f : exp2f(m - M);
-    l += f * p[1];
-    o += f * p[2 + c];
+  // started early (programmatic dependent launch): wait here for the kernel that wrote the partials
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // one pass with a running maximum; the loads of a chunk of partials are independent of one another, so a stream with
+  // up to kChunk partials costs one round trip to memory
+  constexpr int kChunk = 12;
+  float M = -INFINITY, l = 0.f, o = 0.f;
+  for (int i0 = 0; i0 < count; i0 += kChunk) {
+    float m[kChunk], ll[kChunk], oo[kChunk];
+#pragma unroll
+    for (int j = 0; j < kChunk; ++j) {
+      const bool in = i0 + j < count;
+      const float* p = base + (size_t)(in ? i0 + j : i0) * kPartialFloats;
+      m[j] = in ? p[0] : -INFINITY;
+      ll[j] = p[1];
+      oo[j] = p[2 + c];
+    }
+    float Mn = M;
+#pragma unroll
+    for (int j = 0; j < kChunk; ++j) Mn = fmaxf(Mn, m[j]);
+    const float f0 = (M == -INFINITY) ? 0.f : exp2f(M - Mn);
+    l *= f0;
+    o *= f0;
+#pragma unroll
+    for (int j = 0; j < kChunk; ++j) {
+      const float f = (m[j] == -INFINITY) ? 0.f : exp2f(m[j] - Mn);
+      l += f * ll[j];
+      o += f * oo[j];
+    }
+    M = Mn;
   }
   out[((size_t)b * Hq + hk * g + h) * kD + c] = o / l;
 }

@@ -370,9 +370,11 @@ def run_gpu(args, w):
         "tier_mix_mean": {"n16": n16, "n4": n4, "n2": 128 - n16 - n4},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal_8TBs": achieved / 8000.0,
-                     "traffic": measured_traffic(*(("attention_tc_kernel", "attention_tc.cu") if args.layout == 1 else
-                                                   ("attention_mma_kernel", "attention_mma.cu")), w.group_size,
-                                                 tokens_packed, w.batch * w.n_kv_heads),
+                     # the committed counters were taken on the two-tier mix (no UINT4 tier): other mixes have none
+                     "traffic": None if w.tau_u4 < w.tau_bf16 else measured_traffic(
+                         *(("attention_tc_kernel", "attention_tc.cu") if args.layout == 1 else
+                           ("attention_mma_kernel", "attention_mma.cu")), w.group_size, tokens_packed,
+                         w.batch * w.n_kv_heads),
                      "peak_source": peak_src,
                      "kernel": "attention_tc_kernel" if args.layout == 1 else "attention_mma_kernel", "kernel_us": kern_ms * 1e3, "algorithmic_bytes": alg},
         "e2e": {"value": e2e_us, "unit": "us/step", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

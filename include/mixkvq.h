@@ -130,7 +130,11 @@ int mixkvq_quantize_append(mixkvq_cache* cache, int layer, const void* k_dev, co
 /* (3) Eq. 1 for one decode step of `layer` over [packed blocks, residual window], keys and values
  * dequantized on the fly (Eq. 3).
  *   q_dev [B, Hq, 128] bf16  ->  out_dev [B, Hq, 128] float
- *   workspace_dev: at least attn_workspace_bytes (mixkvq_cache_bytes); contents are scratch */
+ *   workspace_dev: at least attn_workspace_bytes (mixkvq_cache_bytes); contents are scratch
+ * Numeric range: the tensor-core operands are fp16, so |q| must stay below 4094, a stored key scale below 2^11 and a
+ * stored value scale below 2^9 (value ranges up to about 1500); beyond that the output overflows to inf or NaN.
+ * The kernels are launched with programmatic stream serialization and wait on the device for all earlier work of
+ * the stream before they touch global memory, so stream order holds as for any other launch. */
 int mixkvq_decode_attention(mixkvq_cache* cache, int layer, const void* q_dev, float* out_dev, float softmax_scale,
                             void* workspace_dev, size_t workspace_bytes, void* stream);
 

@@ -176,6 +176,30 @@ def test_attention_matches_oracle(binding, kind, layout, name, tokens, preset):
 
 
 @pytest.mark.parametrize("kind", [0, 1])
+def test_attention_large_magnitudes(binding, kind):
+    # values 64 times larger (stored value scales around 170: inside the documented fp16 operand range of the default
+    # kernel, s_v * 2^7 < 65504) and queries 4 times larger (logits of several tens, sharply peaked softmax rows, so the
+    # reference maximum of the online softmax jumps by more than its slack); the error bound scales with the values
+    # (the salience is linear in |q|: the threshold moves with it, so the tier mix stays that of the preset)
+    w = small("qwen7b", batch=2, tokens=9 * 128 + 77, **{**W.P24, "tau_bf16": 4.0 * W.P24["tau_bf16"]})
+    k, v, q = W.tokens(w, 0, 0, w.tokens)
+    v = (v.float() * 64.0).to(torch.bfloat16)
+    q = (q.float() * 4.0).to(torch.bfloat16)
+    cache = U.make_cache(binding, w)
+    cache.quantize_append(0, k.cuda(), v.cuda(), q.cuda())
+    cache.set_attention_kernel(kind)
+    orc = U.oracle_streams(w, 0, k, v, q)
+    U.compare_regions(cache, 0, w, orc)
+    for step in range(2):
+        qd = (W.decode_query(w, 0, step).float() * 4.0).to(torch.bfloat16)
+        out = cache.decode_attention(0, qd.cuda(), W.softmax_scale())
+        assert torch.isfinite(out).all()
+        err = U.max_abs_err(w, out, U.oracle_attention(w, orc, qd))
+        assert err <= 64.0 * ATTN_TOL, (err, step)
+    assert cache.status() == 0
+
+
+@pytest.mark.parametrize("kind", [0, 1])
 @pytest.mark.parametrize("R,G,layout", [(128, 128, 0), (64, 32, 0), (256, 64, 0), (32, 32, 0), (96, 32, 0), (128, 128, 1),
                                         (128, 64, 1)])
 def test_attention_other_geometries(binding, kind, R, G, layout):

@@ -97,7 +97,7 @@ def run_reference(args, w):
         "impl": "reference", "metric": METRIC, "value": us, "unit": "us/step", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": workload_config(w),
+        "config": workload_config(w, args.importance_mode),
         "cpu_baseline": {"value": us, "unit": "us/step", "cores": oracle_threads(), "kind": "oracle", "sample": desc},
         "e2e": {"value": us, "unit": "us/step", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "tokens_per_s": w.batch / (us * 1e-6),
@@ -106,10 +106,11 @@ def run_reference(args, w):
 
 
 # ------------------------------------------------------------------------------------------------- GPU leg
-def workload_config(w):
+def workload_config(w, importance_mode=0):
     return {"workload": w.name, "n_layers": w.n_layers, "batch": w.batch, "n_q_heads": w.n_q_heads,
             "n_kv_heads": w.n_kv_heads, "head_dim": 128, "context_tokens": w.tokens, "residual_len": w.residual_len,
             "group_size": w.group_size, "tau_bf16": w.tau_bf16, "tau_u4": w.tau_u4, "score_bits": w.score_bits,
+            "importance_mode": importance_mode,
             "l2": "inputs larger than L2: every step streams all layers' packed cache once"}
 
 
@@ -232,6 +233,7 @@ def run_gpu(args, w):
     cfg = binding.make_config(w.n_layers, w.batch, w.n_q_heads, w.n_kv_heads, w.tokens + n_steps + 2 * w.residual_len,
                               residual_len=w.residual_len, group_size=w.group_size, tau_bf16=w.tau_bf16,
                               tau_u4=w.tau_u4, score_bits=w.score_bits, block_layout=args.layout,
+                              importance_mode=args.importance_mode,
                               extras_budget_bytes=((w.tokens + n_steps) // w.residual_len + 3) * 8192 if w.score_bits == 4 else 0)
     cache = binding.Cache(cfg, device=dev)
     prefill_ms = prefill(cache, w, dev)
@@ -360,7 +362,7 @@ def run_gpu(args, w):
         "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
         "dtype": "f16", "data": "synthetic",
         "arithmetic": "2/4-bit codes and bf16 metadata expanded to fp16 tensor-core operands, fp32 accumulate and softmax",
-        "config": workload_config(w),
+        "config": workload_config(w, args.importance_mode),
         "tokens_per_s": job_tokens_per_s(w.batch, world, us),
         "attention_graph_us_per_step": graph_us,
         "prefill_quantize": {"ms": prefill_ms, "tokens_per_s": w.n_layers * w.batch * w.tokens / (prefill_ms * 1e-3),
@@ -400,6 +402,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", default="qwen7b", choices=sorted(W.CONFIGS))
     ap.add_argument("--group-size", type=int, default=None)
+    ap.add_argument("--residual-len", type=int, default=None, help="R: residual window / block length (32 .. 256)")
+    ap.add_argument("--importance-mode", type=int, default=0, choices=[0, 1, 2],
+                    help="0: window importance (default), 1: cumulative, 2: error-only salience")
     ap.add_argument("--tokens", type=int, default=None)
     ap.add_argument("--layers", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -413,6 +418,8 @@ def main():
     over = {}
     if args.group_size:
         over["group_size"] = args.group_size
+    if args.residual_len:
+        over["residual_len"] = args.residual_len
     if args.tokens:
         over["tokens"] = args.tokens
     if args.layers:

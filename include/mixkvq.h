@@ -121,8 +121,8 @@ int mixkvq_select_channels_raw(const void* q_dev, const void* k_dev, int batch, 
  * for each token, if the residual window already holds R tokens it is first scored, quantized (keys per
  * channel at the tier's bit-width, values per token at 2 bits, groups of G, Eq. 2) and packed; then the
  * token is stored in the window and |q| is added to the importance accumulator.
- * With the window importance mode, complete windows of a long append are quantized straight from the tensors (the
- * prefill path); the result is byte for byte that of n_tokens single appends.
+ * Complete windows of a long append are quantized straight from the tensors (the prefill path); the result is byte for
+ * byte that of n_tokens single appends.
  *   k_dev, v_dev [B, Hkv, n_tokens, 128] bf16;  q_dev [B, Hq, n_tokens, 128] bf16 */
 int mixkvq_quantize_append(mixkvq_cache* cache, int layer, const void* k_dev, const void* v_dev, const void* q_dev,
                            int n_tokens, void* stream);

@@ -232,13 +232,13 @@ int mixkvq_quantize_append(mixkvq_cache* cache, int layer, const void* k_dev, co
       cache->r[layer] = 0;
     }
     // prefill: complete windows go straight from the tensors to packed blocks; the last 1..R tokens stay in the
-    // residual window (the running accumulator is only needed in cumulative mode, which keeps the per-block path)
-    if (cache->cfg.importance_mode != 1 && cache->r[layer] == 0 && n_tokens - t > cache->R) {
+    // residual window
+    if (cache->r[layer] == 0 && n_tokens - t > cache->R) {
       int nb = (n_tokens - t - 1) / cache->R;
       if (nb > 32768) nb = 32768;                  // grid.y limit
       LayerView lv = view(cache, layer);
       if (launch_flush_bulk(lv, k_dev, v_dev, q_dev, n_tokens, t, nb, st) != cudaSuccess) return MIXKVQ_E_CUDA;
-      cache->launches += 3;
+      cache->launches += cache->cfg.importance_mode == 1 ? 4 : 3;
       cache->n_blocks[layer] += nb;
       t += nb * cache->R;
       continue;

@@ -49,6 +49,58 @@ __global__ void bulk_prefix_kernel(LayerView lv, int nb) {
   *used = off16;
 }
 
+// Cumulative importance (Appendix D.2) in a bulk append: the running |q| sums continue across the windows, and the order of
+// the sum is part of its definition, so one CTA per stream walks the nb windows in token order (queries staged 16 tokens at
+// a time, thread d adds channel d).  It leaves the sums and the count as they stand at the end of each window in bytes
+// 128.. of that window's (still unwritten) block, where the first bulk pass reads them, and the final values in the state.
+constexpr int kSnapshotOff = 128, kSnapshotCntOff = 128 + 1024;
+
+__global__ void __launch_bounds__(256)
+bulk_importance_kernel(LayerView lv, BulkSrc src, int nb) {
+  __shared__ __align__(16) uint16_t qS[16 * 8 * kD];      // [token][head][128] bf16 bits
+  const int s = blockIdx.x, tid = threadIdx.x, g = lv.g, R = lv.R;
+  const int b = s / lv.Hkv, hk = s % lv.Hkv;
+  char* state = lv.state + (size_t)s * lv.state_stride;
+  double a = tid < kD ? reinterpret_cast<const double*>(state)[tid] : 0.0;
+  uint32_t cnt = *reinterpret_cast<const uint32_t*>(state + 1024);
+  const uint16_t* qw = src.q + (((size_t)b * lv.Hq + hk * g) * src.n_tokens + src.t0) * kD;
+  const size_t head_stride = (size_t)src.n_tokens * kD;
+  // the queries of the next 16 tokens are requested (into registers) before the sums of the current 16 are taken
+  const int n_rounds = nb * (R / 16), per_round = 16 * g * 16;       // 16-byte pieces per round (<= 2048)
+  uint4 pre[8];
+  auto request = [&](int round) {
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const int i = tid + 256 * k;
+      if (i < per_round) {
+        const int row = i >> 4, c16 = i & 15, jj = row / g, h = row - jj * g;
+        pre[k] = *reinterpret_cast<const uint4*>(qw + (size_t)(round * 16 + jj) * kD + h * head_stride + 8 * c16);
+      }
+    }
+  };
+  request(0);
+  for (int w = 0; w < nb; ++w) {
+    for (int j0 = 0; j0 < R; j0 += 16) {
+      const int round = w * (R / 16) + j0 / 16;
+#pragma unroll
+      for (int k = 0; k < 8; ++k)
+        if (tid + 256 * k < per_round) reinterpret_cast<uint4*>(qS)[tid + 256 * k] = pre[k];
+      __syncthreads();
+      if (round + 1 < n_rounds) request(round + 1);
+      if (tid < kD)
+        for (int row = 0; row < 16 * g; ++row)
+          a = __dadd_rn(a, (double)fabsf(bf16_bits_to_float(qS[row * kD + tid])));
+      __syncthreads();
+    }
+    cnt += (uint32_t)(R * g);
+    char* blk = lv.base + (size_t)s * lv.base_stride + (size_t)(lv.n_blocks + w) * lv.base_bytes;
+    if (tid < kD) reinterpret_cast<double*>(blk + kSnapshotOff)[tid] = a;
+    if (tid == 0) *reinterpret_cast<uint32_t*>(blk + kSnapshotCntOff) = cnt;
+  }
+  if (tid < kD) reinterpret_cast<double*>(state)[tid] = a;
+  if (tid == 0) *reinterpret_cast<uint32_t*>(state + 1024) = cnt;
+}
+
 __global__ void __launch_bounds__(256)
 flush_kernel(LayerView lv, BulkSrc src) {
   extern __shared__ __align__(16) unsigned char smem[];
@@ -83,7 +135,12 @@ flush_kernel(LayerView lv, BulkSrc src) {
   // heads at a time (16-byte loads); thread d then adds |q| of channel d token-major and head-ascending, the order of
   // the running accumulator of the decode path.
   double bulk_acc = 0.0;
-  if (src.phase == 1) {
+  uint32_t bulk_cnt = (uint32_t)(R * lv.g);
+  if (src.phase == 1 && lv.importance_mode == 1) {
+    // cumulative importance: the sums at the end of this window were left in the block by bulk_importance_kernel
+    if (tid < kD) bulk_acc = reinterpret_cast<const double*>(blk + kSnapshotOff)[tid];
+    bulk_cnt = *reinterpret_cast<const uint32_t*>(blk + kSnapshotCntOff);
+  } else if (src.phase == 1) {
     const int b = s / lv.Hkv, hk = s % lv.Hkv;
     const uint16_t* qw = src.q + (((size_t)b * lv.Hq + hk * lv.g) * src.n_tokens + src.t0 + (size_t)blockIdx.y * R) * kD;
     const size_t head_stride = (size_t)src.n_tokens * kD;
@@ -118,7 +175,7 @@ flush_kernel(LayerView lv, BulkSrc src) {
       uint32_t cnt;
       if (bulk) {
         acc = bulk_acc;
-        cnt = (uint32_t)(R * lv.g);
+        cnt = bulk_cnt;
       } else {
         acc = reinterpret_cast<const double*>(state)[d];
         cnt = *reinterpret_cast<const uint32_t*>(state + 1024);
@@ -389,7 +446,7 @@ cudaError_t launch_flush(const LayerView& lv, cudaStream_t stream) {
 }
 
 // nb complete R-token windows starting at token t0 of the append's tensors go straight to packed blocks
-// (three launches).  Preconditions (checked by the caller): window importance mode, empty residual window.
+// (three launches, four with cumulative importance).  Precondition (checked by the caller): empty residual window.
 cudaError_t launch_flush_bulk(const LayerView& lv, const void* k, const void* v, const void* q, int n_tokens, int t0,
                               int nb, cudaStream_t stream) {
   cudaError_t e = cudaFuncSetAttribute(flush_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -398,6 +455,7 @@ cudaError_t launch_flush_bulk(const LayerView& lv, const void* k, const void* v,
   const int S = lv.B * lv.Hkv;
   BulkSrc src{static_cast<const uint16_t*>(k), static_cast<const uint16_t*>(v), static_cast<const uint16_t*>(q), n_tokens, t0, 1};
   const dim3 grid(S, nb);
+  if (lv.importance_mode == 1) bulk_importance_kernel<<<S, 256, 0, stream>>>(lv, src, nb);
   flush_kernel<<<grid, 256, flush_smem_bytes(lv.R), stream>>>(lv, src);
   bulk_prefix_kernel<<<(S + 127) / 128, 128, 0, stream>>>(lv, nb);
   src.phase = 2;

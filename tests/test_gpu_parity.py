@@ -113,18 +113,20 @@ def test_tiny_config_full_parity(binding, layout):
     assert cache.status() == 0
 
 
-def test_streamed_appends_equal_bulk(binding):
-    w = small(batch=1, tokens=128 + 70, **W.P27)
+@pytest.mark.parametrize("mode", [0, 1])
+def test_streamed_appends_equal_bulk(binding, mode):
+    # window importance and cumulative importance (whose bulk path carries the running sums across the windows)
+    w = small(batch=1, tokens=(128 + 70) if mode == 0 else (3 * 128 + 70), **W.P27)
     k, v, q = W.tokens(w, 0, 0, w.tokens)
     kc, vc, qc = k.cuda(), v.cuda(), q.cuda()
-    bulk = U.make_cache(binding, w)
+    bulk = U.make_cache(binding, w, importance_mode=mode)
     bulk.quantize_append(0, kc, vc, qc)
-    one = U.make_cache(binding, w)
+    one = U.make_cache(binding, w, importance_mode=mode)
     for t in range(w.tokens):
         one.quantize_append(0, kc[:, :, t:t + 1].contiguous(), vc[:, :, t:t + 1].contiguous(),
                             qc[:, :, t:t + 1].contiguous())
     # in two ragged pieces as well
-    two = U.make_cache(binding, w)
+    two = U.make_cache(binding, w, importance_mode=mode)
     two.quantize_append(0, kc[:, :, :93].contiguous(), vc[:, :, :93].contiguous(), qc[:, :, :93].contiguous())
     two.quantize_append(0, kc[:, :, 93:].contiguous(), vc[:, :, 93:].contiguous(), qc[:, :, 93:].contiguous())
     for s in range(w.n_kv_heads):
@@ -132,7 +134,7 @@ def test_streamed_appends_equal_bulk(binding):
         r = bulk.describe(0).residual_tokens
         for key in ("table", "base", "extras", "state", "resK", "resV"):
             assert a[key] == b[key] == c[key], key
-    U.compare_regions(bulk, 0, w, U.oracle_streams(w, 0, k, v, q))
+    U.compare_regions(bulk, 0, w, U.oracle_streams(w, 0, k, v, q, importance_mode=mode))
 
 
 @pytest.mark.parametrize("mode", [1, 2])

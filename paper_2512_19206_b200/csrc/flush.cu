@@ -111,6 +111,7 @@ flush_kernel(LayerView lv, BulkSrc src) {
   uint8_t* chan16S = tierS + 128;                         // [128]
   uint8_t* chan4S = chan16S + 128;                        // [128]
   int* misc = reinterpret_cast<int*>(chan4S + 128);       // n16, n4, extras offset (16-byte units)
+  float* wS = reinterpret_cast<float*>(chan4S + 128 + 16); // [2 halves][128]{max, min} of the window, later the tier counts
 
   const int s = blockIdx.x, tid = threadIdx.x;
   const bool bulk = src.phase != 0;
@@ -123,17 +124,22 @@ flush_kernel(LayerView lv, BulkSrc src) {
   const uint16_t* resv = reinterpret_cast<const uint16_t*>(lv.resv + (size_t)s * lv.resv_stride);
   uint2* table_entry = reinterpret_cast<uint2*>(lv.table + (size_t)s * lv.table_stride + (size_t)block_index * 8);
 
-  for (int i = tid; i < R * 16; i += 256) reinterpret_cast<uint4*>(kS)[i] = resk4[i];
-  __syncthreads();
+  // a window of R rows of 256 bytes: the loads of a thread go out together, then the stores
+  auto load_window = [&](const uint4* from) {
+    for (int i0 = 0; i0 < R * 16; i0 += 8 * 256) {
+      uint4 tmp[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k)
+        if (i0 + tid + 256 * k < R * 16) tmp[k] = from[i0 + tid + 256 * k];
+#pragma unroll
+      for (int k = 0; k < 8; ++k)
+        if (i0 + tid + 256 * k < R * 16) reinterpret_cast<uint4*>(kS)[i0 + tid + 256 * k] = tmp[k];
+    }
+  };
 
-  if (src.phase == 2) {
-    // the first pass left the 128 tiers in the first bytes of the block; fetch them before anything is written there
-    if (tid < kD) tierS[tid] = reinterpret_cast<const uint8_t*>(blk)[tid];
-    __syncthreads();
-  }
-  // ---- bulk, first pass: importance of this window from its own queries.  All threads stage a few tokens of the g
-  // heads at a time (16-byte loads); thread d then adds |q| of channel d token-major and head-ascending, the order of
-  // the running accumulator of the decode path.
+  // ---- bulk, first pass: importance of this window from its own queries, before the key window takes the shared
+  // memory.  All threads stage as many tokens of the g heads as the key and code areas hold (16-byte loads); thread d
+  // then adds |q| of channel d token-major and head-ascending, the order of the running accumulator of the decode path.
   double bulk_acc = 0.0;
   uint32_t bulk_cnt = (uint32_t)(R * lv.g);
   if (src.phase == 1 && lv.importance_mode == 1) {
@@ -144,75 +150,118 @@ flush_kernel(LayerView lv, BulkSrc src) {
     const int b = s / lv.Hkv, hk = s % lv.Hkv;
     const uint16_t* qw = src.q + (((size_t)b * lv.Hq + hk * lv.g) * src.n_tokens + src.t0 + (size_t)blockIdx.y * R) * kD;
     const size_t head_stride = (size_t)src.n_tokens * kD;
-    uint16_t* qS = reinterpret_cast<uint16_t*>(cS);                  // [tc tokens][g heads][128], the code area is idle here
-    const int tc = R / 16;                                           // tokens per chunk: R * 128 bytes hold tc * 8 rows
+    uint16_t* qS = reinterpret_cast<uint16_t*>(smem);                // [tc tokens][g heads][128]
+    const int tc = min(R, (R * 384) / (lv.g * 256));                 // tokens per round: R * 384 bytes of key + code area
     for (int j0 = 0; j0 < R; j0 += tc) {
-      for (int i = tid; i < tc * lv.g * 16; i += 256) {
+      const int tn = min(tc, R - j0);
+      for (int i = tid; i < tn * lv.g * 16; i += 256) {
         const int row = i >> 4, c16 = i & 15, jj = row / lv.g, h = row - jj * lv.g;
         reinterpret_cast<uint4*>(qS)[i] = *reinterpret_cast<const uint4*>(qw + (size_t)(j0 + jj) * kD + h * head_stride + 8 * c16);
       }
       __syncthreads();
       if (tid < kD)
-        for (int row = 0; row < tc * lv.g; ++row)
+        for (int row = 0; row < tn * lv.g; ++row)
           bulk_acc = __dadd_rn(bulk_acc, (double)fabsf(bf16_bits_to_float(qS[row * kD + tid])));
       __syncthreads();
     }
   }
-  // ---- statistics, salience, tier and key codes: one thread per channel
-  if (tid < kD) {
-    const int d = tid;
-    float wmx = -INFINITY, wmn = INFINITY;
-    for (int j = 0; j < R; ++j) {
-      float x = bf16_bits_to_float(kS[j * kD + d]);
-      wmx = fmaxf(wmx, x);
-      wmn = fminf(wmn, x);
-    }
-    uint8_t tier;
-    if (src.phase == 2) {
-      tier = tierS[d];
-    } else {
-      double acc;
-      uint32_t cnt;
-      if (bulk) {
-        acc = bulk_acc;
-        cnt = bulk_cnt;
-      } else {
-        acc = reinterpret_cast<const double*>(state)[d];
-        cnt = *reinterpret_cast<const uint32_t*>(state + 1024);
+
+  load_window(resk4);
+  if (src.phase == 2) {
+    // the first pass left the 128 tiers in the first bytes of the block; fetch them before anything is written there
+    if (tid < kD) tierS[tid] = reinterpret_cast<const uint8_t*>(blk)[tid];
+  }
+  __syncthreads();
+
+  // ---- statistics, salience, tier and key codes: two threads per channel (halves of the window for its extrema,
+  // alternate key groups for the codes)
+  {
+    const int d = tid & (kD - 1), half = tid >> 7;
+    if (src.phase != 2) {
+      float wmx = -INFINITY, wmn = INFINITY;
+      for (int j = half * (R / 2); j < (half + 1) * (R / 2); ++j) {
+        float x = bf16_bits_to_float(kS[j * kD + d]);
+        wmx = fmaxf(wmx, x);
+        wmn = fminf(wmn, x);
       }
-      tier = salience_tier(acc, cnt, wmx, wmn, lv.score_bits, lv.tau_bf16, lv.tau_u4, nullptr, lv.importance_mode == 2);
-      if (src.phase == 1) reinterpret_cast<uint8_t*>(blk)[d] = tier;
-    }
-    tierS[d] = tier;
-    const int max_code = (tier == kU4) ? 15 : 3;
-    for (int kg = 0; kg < NG && src.phase != 1; ++kg) {
-      uint32_t meta = 0;
-      if (tier == kBF16) {
-        for (int j = kg * G; j < (kg + 1) * G; ++j) cS[j * kD + d] = 0;
-      } else {
-        float gmx = -INFINITY, gmn = INFINITY;
-        for (int j = kg * G; j < (kg + 1) * G; ++j) {
-          float x = bf16_bits_to_float(kS[j * kD + d]);
-          gmx = fmaxf(gmx, x);
-          gmn = fminf(gmn, x);
+      wS[(half * kD + d) * 2] = wmx;
+      wS[(half * kD + d) * 2 + 1] = wmn;
+      __syncthreads();
+      if (half == 0) {
+        wmx = fmaxf(wS[d * 2], wS[(kD + d) * 2]);
+        wmn = fminf(wS[d * 2 + 1], wS[(kD + d) * 2 + 1]);
+        double acc;
+        uint32_t cnt;
+        if (bulk) {
+          acc = bulk_acc;
+          cnt = bulk_cnt;
+        } else {
+          acc = reinterpret_cast<const double*>(state)[d];
+          cnt = *reinterpret_cast<const uint32_t*>(state + 1024);
         }
-        float sc = stored_scale(gmx, gmn, (float)max_code);
-        for (int j = kg * G; j < (kg + 1) * G; ++j)
-          cS[j * kD + d] = (uint8_t)quant_code(bf16_bits_to_float(kS[j * kD + d]), gmn, sc, max_code);
-        meta = float_to_bf16_bits_exact(sc) | (float_to_bf16_bits_exact(gmn) << 16);
+        const uint8_t tier =
+            salience_tier(acc, cnt, wmx, wmn, lv.score_bits, lv.tau_bf16, lv.tau_u4, nullptr, lv.importance_mode == 2);
+        if (src.phase == 1) reinterpret_cast<uint8_t*>(blk)[d] = tier;
+        tierS[d] = tier;
       }
-      reinterpret_cast<uint32_t*>(blk + (lv.tile ? (uint32_t)kg * 512u : frag_meta_off(kg, G, lv.unit_bytes)))[d] = meta;
+      __syncthreads();
+    }
+    if (src.phase != 1) {
+      const uint8_t tier = tierS[d];
+      const int max_code = (tier == kU4) ? 15 : 3;
+      for (int kg = half; kg < NG; kg += 2) {
+        uint32_t meta = 0;
+        if (tier == kBF16) {
+          for (int j = kg * G; j < (kg + 1) * G; ++j) cS[j * kD + d] = 0;
+        } else {
+          float gmx = -INFINITY, gmn = INFINITY;
+          for (int j = kg * G; j < (kg + 1) * G; ++j) {
+            float x = bf16_bits_to_float(kS[j * kD + d]);
+            gmx = fmaxf(gmx, x);
+            gmn = fminf(gmn, x);
+          }
+          float sc = stored_scale(gmx, gmn, (float)max_code);
+#pragma unroll 4
+          for (int j = kg * G; j < (kg + 1) * G; ++j)
+            cS[j * kD + d] = (uint8_t)quant_code(bf16_bits_to_float(kS[j * kD + d]), gmn, sc, max_code);
+          meta = float_to_bf16_bits_exact(sc) | (float_to_bf16_bits_exact(gmn) << 16);
+        }
+        reinterpret_cast<uint32_t*>(blk + (lv.tile ? (uint32_t)kg * 512u : frag_meta_off(kg, G, lv.unit_bytes)))[d] = meta;
+      }
     }
   }
   __syncthreads();
 
-  // ---- channel lists, extras allocation, table entry
-  if (tid == 0) {
-    int n16 = 0, n4 = 0;
-    for (int d = 0; d < kD; ++d) {
-      if (tierS[d] == kBF16) chan16S[n16++] = (uint8_t)d;
-      else if (tierS[d] == kU4) chan4S[n4++] = (uint8_t)d;
+  // ---- channel lists (ascending channel order inside each tier: warp ballots and a prefix over the four warps)
+  {
+    int* cntS = reinterpret_cast<int*>(wS);          // [2][4] per-warp counts (the extrema are no longer needed)
+    unsigned m16 = 0, m4 = 0;
+    const int warp = tid >> 5, lane = tid & 31;
+    if (tid < kD) {
+      const uint8_t tier = tierS[tid];
+      m16 = __ballot_sync(0xffffffffu, tier == kBF16);
+      m4 = __ballot_sync(0xffffffffu, tier == kU4);
+      if (lane == 0) {
+        cntS[warp] = __popc(m16);
+        cntS[4 + warp] = __popc(m4);
+      }
     }
+    __syncthreads();
+    if (tid < kD) {
+      int b16 = 0, b4 = 0;
+      for (int w2 = 0; w2 < warp; ++w2) {
+        b16 += cntS[w2];
+        b4 += cntS[4 + w2];
+      }
+      const unsigned below = (1u << lane) - 1u;
+      if (m16 & (1u << lane)) chan16S[b16 + __popc(m16 & below)] = (uint8_t)tid;
+      if (m4 & (1u << lane)) chan4S[b4 + __popc(m4 & below)] = (uint8_t)tid;
+    }
+  }
+  // ---- extras allocation, table entry
+  if (tid == 0) {
+    const int* cntS = reinterpret_cast<const int*>(wS);
+    int n16 = cntS[0] + cntS[1] + cntS[2] + cntS[3], n4 = cntS[4] + cntS[5] + cntS[6] + cntS[7];
     uint32_t off16 = 0;
     if (src.phase == 1) {
       // bulk, first pass: only the tier counts; the offsets come from the per-stream prefix sum
@@ -354,7 +403,7 @@ flush_kernel(LayerView lv, BulkSrc src) {
   // takes its place in shared memory (token-major in the residual store and in a tensor alike).
   {
     const uint4* vsrc = bulk ? reinterpret_cast<const uint4*>(src.v + tok0 * kD) : reinterpret_cast<const uint4*>(resv);
-    for (int i = tid; i < R * 16; i += 256) reinterpret_cast<uint4*>(kS)[i] = vsrc[i];
+    load_window(vsrc);
   }
   __syncthreads();
   auto vmeta_of = [&](int j) -> uint32_t* {
@@ -363,34 +412,26 @@ flush_kernel(LayerView lv, BulkSrc src) {
                    : reinterpret_cast<uint32_t*>(blk + frag_unit_off(u, G, lv.unit_bytes) + 2048) + jj * VG;
   };
   {
-    // token-major window: a warp takes a token, lane l the channels l, l+32, l+64, l+96; group extrema by shuffles
+    // token-major window: a warp takes a token, lane l the channels 4l .. 4l+3 (one 8-byte load); a group of G channels
+    // is G / 4 neighbouring lanes, its extrema a butterfly over those lanes
     const int warp = tid >> 5, lane = tid & 31;
+#pragma unroll 2
     for (int j = warp; j < R; j += 8) {
-      float x[4], gmx[4], gmn[4];
-#pragma unroll
-      for (int k = 0; k < 4; ++k) x[k] = gmx[k] = gmn[k] = bf16_bits_to_float(kS[j * kD + lane + 32 * k]);
-      if (G >= 64) {
-        gmx[0] = gmx[1] = fmaxf(x[0], x[1]); gmn[0] = gmn[1] = fminf(x[0], x[1]);
-        gmx[2] = gmx[3] = fmaxf(x[2], x[3]); gmn[2] = gmn[3] = fminf(x[2], x[3]);
+      const uint2 raw = *reinterpret_cast<const uint2*>(&kS[j * kD + 4 * lane]);
+      const float x[4] = {bf16_bits_to_float(raw.x & 0xFFFFu), bf16_bits_to_float(raw.x >> 16),
+                          bf16_bits_to_float(raw.y & 0xFFFFu), bf16_bits_to_float(raw.y >> 16)};
+      float gmx = fmaxf(fmaxf(x[0], x[1]), fmaxf(x[2], x[3])), gmn = fminf(fminf(x[0], x[1]), fminf(x[2], x[3]));
+      for (int off = 1; off < G / 4; off <<= 1) {
+        gmx = fmaxf(gmx, __shfl_xor_sync(0xffffffffu, gmx, off));
+        gmn = fminf(gmn, __shfl_xor_sync(0xffffffffu, gmn, off));
       }
-      if (G == 128) {
-        gmx[0] = gmx[1] = gmx[2] = gmx[3] = fmaxf(gmx[0], gmx[2]);
-        gmn[0] = gmn[1] = gmn[2] = gmn[3] = fminf(gmn[0], gmn[2]);
-      }
+      const float sc = stored_scale(gmx, gmn, 3.0f);
+      uint32_t codes = 0;
 #pragma unroll
-      for (int off = 16; off; off >>= 1)
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          gmx[k] = fmaxf(gmx[k], __shfl_xor_sync(0xffffffffu, gmx[k], off));
-          gmn[k] = fminf(gmn[k], __shfl_xor_sync(0xffffffffu, gmn[k], off));
-        }
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const float sc = stored_scale(gmx[k], gmn[k], 3.0f);
-        cS[j * kD + lane + 32 * k] = (uint8_t)quant_code(x[k], gmn[k], sc, 3);
-        const int vg = (32 * k) / G;
-        if (lane == 0 && (32 * k) % G == 0) vmeta_of(j)[vg] = float_to_bf16_bits_exact(sc) | (float_to_bf16_bits_exact(gmn[k]) << 16);
-      }
+      for (int k = 0; k < 4; ++k) codes |= (uint32_t)quant_code(x[k], gmn, sc, 3) << (8 * k);
+      *reinterpret_cast<uint32_t*>(&cS[j * kD + 4 * lane]) = codes;
+      if ((4 * lane) % G == 0)
+        vmeta_of(j)[(4 * lane) / G] = float_to_bf16_bits_exact(sc) | (float_to_bf16_bits_exact(gmn) << 16);
     }
   }
   __syncthreads();
@@ -435,7 +476,7 @@ flush_kernel(LayerView lv, BulkSrc src) {
   }
 }
 
-static size_t flush_smem_bytes(int R) { return (size_t)R * 384 + 3 * 128 + 16; }
+static size_t flush_smem_bytes(int R) { return (size_t)R * 384 + 3 * 128 + 16 + 2048; }
 
 cudaError_t launch_flush(const LayerView& lv, cudaStream_t stream) {
   cudaError_t e = cudaFuncSetAttribute(flush_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -153,10 +153,20 @@ flush_kernel(LayerView lv, BulkSrc src) {
     uint16_t* qS = reinterpret_cast<uint16_t*>(smem);                // [tc tokens][g heads][128]
     const int tc = min(R, (R * 384) / (lv.g * 256));                 // tokens per round: R * 384 bytes of key + code area
     for (int j0 = 0; j0 < R; j0 += tc) {
-      const int tn = min(tc, R - j0);
-      for (int i = tid; i < tn * lv.g * 16; i += 256) {
-        const int row = i >> 4, c16 = i & 15, jj = row / lv.g, h = row - jj * lv.g;
-        reinterpret_cast<uint4*>(qS)[i] = *reinterpret_cast<const uint4*>(qw + (size_t)(j0 + jj) * kD + h * head_stride + 8 * c16);
+      const int tn = min(tc, R - j0), pieces = tn * lv.g * 16;
+      for (int i0 = 0; i0 < pieces; i0 += 4 * 256) {       // four loads per thread in flight, then the stores
+        uint4 tmp[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int i = i0 + tid + 256 * k;
+          if (i < pieces) {
+            const int row = i >> 4, c16 = i & 15, jj = row / lv.g, h = row - jj * lv.g;
+            tmp[k] = *reinterpret_cast<const uint4*>(qw + (size_t)(j0 + jj) * kD + h * head_stride + 8 * c16);
+          }
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          if (i0 + tid + 256 * k < pieces) reinterpret_cast<uint4*>(qS)[i0 + tid + 256 * k] = tmp[k];
       }
       __syncthreads();
       if (tid < kD)
@@ -221,9 +231,10 @@ flush_kernel(LayerView lv, BulkSrc src) {
             gmn = fminf(gmn, x);
           }
           float sc = stored_scale(gmx, gmn, (float)max_code);
+          const float rs = __frcp_rn(sc);
 #pragma unroll 4
           for (int j = kg * G; j < (kg + 1) * G; ++j)
-            cS[j * kD + d] = (uint8_t)quant_code(bf16_bits_to_float(kS[j * kD + d]), gmn, sc, max_code);
+            cS[j * kD + d] = (uint8_t)quant_code_fast(bf16_bits_to_float(kS[j * kD + d]), gmn, sc, rs, max_code);
           meta = float_to_bf16_bits_exact(sc) | (float_to_bf16_bits_exact(gmn) << 16);
         }
         reinterpret_cast<uint32_t*>(blk + (lv.tile ? (uint32_t)kg * 512u : frag_meta_off(kg, G, lv.unit_bytes)))[d] = meta;
@@ -426,9 +437,10 @@ flush_kernel(LayerView lv, BulkSrc src) {
         gmn = fminf(gmn, __shfl_xor_sync(0xffffffffu, gmn, off));
       }
       const float sc = stored_scale(gmx, gmn, 3.0f);
+      const float rs = __frcp_rn(sc);
       uint32_t codes = 0;
 #pragma unroll
-      for (int k = 0; k < 4; ++k) codes |= (uint32_t)quant_code(x[k], gmn, sc, 3) << (8 * k);
+      for (int k = 0; k < 4; ++k) codes |= (uint32_t)quant_code_fast(x[k], gmn, sc, rs, 3) << (8 * k);
       *reinterpret_cast<uint32_t*>(&cS[j * kD + 4 * lane]) = codes;
       if ((4 * lane) % G == 0)
         vmeta_of(j)[(4 * lane) / G] = float_to_bf16_bits_exact(sc) | (float_to_bf16_bits_exact(gmn) << 16);

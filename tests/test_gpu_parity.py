@@ -155,6 +155,30 @@ def test_other_importance_modes(binding, mode):
     assert len({int(x) for st in orc.values() for blk in st.blocks for x in blk.tiers}) == 3
 
 
+def test_rounding_ties_are_bit_exact(binding):
+    # keys and values on a grid of half-steps of their scale: every group spans 0 .. 3 (2-bit scale exactly 1, a
+    # second stream 0 .. 3 * 0.75 with a scale that is not a power of two), so (x - z) / s falls on exact half-integers
+    # for about half of the elements; the codes must follow round-half-even of the IEEE quotient like the oracle's
+    w = small("qwen7b", batch=2, tokens=4 * 128 + 40, **W.P24)
+    gen = torch.Generator().manual_seed(1234)
+    shape = (w.batch, w.n_kv_heads, w.tokens, 128)
+    k = torch.randint(0, 7, shape, generator=gen).float() * 0.5
+    v = torch.randint(0, 7, shape, generator=gen).float() * 0.5
+    k[:, :, 0::32] = 0.0; k[:, :, 1::32] = 3.0          # every 32-token key group holds its extremes
+    v[..., 0::32] = 0.0; v[..., 1::32] = 3.0            # every 32-channel value group too
+    k[1] *= 0.75; v[1] *= 0.75
+    k, v = k.to(torch.bfloat16), v.to(torch.bfloat16)
+    _, _, q = W.tokens(w, 0, 0, w.tokens)
+    cache = U.make_cache(binding, w)
+    cache.quantize_append(0, k.cuda(), v.cuda(), q.cuda())
+    orc = U.oracle_streams(w, 0, k, v, q)
+    U.compare_regions(cache, 0, w, orc)
+    codes = np.concatenate([blk.kcodes.ravel() for st in orc.values() for blk in st.blocks] +
+                           [blk.vcodes.ravel() for st in orc.values() for blk in st.blocks])
+    assert set(np.unique(codes)) == {0, 1, 2, 3}
+    assert cache.status() == 0
+
+
 # ------------------------------------------------------------------------------------------- attention
 @pytest.mark.parametrize("kind,layout", [(0, 0), (1, 0), (0, 1), (1, 1)])
 @pytest.mark.parametrize("name,tokens,preset", [

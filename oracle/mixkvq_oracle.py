@@ -125,6 +125,24 @@ def assign_tiers(A, tau_bf16, tau_u4):
     return tiers
 
 
+def assign_tiers_by_budget(A, budget_bf16, budget_u4):
+    """Fixed-budget form of the tier rule of Section 4.2: the budget_bf16 channels of highest salience go to BF16, the next
+    budget_u4 to UINT4, the rest to UINT2 (equal saliences: the lower channel index ranks first).  With no ties this is
+    the threshold rule for any tau_bf16 between the budget_bf16-th and the next salience (and likewise tau_u4)."""
+    A = np.asarray(A, np.float64)
+    tiers = np.full(A.shape, TIER_U2, np.uint8)
+    for d in range(A.shape[0]):
+        rank = 0
+        for e in range(A.shape[0]):
+            if A[e] > A[d] or (A[e] == A[d] and e < d):
+                rank += 1
+        if rank < budget_bf16:
+            tiers[d] = TIER_BF16
+        elif rank < budget_bf16 + budget_u4:
+            tiers[d] = TIER_U4
+    return tiers
+
+
 def importance_from_queries(q):
     """|q| summed in token-major, head-ascending order.  q float32 [g, n, D] -> (acc fp64 [D], cnt)."""
     q = np.asarray(q, np.float32)
@@ -160,11 +178,13 @@ class Block:
 
 
 class OracleStream:
-    def __init__(self, g, R=128, G=32, score_bits=2, tau_bf16=1e30, tau_u4=1e30, importance_mode=0):
+    def __init__(self, g, R=128, G=32, score_bits=2, tau_bf16=1e30, tau_u4=1e30, importance_mode=0, budget_bf16=0,
+                 budget_u4=0):
         assert R % 32 == 0 and R % G == 0 and D % G == 0
         self.g, self.R, self.G = g, R, G
         self.score_bits, self.tau_bf16, self.tau_u4 = score_bits, tau_bf16, tau_u4
         self.importance_mode = importance_mode
+        self.budget_bf16, self.budget_u4 = budget_bf16, budget_u4      # both 0: thresholds decide
         self.blocks: list[Block] = []
         self.resK = np.zeros((R, D), np.float32)
         self.resV = np.zeros((R, D), np.float32)
@@ -208,6 +228,8 @@ class OracleStream:
 
     def current_tiers(self):
         _, _, A = self.current_scores()
+        if self.budget_bf16 + self.budget_u4 > 0:
+            return assign_tiers_by_budget(A, self.budget_bf16, self.budget_u4), A
         return assign_tiers(A, self.tau_bf16, self.tau_u4), A
 
     def flush(self):
@@ -592,7 +614,7 @@ def pack_stream(st: OracleStream, layout=LAYOUT_FRAGMENT):
             ex, n16, n4 = pack_extras_tile(blk)
         else:
             base.append(pack_base(blk, st.R, st.G))
-            ex, n16, n4 = pack_extras(blk, st.R, dense_high_plane(st.tau_u4))
+            ex, n16, n4 = pack_extras(blk, st.R, dense_high_plane(st.tau_u4) and st.budget_bf16 + st.budget_u4 == 0)
         table.append(table_entry(used16, n16, n4))
         extras.append(ex)
         used16 += len(ex) // 16

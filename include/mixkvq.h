@@ -73,6 +73,11 @@ typedef struct mixkvq_config {
                                          1: tile layout (R must be 128; tcgen05 attention kernel)        */
   uint64_t extras_budget_bytes;       /* per stream, for promoted channels; 0 = library default
                                          (1/8 of the bf16 size of max_tokens keys)                   */
+  int32_t budget_bf16;                /* fixed-budget form of the tier rule of Section 4.2: when budget_bf16 +     */
+  int32_t budget_u4;                  /* budget_u4 > 0 the thresholds are ignored; the budget_bf16 channels of highest
+                                         salience A_d of a window go to BF16, the next budget_u4 to UINT4, the rest to
+                                         UINT2 (equal saliences: lower channel first).  Every block then has the same
+                                         tier counts.  Sum <= 128                                       */
 } mixkvq_config;
 
 typedef struct mixkvq_cache mixkvq_cache;

@@ -30,6 +30,7 @@ class Config(C.Structure):
         ("head_dim", C.c_int32), ("max_tokens", C.c_int32), ("residual_len", C.c_int32), ("group_size", C.c_int32),
         ("v_bits", C.c_int32), ("score_bits", C.c_int32), ("tau_bf16", C.c_float), ("tau_u4", C.c_float),
         ("importance_mode", C.c_int32), ("block_layout", C.c_int32), ("extras_budget_bytes", C.c_uint64),
+        ("budget_bf16", C.c_int32), ("budget_u4", C.c_int32),
     ]
 
 
@@ -104,9 +105,9 @@ def _ptr(t: torch.Tensor | None):
 
 def make_config(n_layers, batch, n_q_heads, n_kv_heads, max_tokens, residual_len=128, group_size=32,
                 tau_bf16=1e30, tau_u4=1e30, score_bits=2, importance_mode=0, extras_budget_bytes=0,
-                block_layout=0) -> Config:
+                block_layout=0, budget_bf16=0, budget_u4=0) -> Config:
     return Config(n_layers, batch, n_q_heads, n_kv_heads, 128, max_tokens, residual_len, group_size, 2, score_bits,
-                  tau_bf16, tau_u4, importance_mode, block_layout, extras_budget_bytes)
+                  tau_bf16, tau_u4, importance_mode, block_layout, extras_budget_bytes, budget_bf16, budget_u4)
 
 
 def cache_bytes(cfg: Config):

@@ -43,6 +43,7 @@ int check_config(const mixkvq_config* c) {
   if (c->score_bits != 2 && c->score_bits != 4) return MIXKVQ_E_UNSUPPORTED;
   if (c->importance_mode < 0 || c->importance_mode > 2) return MIXKVQ_E_INVALID_ARG;
   if (c->block_layout != 0 && c->block_layout != 1) return MIXKVQ_E_INVALID_ARG;
+  if (c->budget_bf16 < 0 || c->budget_u4 < 0 || c->budget_bf16 + c->budget_u4 > kD) return MIXKVQ_E_INVALID_ARG;
   if (c->block_layout == 1 && c->residual_len != 128) return MIXKVQ_E_UNSUPPORTED;
   return MIXKVQ_OK;
 }
@@ -90,7 +91,8 @@ LayerView view(const mixkvq_cache* h, int layer) {
   v.max_blocks = h->max_blocks;
   v.n_blocks = h->n_blocks[layer]; v.r = h->r[layer];
   v.tile = h->tile;
-  v.dense_hi = (h->cfg.tau_u4 < 0.0f) ? 1 : 0;
+  v.budget_bf16 = h->cfg.budget_bf16; v.budget_u4 = h->cfg.budget_u4;
+  v.dense_hi = (h->cfg.tau_u4 < 0.0f && v.budget_bf16 + v.budget_u4 == 0) ? 1 : 0;
   v.base_bytes = h->base_bytes; v.unit_bytes = h->unit_bytes;
   v.extras_budget = h->extras_budget;
   v.score_bits = h->cfg.score_bits; v.importance_mode = h->cfg.importance_mode;

@@ -882,7 +882,8 @@ cudaError_t launch_g(const LayerView& lv, const void* q, float scale, float* ws,
   const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q);
   const float sl = scale * 1.4426950408889634f;
   if (lv.dense_hi) return launch_one<G, 2>(lv, qb, sl, ws, grid, stream);
-  if (lv.tau_u4 < lv.tau_bf16) return launch_one<G, 1>(lv, qb, sl, ws, grid, stream);
+  const bool uses_u4 = (lv.budget_bf16 + lv.budget_u4 > 0) ? lv.budget_u4 > 0 : lv.tau_u4 < lv.tau_bf16;
+  if (uses_u4) return launch_one<G, 1>(lv, qb, sl, ws, grid, stream);
   return launch_one<G, 0>(lv, qb, sl, ws, grid, stream);
 }
 

@@ -32,6 +32,7 @@ struct LayerView {
   // method parameters
   int score_bits, importance_mode;
   float tau_bf16, tau_u4;
+  int budget_bf16, budget_u4; // fixed-budget tiering when their sum is positive (the thresholds are then unused)
   // per-stream arrays (base pointer + stride in bytes)
   char* state;  uint64_t state_stride;
   char* table;  uint64_t table_stride;
@@ -122,6 +123,18 @@ __device__ inline uint8_t salience_tier(double acc, uint32_t cnt, float mx, floa
   if (A > (double)tau_bf16) return kBF16;
   if (A > (double)tau_u4) return kU4;
   return kU2;
+}
+
+// Fixed-budget form of the tier rule: channel d's rank among the 128 saliences (descending, equal values by channel
+// index) against the two quotas.
+__device__ inline uint8_t budget_tier(const double* A, int d, int budget_bf16, int budget_u4) {
+  const double a = A[d];
+  int rank = 0;
+  for (int e = 0; e < kD; ++e) {
+    const double b = A[e];
+    rank += (b > a || (b == a && e < d)) ? 1 : 0;
+  }
+  return rank < budget_bf16 ? kBF16 : (rank < budget_bf16 + budget_u4 ? kU4 : kU2);
 }
 
 // ---- fragment layout: positions inside a 32-token unit.  The codes are ordered so that one 16-byte load per lane

@@ -112,6 +112,7 @@ flush_kernel(LayerView lv, BulkSrc src) {
   uint8_t* chan4S = chan16S + 128;                        // [128]
   int* misc = reinterpret_cast<int*>(chan4S + 128);       // n16, n4, extras offset (16-byte units)
   float* wS = reinterpret_cast<float*>(chan4S + 128 + 16); // [2 halves][128]{max, min} of the window, later the tier counts
+  double* aS = reinterpret_cast<double*>(chan4S + 128 + 16 + 2048);   // [128] saliences of the window
 
   const int s = blockIdx.x, tid = threadIdx.x;
   const bool bulk = src.phase != 0;
@@ -209,11 +210,17 @@ flush_kernel(LayerView lv, BulkSrc src) {
           acc = reinterpret_cast<const double*>(state)[d];
           cnt = *reinterpret_cast<const uint32_t*>(state + 1024);
         }
+        double A;
         const uint8_t tier =
-            salience_tier(acc, cnt, wmx, wmn, lv.score_bits, lv.tau_bf16, lv.tau_u4, nullptr, lv.importance_mode == 2);
-        if (src.phase == 1) reinterpret_cast<uint8_t*>(blk)[d] = tier;
+            salience_tier(acc, cnt, wmx, wmn, lv.score_bits, lv.tau_bf16, lv.tau_u4, &A, lv.importance_mode == 2);
+        aS[d] = A;
         tierS[d] = tier;
       }
+      if (lv.budget_bf16 + lv.budget_u4 > 0) {     // fixed budget: the rank among the window's saliences decides
+        __syncthreads();
+        if (half == 0) tierS[d] = budget_tier(aS, d, lv.budget_bf16, lv.budget_u4);
+      }
+      if (half == 0 && src.phase == 1) reinterpret_cast<uint8_t*>(blk)[d] = tierS[d];
       __syncthreads();
     }
     if (src.phase != 1) {
@@ -488,7 +495,7 @@ flush_kernel(LayerView lv, BulkSrc src) {
   }
 }
 
-static size_t flush_smem_bytes(int R) { return (size_t)R * 384 + 3 * 128 + 16 + 2048; }
+static size_t flush_smem_bytes(int R) { return (size_t)R * 384 + 3 * 128 + 16 + 2048 + 1024; }
 
 cudaError_t launch_flush(const LayerView& lv, cudaStream_t stream) {
   cudaError_t e = cudaFuncSetAttribute(flush_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,

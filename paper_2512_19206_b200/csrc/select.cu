@@ -19,6 +19,12 @@ select_window_kernel(LayerView lv, uint8_t* __restrict__ tiers, double* __restri
   uint32_t cnt = *reinterpret_cast<const uint32_t*>(st + 1024);
   double A;
   uint8_t t = salience_tier(acc, cnt, mx, mn, lv.score_bits, lv.tau_bf16, lv.tau_u4, &A, lv.importance_mode == 2);
+  if (lv.budget_bf16 + lv.budget_u4 > 0) {       // fixed budget: rank among the 128 saliences
+    __shared__ double aS[kD];
+    aS[d] = A;
+    __syncthreads();
+    t = budget_tier(aS, d, lv.budget_bf16, lv.budget_u4);
+  }
   tiers[(size_t)s * kD + d] = t;
   if (salience) salience[(size_t)s * kD + d] = A;
 }

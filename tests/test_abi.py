@@ -28,7 +28,7 @@ def test_library_exports_every_declared_symbol(binding):
 
 
 def test_config_struct_matches_header(binding):
-    assert C.sizeof(binding.Config) == 64
+    assert C.sizeof(binding.Config) == 72          # 14 int32/float fields, one uint64, the two budgets
     assert C.sizeof(binding.LayoutDesc) == 13 * 8 + 4 * 4
 
 

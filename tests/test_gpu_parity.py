@@ -179,6 +179,29 @@ def test_rounding_ties_are_bit_exact(binding):
     assert cache.status() == 0
 
 
+@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("k16,k4", [(4, 0), (3, 24), (0, 9)])
+def test_fixed_budget_tiering(binding, layout, k16, k4):
+    # the top k16 channels by salience in BF16, the next k4 in UINT4, whatever the thresholds say: constant tier counts per
+    # block, bytes and scores equal to the oracle's, attention within tolerance
+    w = small("qwen7b", batch=2, tokens=5 * 128 + 33, **W.P24)
+    k, v, q = W.tokens(w, 0, 0, w.tokens)
+    cache = U.make_cache(binding, w, layout=layout, budget_bf16=k16, budget_u4=k4)
+    cache.quantize_append(0, k.cuda(), v.cuda(), q.cuda())
+    orc = U.oracle_streams(w, 0, k, v, q, budget_bf16=k16, budget_u4=k4)
+    U.compare_regions(cache, 0, w, orc)
+    tiers, sal = cache.select_channels(0)
+    for (b, hk), st in orc.items():
+        t, A = st.current_tiers()
+        assert np.array_equal(tiers[b, hk].cpu().numpy(), t) and np.array_equal(sal[b, hk].cpu().numpy(), A)
+        assert all(int((blk.tiers == O.TIER_BF16).sum()) == k16 and int((blk.tiers == O.TIER_U4).sum()) == k4
+                   for blk in st.blocks)
+    qd = W.decode_query(w, 0, 0)
+    out = cache.decode_attention(0, qd.cuda(), W.softmax_scale())
+    assert U.max_abs_err(w, out, U.oracle_attention(w, orc, qd)) <= ATTN_TOL
+    assert cache.status() == 0
+
+
 # ------------------------------------------------------------------------------------------- attention
 @pytest.mark.parametrize("kind,layout", [(0, 0), (1, 0), (0, 1), (1, 1)])
 @pytest.mark.parametrize("name,tokens,preset", [

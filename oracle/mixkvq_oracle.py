@@ -179,12 +179,19 @@ class Block:
 
 class OracleStream:
     def __init__(self, g, R=128, G=32, score_bits=2, tau_bf16=1e30, tau_u4=1e30, importance_mode=0, budget_bf16=0,
-                 budget_u4=0):
+                 budget_u4=0, sink_len=0):
         assert R % 32 == 0 and R % G == 0 and D % G == 0
         self.g, self.R, self.G = g, R, G
         self.score_bits, self.tau_bf16, self.tau_u4 = score_bits, tau_bf16, tau_u4
         self.importance_mode = importance_mode
         self.budget_bf16, self.budget_u4 = budget_bf16, budget_u4      # both 0: thresholds decide
+        # sink tokens (the "sink length" of the paper's experimental settings, Appendix E): the first sink_len tokens of
+        # the sequence stay in full precision for good; they never enter the residual window, the importance
+        # accumulator or a quantized block
+        self.sink_len = sink_len
+        self.sinkK = np.zeros((sink_len, D), np.float32)
+        self.sinkV = np.zeros((sink_len, D), np.float32)
+        self.n_sink = 0
         self.blocks: list[Block] = []
         self.resK = np.zeros((R, D), np.float32)
         self.resV = np.zeros((R, D), np.float32)
@@ -196,6 +203,11 @@ class OracleStream:
     # -- Appendix D.1: append into the residual buffer; flush lazily when it already holds R tokens
     def append(self, k, v, q):
         """k, v float32 [D]; q float32 [g, D] (all bf16-valued)."""
+        if self.n_sink < self.sink_len:
+            self.sinkK[self.n_sink] = k
+            self.sinkV[self.n_sink] = v
+            self.n_sink += 1
+            return
         if self.r == self.R:
             self.flush()
         self.resK[self.r] = k
@@ -208,6 +220,9 @@ class OracleStream:
         """k, v [n, D]; q [g, n, D].  Defined as n single appends in token order."""
         n = k.shape[0]
         t = 0
+        while t < n and self.n_sink < self.sink_len:
+            self.append(k[t], v[t], q[:, t])
+            t += 1
         while t < n:
             if self.r == self.R:
                 self.flush()
@@ -262,7 +277,7 @@ class OracleStream:
 
     # -- dequantized views (fp64)
     def keys(self):
-        parts = []
+        parts = [self.sinkK[:self.n_sink].astype(np.float64)]
         for b in self.blocks:
             NG = b.ks.shape[0]
             kq = (b.kcodes.reshape(NG, self.G, D).astype(np.float64) * b.ks.astype(np.float64)[:, None, :]
@@ -272,7 +287,7 @@ class OracleStream:
         return np.concatenate(parts, axis=0)
 
     def values(self):
-        parts = []
+        parts = [self.sinkV[:self.n_sink].astype(np.float64)]
         for b in self.blocks:
             VG = D // self.G
             vq = (b.vcodes.reshape(self.R, VG, self.G).astype(np.float64) * b.vs.astype(np.float64)[..., None]
@@ -283,7 +298,7 @@ class OracleStream:
 
     @property
     def n_tokens(self):
-        return len(self.blocks) * self.R + self.r
+        return self.n_sink + len(self.blocks) * self.R + self.r
 
     # -- Eq. 1
     def attention(self, q, scale, return_probs=False):
@@ -629,4 +644,6 @@ def pack_stream(st: OracleStream, layout=LAYOUT_FRAGMENT):
         "state": bytes(state),
         "resK": bf16_to_u16(st.resK[:st.r]).astype("<u2").tobytes(),
         "resV": bf16_to_u16(st.resV[:st.r]).astype("<u2").tobytes(),
+        "sinkK": bf16_to_u16(st.sinkK[:st.n_sink]).astype("<u2").tobytes(),
+        "sinkV": bf16_to_u16(st.sinkV[:st.n_sink]).astype("<u2").tobytes(),
     }

@@ -233,7 +233,7 @@ def run_gpu(args, w):
     cfg = binding.make_config(w.n_layers, w.batch, w.n_q_heads, w.n_kv_heads, w.tokens + n_steps + 2 * w.residual_len,
                               residual_len=w.residual_len, group_size=w.group_size, tau_bf16=w.tau_bf16,
                               tau_u4=w.tau_u4, score_bits=w.score_bits, block_layout=args.layout,
-                              importance_mode=args.importance_mode,
+                              importance_mode=args.importance_mode, sink_len=args.sink_len,
                               extras_budget_bytes=((w.tokens + n_steps) // w.residual_len + 3) * 8192 if w.score_bits == 4 else 0)
     cache = binding.Cache(cfg, device=dev)
     prefill_ms = prefill(cache, w, dev)
@@ -405,6 +405,7 @@ def main():
     ap.add_argument("--residual-len", type=int, default=None, help="R: residual window / block length (32 .. 256)")
     ap.add_argument("--importance-mode", type=int, default=0, choices=[0, 1, 2],
                     help="0: window importance (default), 1: cumulative, 2: error-only salience")
+    ap.add_argument("--sink-len", type=int, default=0, help="sink tokens kept in bf16 (0, or a multiple of 32 up to 256)")
     ap.add_argument("--tokens", type=int, default=None)
     ap.add_argument("--layers", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

@@ -78,6 +78,10 @@ typedef struct mixkvq_config {
                                          salience A_d of a window go to BF16, the next budget_u4 to UINT4, the rest to
                                          UINT2 (equal saliences: lower channel first).  Every block then has the same
                                          tier counts.  Sum <= 128                                       */
+  int32_t sink_len;                   /* sink tokens (the "sink length" of the settings in Appendix E): the first sink_len
+                                         tokens of every sequence stay in bf16 for good, outside the residual window, the
+                                         importance accumulator and the quantized blocks.  0, or a multiple of 32 <= 256 */
+  int32_t reserved;                   /* must be 0                                                    */
 } mixkvq_config;
 
 typedef struct mixkvq_cache mixkvq_cache;
@@ -94,6 +98,8 @@ typedef struct mixkvq_layout_desc {
   uint64_t base_bytes;                    /* size of one block's fixed part                          */
   uint32_t max_blocks, n_streams;
   uint32_t n_blocks, residual_tokens;     /* current fill of this layer (same for all streams)       */
+  uint64_t sink_off, sink_stride;         /* per stream: [sink_len][128] bf16 keys, then the same for values */
+  uint32_t sink_tokens, sink_len;         /* sink rows filled so far, and their capacity              */
 } mixkvq_layout_desc;
 
 /* Sizes the caller must provide: the cache memory for all layers and the workspace of one

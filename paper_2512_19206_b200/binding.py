@@ -30,7 +30,7 @@ class Config(C.Structure):
         ("head_dim", C.c_int32), ("max_tokens", C.c_int32), ("residual_len", C.c_int32), ("group_size", C.c_int32),
         ("v_bits", C.c_int32), ("score_bits", C.c_int32), ("tau_bf16", C.c_float), ("tau_u4", C.c_float),
         ("importance_mode", C.c_int32), ("block_layout", C.c_int32), ("extras_budget_bytes", C.c_uint64),
-        ("budget_bf16", C.c_int32), ("budget_u4", C.c_int32),
+        ("budget_bf16", C.c_int32), ("budget_u4", C.c_int32), ("sink_len", C.c_int32), ("reserved", C.c_int32),
     ]
 
 
@@ -38,7 +38,8 @@ class LayoutDesc(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in (
         "state_off", "state_stride", "table_off", "table_stride", "resk_off", "resk_stride",
         "resv_off", "resv_stride", "base_off", "base_stride", "extras_off", "extras_stride", "base_bytes")] + [
-        (n, C.c_uint32) for n in ("max_blocks", "n_streams", "n_blocks", "residual_tokens")]
+        (n, C.c_uint32) for n in ("max_blocks", "n_streams", "n_blocks", "residual_tokens")] + [
+        ("sink_off", C.c_uint64), ("sink_stride", C.c_uint64), ("sink_tokens", C.c_uint32), ("sink_len", C.c_uint32)]
 
 
 class MixKVQError(RuntimeError):
@@ -105,9 +106,10 @@ def _ptr(t: torch.Tensor | None):
 
 def make_config(n_layers, batch, n_q_heads, n_kv_heads, max_tokens, residual_len=128, group_size=32,
                 tau_bf16=1e30, tau_u4=1e30, score_bits=2, importance_mode=0, extras_budget_bytes=0,
-                block_layout=0, budget_bf16=0, budget_u4=0) -> Config:
+                block_layout=0, budget_bf16=0, budget_u4=0, sink_len=0) -> Config:
     return Config(n_layers, batch, n_q_heads, n_kv_heads, 128, max_tokens, residual_len, group_size, 2, score_bits,
-                  tau_bf16, tau_u4, importance_mode, block_layout, extras_budget_bytes, budget_bf16, budget_u4)
+                  tau_bf16, tau_u4, importance_mode, block_layout, extras_budget_bytes, budget_bf16, budget_u4,
+                  sink_len, 0)
 
 
 def cache_bytes(cfg: Config):
@@ -234,4 +236,6 @@ class Cache:
             "state": state,
             "resK": resk[: r * 256],
             "resV": resv[: r * 256],
+            "sinkK": cut(d.sink_off, d.sink_stride, d.sink_tokens * 256),
+            "sinkV": cut(d.sink_off + d.sink_len * 256, d.sink_stride, d.sink_tokens * 256),
         }

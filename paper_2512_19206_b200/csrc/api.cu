@@ -15,9 +15,9 @@ struct mixkvq_cache {
   uint32_t base_bytes, unit_bytes;
   uint64_t extras_budget;
   // byte offsets inside one layer and per-stream strides
-  uint64_t state_off, table_off, resk_off, resv_off, base_off, extras_off, layer_stride;
-  uint64_t state_stride, table_stride, resk_stride, resv_stride, base_stride, extras_stride;
-  std::vector<int> n_blocks, r;
+  uint64_t state_off, table_off, resk_off, resv_off, base_off, extras_off, sink_off, layer_stride;
+  uint64_t state_stride, table_stride, resk_stride, resv_stride, base_stride, extras_stride, sink_stride;
+  std::vector<int> n_blocks, r, n_sink;
   int n_sms;
   int attn_kind;
   uint64_t launches;
@@ -44,6 +44,7 @@ int check_config(const mixkvq_config* c) {
   if (c->importance_mode < 0 || c->importance_mode > 2) return MIXKVQ_E_INVALID_ARG;
   if (c->block_layout != 0 && c->block_layout != 1) return MIXKVQ_E_INVALID_ARG;
   if (c->budget_bf16 < 0 || c->budget_u4 < 0 || c->budget_bf16 + c->budget_u4 > kD) return MIXKVQ_E_INVALID_ARG;
+  if (c->sink_len < 0 || c->sink_len > 256 || c->sink_len % 32 != 0 || c->reserved != 0) return MIXKVQ_E_INVALID_ARG;
   if (c->block_layout == 1 && c->residual_len != 128) return MIXKVQ_E_UNSUPPORTED;
   return MIXKVQ_OK;
 }
@@ -71,6 +72,7 @@ uint64_t plan(const mixkvq_config* c, mixkvq_cache* h) {
   h->resv_stride = (uint64_t)h->R * 256;
   h->base_stride = (uint64_t)h->max_blocks * h->base_bytes;
   h->extras_stride = align_up(h->extras_budget, 256);
+  h->sink_stride = (uint64_t)c->sink_len * 512;      // keys then values, 256 bytes a row
   uint64_t off = 0;
   h->state_off = off;  off = align_up(off + h->state_stride * h->S, 256);
   h->table_off = off;  off = align_up(off + h->table_stride * h->S, 256);
@@ -78,6 +80,7 @@ uint64_t plan(const mixkvq_config* c, mixkvq_cache* h) {
   h->resv_off = off;   off = align_up(off + h->resv_stride * h->S, 256);
   h->base_off = off;   off = align_up(off + h->base_stride * h->S, 256);
   h->extras_off = off; off = align_up(off + h->extras_stride * h->S, 256);
+  h->sink_off = off;   off = align_up(off + h->sink_stride * h->S, 256);
   h->layer_stride = off;
   return kHeaderBytes + h->layer_stride * (uint64_t)c->n_layers;
 }
@@ -104,6 +107,8 @@ LayerView view(const mixkvq_cache* h, int layer) {
   v.resv = L + h->resv_off;     v.resv_stride = h->resv_stride;
   v.base = L + h->base_off;     v.base_stride = h->base_stride;
   v.extras = L + h->extras_off; v.extras_stride = h->extras_stride;
+  v.sink = L + h->sink_off;     v.sink_stride = h->sink_stride;
+  v.sink_len = h->cfg.sink_len; v.n_sink = h->n_sink[layer];
   v.status = reinterpret_cast<uint32_t*>(h->mem);
   return v;
 }
@@ -115,6 +120,7 @@ int zero_layer_state(mixkvq_cache* h, int layer, cudaStream_t st) {
   if (cudaMemsetAsync(L + h->state_off, 0, h->state_stride * h->S, st) != cudaSuccess) return MIXKVQ_E_CUDA;
   h->n_blocks[layer] = 0;
   h->r[layer] = 0;
+  h->n_sink[layer] = 0;
   return MIXKVQ_OK;
 }
 
@@ -163,6 +169,7 @@ int mixkvq_cache_init(const mixkvq_config* cfg, void* cache_dev, size_t bytes, v
   h->bytes = bytes;
   h->n_blocks.assign(cfg->n_layers, 0);
   h->r.assign(cfg->n_layers, 0);
+  h->n_sink.assign(cfg->n_layers, 0);
   h->attn_kind = 0;
   h->launches = 0;
   int dev = 0;
@@ -221,11 +228,22 @@ int mixkvq_quantize_append(mixkvq_cache* cache, int layer, const void* k_dev, co
   if (!cache || !k_dev || !v_dev || !q_dev || layer < 0 || layer >= cache->cfg.n_layers || n_tokens < 1)
     return MIXKVQ_E_INVALID_ARG;
   if (!aligned16(k_dev) || !aligned16(v_dev) || !aligned16(q_dev)) return MIXKVQ_E_ALIGNMENT;
-  const long long have = (long long)cache->n_blocks[layer] * cache->R + cache->r[layer];
+  const long long have = (long long)cache->n_sink[layer] + (long long)cache->n_blocks[layer] * cache->R + cache->r[layer];
   if (have + n_tokens > cache->cfg.max_tokens) return MIXKVQ_E_CAPACITY;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int t = 0;
   while (t < n_tokens) {
+    if (cache->n_sink[layer] < cache->cfg.sink_len) {
+      // the first tokens of the sequence are sink tokens: stored as they are, outside everything else
+      const int room = cache->cfg.sink_len - cache->n_sink[layer];
+      const int m = n_tokens - t < room ? n_tokens - t : room;
+      LayerView lv = view(cache, layer);
+      if (launch_sink_append(lv, k_dev, v_dev, n_tokens, t, m, st) != cudaSuccess) return MIXKVQ_E_CUDA;
+      cache->launches += 1;
+      cache->n_sink[layer] += m;
+      t += m;
+      continue;
+    }
     if (cache->r[layer] == cache->R) {
       LayerView lv = view(cache, layer);
       if (launch_flush(lv, st) != cudaSuccess) return MIXKVQ_E_CUDA;
@@ -261,7 +279,7 @@ int mixkvq_decode_attention(mixkvq_cache* cache, int layer, const void* q_dev, f
     return MIXKVQ_E_INVALID_ARG;
   if (!aligned16(q_dev) || !aligned16(out_dev) || !aligned16(workspace_dev)) return MIXKVQ_E_ALIGNMENT;
   if (workspace_bytes_given < workspace_bytes(cache->S)) return MIXKVQ_E_BUFFER_TOO_SMALL;
-  if (cache->n_blocks[layer] == 0 && cache->r[layer] == 0) return MIXKVQ_E_EMPTY;
+  if (cache->n_blocks[layer] == 0 && cache->r[layer] == 0 && cache->n_sink[layer] == 0) return MIXKVQ_E_EMPTY;
   return run_attention(cache, layer, q_dev, out_dev, softmax_scale, static_cast<float*>(workspace_dev),
                        static_cast<cudaStream_t>(stream));
 }
@@ -274,11 +292,12 @@ int mixkvq_decode_step(mixkvq_cache* cache, int layer, const void* k_dev, const 
   if (!aligned16(k_dev) || !aligned16(v_dev) || !aligned16(q_dev) || !aligned16(out_dev) || !aligned16(workspace_dev))
     return MIXKVQ_E_ALIGNMENT;
   if (workspace_bytes_given < workspace_bytes(cache->S)) return MIXKVQ_E_BUFFER_TOO_SMALL;
-  const long long have = (long long)cache->n_blocks[layer] * cache->R + cache->r[layer];
+  const long long have = (long long)cache->n_sink[layer] + (long long)cache->n_blocks[layer] * cache->R + cache->r[layer];
   if (have + 1 > cache->cfg.max_tokens) return MIXKVQ_E_CAPACITY;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (cache->attn_kind != 0) {
-    // the comparison kernels do not take the new token themselves: plain append, then attention
+  if (cache->attn_kind != 0 || cache->n_sink[layer] < cache->cfg.sink_len) {
+    // the comparison kernels do not take the new token themselves, and a sink token is not a residual token:
+    // plain append, then attention
     int rc = mixkvq_quantize_append(cache, layer, k_dev, v_dev, q_dev, 1, stream);
     if (rc != MIXKVQ_OK) return rc;
     return run_attention(cache, layer, q_dev, out_dev, softmax_scale, static_cast<float*>(workspace_dev), st);
@@ -309,7 +328,7 @@ int mixkvq_decode_attention_noalloc(mixkvq_cache* cache, int layer, const void* 
   if (!cache || !q_dev || !out_dev || layer < 0 || layer >= cache->cfg.n_layers) return MIXKVQ_E_INVALID_ARG;
   if (!aligned16(q_dev) || !aligned16(out_dev)) return MIXKVQ_E_ALIGNMENT;
   if (cache->S > MIXKVQ_NOALLOC_MAX_STREAMS) return MIXKVQ_E_BUILTIN_SCRATCH;
-  if (cache->n_blocks[layer] == 0 && cache->r[layer] == 0) return MIXKVQ_E_EMPTY;
+  if (cache->n_blocks[layer] == 0 && cache->r[layer] == 0 && cache->n_sink[layer] == 0) return MIXKVQ_E_EMPTY;
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MIXKVQ_E_CUDA;
   if (!g_builtin_scratch_addr[dev]) {
@@ -352,6 +371,9 @@ int mixkvq_cache_describe(const mixkvq_cache* cache, int layer, mixkvq_layout_de
   out->n_streams = (uint32_t)cache->S;
   out->n_blocks = (uint32_t)cache->n_blocks[layer];
   out->residual_tokens = (uint32_t)cache->r[layer];
+  out->sink_off = L + cache->sink_off;     out->sink_stride = cache->sink_stride;
+  out->sink_tokens = (uint32_t)cache->n_sink[layer];
+  out->sink_len = (uint32_t)cache->cfg.sink_len;
   return MIXKVQ_OK;
 }
 

@@ -51,6 +51,28 @@ append_tokens_kernel(LayerView lv, const __nv_bfloat16* __restrict__ k, const __
   }
 }
 
+// Sink tokens: m rows of keys and of values go to sink slots n_sink .. n_sink + m - 1 of every stream, nothing else happens.
+__global__ void __launch_bounds__(256)
+sink_append_kernel(LayerView lv, const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __restrict__ v, int n_tokens,
+                   int t0, int m) {
+  const int s = blockIdx.x, tid = threadIdx.x;
+  const uint4* ksrc = reinterpret_cast<const uint4*>(k + ((size_t)s * n_tokens + t0) * kD);
+  const uint4* vsrc = reinterpret_cast<const uint4*>(v + ((size_t)s * n_tokens + t0) * kD);
+  uint4* kdst = reinterpret_cast<uint4*>(lv.sink + (size_t)s * lv.sink_stride) + (size_t)lv.n_sink * 16;
+  uint4* vdst = kdst + (size_t)lv.sink_len * 16;
+  for (int i = tid; i < m * 16; i += 256) {
+    kdst[i] = ksrc[i];
+    vdst[i] = vsrc[i];
+  }
+}
+
+cudaError_t launch_sink_append(const LayerView& lv, const void* k, const void* v, int n_tokens, int t0, int m,
+                               cudaStream_t stream) {
+  sink_append_kernel<<<lv.B * lv.Hkv, 256, 0, stream>>>(lv, static_cast<const __nv_bfloat16*>(k),
+                                                        static_cast<const __nv_bfloat16*>(v), n_tokens, t0, m);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_append(const LayerView& lv, const void* k, const void* v, const void* q, int n_tokens, int t0,
                           int m, cudaStream_t stream) {
   append_tokens_kernel<<<lv.B * lv.Hkv, 256, 0, stream>>>(

@@ -183,7 +183,9 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
 
   const int S = lv.B * lv.Hkv, U = lv.U, g = lv.g;
   const int packed_units = lv.n_blocks * U;
-  const int Us = packed_units + kResidualWeight * ((lv.r + 31) / 32);     // split positions; a residual unit spans several
+  // unquantized 32-token units: those of the residual window, then those of the sink
+  const int res_units = (lv.r + 31) / 32, bf16_units = res_units + (lv.n_sink + 31) / 32;
+  const int Us = packed_units + kResidualWeight * bf16_units;             // split positions; an unquantized unit spans several
   const long long total = (long long)Us * S;
   const long long cb = split_begin(total, gridDim.x, blockIdx.x), ce = split_begin(total, gridDim.x, blockIdx.x + 1);
 
@@ -650,16 +652,21 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
     // ring with ONE bulk copy, first the keys, then the values over them (small bulk copies are slow: a copy per row
     // cost tens of microseconds).  Value tiles are transposed on the way to registers with ldmatrix.trans.
     for (int ri = kWarps - 1 - warp; ri < n_res && !gave_up; ri += kWarps) {
-      const int x = packed_units + res_b + ri;
+      const int bu = res_b + ri;                        // unquantized unit: residual window first, then the sink
+      const bool in_sink = bu >= res_units;
+      const int wu = in_sink ? bu - res_units : bu;     // unit inside its window
+      const int rt = in_sink ? lv.n_sink : lv.r;        // tokens in that window
       const uint32_t rbar = smem_u32(&bars[kWarps * kStages + warp]);
-      const uint16_t* resk = reinterpret_cast<const uint16_t*>(lv.resk + (size_t)s * lv.resk_stride);
-      const uint16_t* resv = reinterpret_cast<const uint16_t*>(lv.resv + (size_t)s * lv.resv_stride);
+      const uint16_t* resk = reinterpret_cast<const uint16_t*>(in_sink ? lv.sink + (size_t)s * lv.sink_stride
+                                                                       : lv.resk + (size_t)s * lv.resk_stride);
+      const uint16_t* resv = reinterpret_cast<const uint16_t*>(in_sink ? lv.sink + (size_t)s * lv.sink_stride + (size_t)lv.sink_len * 256
+                                                                       : lv.resv + (size_t)s * lv.resv_stride);
       // fused decode step: the newest token (slot r - 1) is not in the residual store yet; the warp whose unit holds it
       // takes its rows from the step's tensors (into the staged tile and into the store) and updates the accumulator
       const int jn = lv.r - 1;
-      const bool holds_new = lv.new_k != nullptr && jn >= (x - packed_units) * 32 && jn < (x - packed_units) * 32 + 32;
+      const bool holds_new = !in_sink && lv.new_k != nullptr && jn >= wu * 32 && jn < wu * 32 + 32;
       {
-        const int j0s = (x - packed_units) * 32, nv = min(32, lv.r - j0s) - (holds_new ? 1 : 0);
+        const int j0s = wu * 32, nv = min(32, rt - j0s) - (holds_new ? 1 : 0);
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         if (nv > 0) {
           if (lane == 0) {
@@ -697,7 +704,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
           for (int j = 0; j < 4; ++j) O[ct][j] *= 1048576.0f;
         o_true_scale = true;
       }
-      const int j0 = (x - packed_units) * 32, rt = lv.r;
+      const int j0 = wu * 32;
       float Sx[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
       for (int kt = 0; kt < 8; ++kt) {
@@ -917,7 +924,7 @@ cudaError_t attention_mma_setup() {
 // Number of CTAs the split kernel runs for this layer state (also the number of partial-slot owners).
 // Split positions per stream: packed units plus the weighted units of the residual window.
 long long attention_mma_positions(const LayerView& lv) {
-  return (long long)lv.n_blocks * lv.U + (long long)kResidualWeight * ((lv.r + 31) / 32);
+  return (long long)lv.n_blocks * lv.U + (long long)kResidualWeight * ((lv.r + 31) / 32 + (lv.n_sink + 31) / 32);
 }
 
 // Number of CTAs the split kernel runs for this layer state (also the number of partial-slot owners).  When there are

@@ -26,7 +26,8 @@ attention_simt_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float s
   __syncthreads();
 
   const int packed_units = lv.n_blocks * lv.U;
-  const int units = packed_units + (lv.r + 31) / 32;
+  const int res_units = (lv.r + 31) / 32;                            // then the units of the sink
+  const int units = packed_units + res_units + (lv.n_sink + 31) / 32;
   const int ub = (int)split_begin(units, nsplit, split), ue = (int)split_begin(units, nsplit, split + 1);
   const int wb = ub + (int)split_begin(ue - ub, 4, warp), we = ub + (int)split_begin(ue - ub, 4, warp + 1);
 
@@ -35,6 +36,8 @@ attention_simt_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float s
   const uint32_t* table = reinterpret_cast<const uint32_t*>(lv.table + (size_t)s * lv.table_stride);
   const uint16_t* resk = reinterpret_cast<const uint16_t*>(lv.resk + (size_t)s * lv.resk_stride);
   const uint16_t* resv = reinterpret_cast<const uint16_t*>(lv.resv + (size_t)s * lv.resv_stride);
+  const uint16_t* sinkk = reinterpret_cast<const uint16_t*>(lv.sink + (size_t)s * lv.sink_stride);
+  const uint16_t* sinkv = sinkk + (size_t)lv.sink_len * kD;
 
   float m[8], l[8], o[8][4];
   for (int h = 0; h < 8; ++h) {
@@ -112,11 +115,14 @@ attention_simt_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float s
         for (int h = 0; h < 8; ++h) dot[h] = fmaf(qS[h][d], kval, dot[h]);
       }
     } else {
-      const int j = (unit - packed_units) * 32 + lane;
-      valid = j < lv.r;
+      const int bu = unit - packed_units;
+      const bool in_sink = bu >= res_units;
+      const int j = (in_sink ? bu - res_units : bu) * 32 + lane;
+      const uint16_t* rows = in_sink ? sinkk : resk;
+      valid = j < (in_sink ? lv.n_sink : lv.r);
       if (valid)
         for (int d = 0; d < kD; ++d) {
-          const float kval = bf16_bits_to_float(resk[(size_t)j * kD + d]);
+          const float kval = bf16_bits_to_float(rows[(size_t)j * kD + d]);
           for (int h = 0; h < 8; ++h) dot[h] = fmaf(qS[h][d], kval, dot[h]);
         }
     }
@@ -160,9 +166,12 @@ attention_simt_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float s
           vv[i] = fmaf((float)code, bf16_bits_to_float(mz & 0xFFFF), bf16_bits_to_float(mz >> 16));
         }
       } else {
-        const int j = (unit - packed_units) * 32 + jj;
+        const int bu = unit - packed_units;
+        const bool in_sink = bu >= res_units;
+        const int j = (in_sink ? bu - res_units : bu) * 32 + jj;
+        const uint16_t* rows = in_sink ? sinkv : resv;
         for (int i = 0; i < 4; ++i)
-          vv[i] = (j < lv.r) ? bf16_bits_to_float(resv[(size_t)j * kD + 4 * lane + i]) : 0.f;
+          vv[i] = (j < (in_sink ? lv.n_sink : lv.r)) ? bf16_bits_to_float(rows[(size_t)j * kD + 4 * lane + i]) : 0.f;
       }
       for (int h = 0; h < 8; ++h) {
         const float ph = __shfl_sync(0xffffffffu, p[h], jj);
@@ -202,7 +211,7 @@ attention_simt_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float s
 cudaError_t launch_attention_simt(const LayerView& lv, const void* q, float* out, float scale, float* ws, int n_sms,
                                   cudaStream_t stream, int* launches) {
   const int S = lv.B * lv.Hkv;
-  const int units = lv.n_blocks * lv.U + (lv.r + 31) / 32;
+  const int units = lv.n_blocks * lv.U + (lv.r + 31) / 32 + (lv.n_sink + 31) / 32;
   int nsplit = (4 * n_sms + S - 1) / S;
   nsplit = max(1, min(nsplit, min(units, kMaxCtas / S > 0 ? kMaxCtas / S : 1)));
   attention_simt_kernel<<<dim3(S, nsplit), 128, 0, stream>>>(lv, static_cast<const __nv_bfloat16*>(q),

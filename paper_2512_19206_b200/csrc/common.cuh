@@ -40,6 +40,8 @@ struct LayerView {
   char* resv;   uint64_t resv_stride;
   char* base;   uint64_t base_stride;
   char* extras; uint64_t extras_stride;
+  char* sink;   uint64_t sink_stride;   // per stream: keys [sink_len][128] bf16, then values
+  int sink_len, n_sink;       // capacity and current fill of the sink (same for all streams)
   uint32_t* status;           // sticky device status word
   // fused decode step: the new token's key and value rows [S][128] (bf16 bits); null for plain attention.
   // The attention kernel then stores them at residual slot r - 1 and adds |q| to the importance accumulator itself.
@@ -171,6 +173,8 @@ __host__ __device__ inline long long split_begin(long long total, int parts, int
 namespace mixkvq {
 cudaError_t launch_append(const LayerView& lv, const void* k, const void* v, const void* q, int n_tokens, int t0,
                           int m, cudaStream_t stream);
+cudaError_t launch_sink_append(const LayerView& lv, const void* k, const void* v, int n_tokens, int t0, int m,
+                               cudaStream_t stream);
 cudaError_t launch_flush(const LayerView& lv, cudaStream_t stream);
 cudaError_t launch_flush_bulk(const LayerView& lv, const void* k, const void* v, const void* q, int n_tokens, int t0,
                               int nb, cudaStream_t stream);

@@ -28,8 +28,8 @@ def test_library_exports_every_declared_symbol(binding):
 
 
 def test_config_struct_matches_header(binding):
-    assert C.sizeof(binding.Config) == 72          # 14 int32/float fields, one uint64, the two budgets
-    assert C.sizeof(binding.LayoutDesc) == 13 * 8 + 4 * 4
+    assert C.sizeof(binding.Config) == 80          # 14 int32/float fields, one uint64, two budgets, sink length, pad
+    assert C.sizeof(binding.LayoutDesc) == 13 * 8 + 4 * 4 + 2 * 8 + 2 * 4
 
 
 def test_cache_bytes_and_argument_validation(binding):

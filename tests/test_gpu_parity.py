@@ -202,6 +202,47 @@ def test_fixed_budget_tiering(binding, layout, k16, k4):
     assert cache.status() == 0
 
 
+@pytest.mark.parametrize("kind,layout", [(0, 0), (1, 0), (0, 1)])
+@pytest.mark.parametrize("tokens", [20, 37, 32 + 2 * 128 + 17])
+def test_sink_tokens(binding, kind, layout, tokens):
+    # the first 32 tokens stay in bf16 outside the residual window, the scoring and the blocks; attention sees them
+    w = small("qwen7b", batch=2, tokens=tokens, **W.P27)
+    k, v, q = W.tokens(w, 0, 0, tokens)
+    cache = U.make_cache(binding, w, layout=layout, sink_len=32)
+    cache.quantize_append(0, k.cuda(), v.cuda(), q.cuda())
+    cache.set_attention_kernel(kind)
+    orc = U.oracle_streams(w, 0, k, v, q, sink_len=32)
+    U.compare_regions(cache, 0, w, orc)
+    d = cache.describe(0)
+    assert d.sink_tokens == min(tokens, 32) and d.n_blocks * 128 + d.residual_tokens == max(tokens - 32, 0)
+    qd = W.decode_query(w, 0, 0)
+    out = cache.decode_attention(0, qd.cuda(), W.softmax_scale())
+    assert U.max_abs_err(w, out, U.oracle_attention(w, orc, qd)) <= ATTN_TOL
+    assert cache.status() == 0
+
+
+@pytest.mark.parametrize("kind", [0, 1])
+def test_decode_steps_through_the_sink(binding, kind):
+    # decode steps from a short prompt: the sink fills first (plain append + attention), then the fused step takes over
+    w = small("qwen7b", batch=1, tokens=10 + 60, **W.P24)
+    k, v, q = W.tokens(w, 0, 0, w.tokens)
+    kc, vc, qc = k.cuda(), v.cuda(), q.cuda()
+    cache = U.make_cache(binding, w, sink_len=32)
+    cache.set_attention_kernel(kind)
+    cache.quantize_append(0, kc[:, :, :10].contiguous(), vc[:, :, :10].contiguous(), qc[:, :, :10].contiguous())
+    orc = U.oracle_streams(w, 0, k[:, :, :10], v[:, :, :10], q[:, :, :10], sink_len=32)
+    for t in range(10, w.tokens):
+        out = cache.decode_step(0, kc[:, :, t:t + 1].contiguous(), vc[:, :, t:t + 1].contiguous(),
+                                qc[:, :, t:t + 1].contiguous(), W.softmax_scale())
+        for (b, hk), st in orc.items():
+            st.append(U.f32(k[b, hk, t]), U.f32(v[b, hk, t]), U.f32(q[b, hk * w.g:(hk + 1) * w.g, t]))
+        if t in (10, 31, 32, 33, 69):
+            qd = q[:, :, t]
+            assert U.max_abs_err(w, out, U.oracle_attention(w, orc, qd)) <= ATTN_TOL, t
+    U.compare_regions(cache, 0, w, orc)
+    assert cache.status() == 0
+
+
 # ------------------------------------------------------------------------------------------- attention
 @pytest.mark.parametrize("kind,layout", [(0, 0), (1, 0), (0, 1), (1, 1)])
 @pytest.mark.parametrize("name,tokens,preset", [

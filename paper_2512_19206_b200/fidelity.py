@@ -54,7 +54,8 @@ def reference_attention(k: torch.Tensor, v: torch.Tensor, q: torch.Tensor, scale
 
 
 def measure(w: "W.Workload", tau_bf16: float, tau_u4: float, score_bits: int = 2, importance_mode: int = 0,
-            n_queries: int = 4, chunk: int = 4096, return_outputs: bool = False):
+            n_queries: int = 4, chunk: int = 4096, return_outputs: bool = False, budget_bf16: int = 0, budget_u4: int = 0,
+            sink_len: int = 0):
     """Builds one layer of the workload with the given thresholds and returns (B_eff, n16, n4, max error, rms error)
     of decode attention against the unquantized reference, over n_queries decode queries (and, on request, the
     attention outputs themselves)."""
@@ -63,7 +64,8 @@ def measure(w: "W.Workload", tau_bf16: float, tau_u4: float, score_bits: int = 2
     budget = n_blocks * ((w.residual_len // 32) * (128 * 64 + 1024) + 512)
     cfg = B.make_config(1, w.batch, w.n_q_heads, w.n_kv_heads, w.tokens + 2 * w.residual_len,
                         residual_len=w.residual_len, group_size=w.group_size, tau_bf16=tau_bf16, tau_u4=tau_u4,
-                        score_bits=score_bits, importance_mode=importance_mode, extras_budget_bytes=budget)
+                        score_bits=score_bits, importance_mode=importance_mode, extras_budget_bytes=budget,
+                        budget_bf16=budget_bf16, budget_u4=budget_u4, sink_len=sink_len)
     cache = B.Cache(cfg)
     ks, vs = [], []
     t = 0
@@ -101,9 +103,10 @@ def sweep(w: "W.Workload", pairs, **kw):
     the error that the key tiers control."""
     *_, keys_bf16 = measure(w, -1.0, -1.0, return_outputs=True, **kw)
     rows = []
-    for name, tau_bf16, tau_u4, score_bits, mode in pairs:
+    for name, tau_bf16, tau_u4, score_bits, mode, *extra in pairs:
+        more = extra[0] if extra else {}
         beff, n16, n4, worst, rms, outs = measure(w, tau_bf16, tau_u4, score_bits=score_bits, importance_mode=mode,
-                                                  return_outputs=True, **kw)
+                                                  return_outputs=True, **more, **kw)
         sq = sum(float(((a - b).double() ** 2).sum()) for a, b in zip(outs, keys_bf16))
         key_rms = math.sqrt(sq / sum(a.numel() for a in outs))
         rows.append({"setting": name, "tau_bf16": tau_bf16, "tau_u4": tau_u4, "importance_mode": mode,
@@ -112,13 +115,16 @@ def sweep(w: "W.Workload", pairs, **kw):
 
 
 def default_pairs():
-    """(name, tau_bf16, tau_u4, score_bits, importance_mode): uniform 2-bit, a sweep of the BF16 threshold, the two
+    """(name, tau_bf16, tau_u4, score_bits, importance_mode[, further configuration fields]): uniform 2-bit, a sweep of the BF16 threshold, the two
     presets with a UINT4 tier, the error-only ablation at the first preset's threshold, and unquantized keys."""
     inf = 1e30
     pairs = [("uniform 2-bit keys", inf, inf, 2, 0)]
     pairs += [(f"two tiers, tau_bf16 = {t:g}", t, inf, 2, 0) for t in (13.0, 6.5, 3.25)]
     pairs += [("three tiers (6.5, 4.0)", 6.5, 4.0, 2, 0), ("three tiers (6.5, 2.0)", 6.5, 2.0, 2, 0)]
     pairs += [("error-only salience, tau_bf16 = 6.5", 6.5, inf, 2, 2)]
+    pairs += [("fixed budget: 4 BF16", inf, inf, 2, 0, {"budget_bf16": 4}),
+              ("fixed budget: 4 BF16 + 24 UINT4", inf, inf, 2, 0, {"budget_bf16": 4, "budget_u4": 24}),
+              ("two tiers (6.5) + 32 sink tokens", 6.5, inf, 2, 0, {"sink_len": 32})]
     pairs += [("4-bit base (2.17)", W.P4BASE["tau_bf16"], -1.0, 4, 0), ("all keys bf16 (values 2-bit)", -1.0, -1.0, 2, 0)]
     return pairs
 

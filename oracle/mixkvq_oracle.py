@@ -179,7 +179,7 @@ class Block:
 
 class OracleStream:
     def __init__(self, g, R=128, G=32, score_bits=2, tau_bf16=1e30, tau_u4=1e30, importance_mode=0, budget_bf16=0,
-                 budget_u4=0, sink_len=0):
+                 budget_u4=0, sink_len=0, v_bits=2):
         assert R % 32 == 0 and R % G == 0 and D % G == 0
         self.g, self.R, self.G = g, R, G
         self.score_bits, self.tau_bf16, self.tau_u4 = score_bits, tau_bf16, tau_u4
@@ -189,6 +189,8 @@ class OracleStream:
         # the sequence stay in full precision for good; they never enter the residual window, the importance
         # accumulator or a quantized block
         self.sink_len = sink_len
+        assert v_bits in (2, 4)
+        self.v_bits = v_bits               # values: 2 bits per token-group code (Section 4.2), or 4
         self.sinkK = np.zeros((sink_len, D), np.float32)
         self.sinkV = np.zeros((sink_len, D), np.float32)
         self.n_sink = 0
@@ -266,7 +268,7 @@ class OracleStream:
             blk.kcodes[:, sel] = c.reshape(D, R).T[:, sel]
             blk.ks[:, sel], blk.kz[:, sel] = s.T[:, sel], z.T[:, sel]
         V = self.resV.reshape(R, D // G, G)                    # G consecutive channels of a token
-        c, s, z = quantize_groups(V, 2)
+        c, s, z = quantize_groups(V, self.v_bits)
         blk.vcodes, blk.vs, blk.vz = c.reshape(R, D), s, z
         self.blocks.append(blk)
         self.r = 0
@@ -327,8 +329,14 @@ def unquantized_attention(q, K, V, scale):
 # byte layout (one element at a time, from the stated position formulas)
 # fragment layout (the default): blocks of any R
 # --------------------------------------------------------------------------------------------
-def base_bytes(R, G):
-    return (R // G) * 512 + (R // 32) * (2048 + 128 * (D // G))
+def unit_bytes_of(G, v_bits=2):
+    """One 32-token unit: key low plane 1024, value low plane 1024, value scales and zero-points, and with 4-bit values the
+    value high plane (codes >> 2, in the low plane's bit positions) 1024."""
+    return 2048 + 128 * (D // G) + (1024 if v_bits == 4 else 0)
+
+
+def base_bytes(R, G, v_bits=2):
+    return (R // G) * 512 + (R // 32) * unit_bytes_of(G, v_bits)
 
 
 def dense_high_plane(tau_u4):
@@ -409,15 +417,15 @@ def _scatter_codes(words, word_idx, bit_idx, codes):
     np.add.at(words, word_idx.ravel(), (codes.astype(np.uint32) << bit_idx.astype(np.uint32)).ravel())
 
 
-def pack_base(blk: Block, R, G):
+def pack_base(blk: Block, R, G, v_bits=2):
     NG, U, VG = R // G, R // 32, D // G
     kw, kb, vw, vb, _, _ = _tables()
-    words = np.zeros(base_bytes(R, G) // 4, np.uint32)
+    words = np.zeros(base_bytes(R, G, v_bits) // 4, np.uint32)
     quant = blk.tiers != TIER_BF16
     # K meta: entry (kg, d) at kg*512 + d*4 = {s, z}
     ks16 = np.where(quant[None, :], bf16_to_u16(blk.ks), 0).astype(np.uint32)
     kz16 = np.where(quant[None, :], bf16_to_u16(blk.kz), 0).astype(np.uint32)
-    unit_bytes = 2048 + 128 * VG
+    unit_bytes = unit_bytes_of(G, v_bits)
     meta = ks16 | (kz16 << 16)                                   # entry (kg, d) at frag_meta_off(kg) + d*4
     for kg in range(NG):
         mo = frag_meta_off(kg, G, unit_bytes) // 4
@@ -428,8 +436,10 @@ def pack_base(blk: Block, R, G):
         ubase = frag_unit_off(u, G, unit_bytes) // 4
         sl = slice(32 * u, 32 * u + 32)
         _scatter_codes(words, ubase + kw, kb, klow[sl])
-        _scatter_codes(words, ubase + 256 + vw, vb, blk.vcodes[sl])
+        _scatter_codes(words, ubase + 256 + vw, vb, blk.vcodes[sl] & 3)
         words[ubase + 512:ubase + 512 + 32 * VG] = (vs16[sl] | (vz16[sl] << 16)).reshape(32 * VG)
+        if v_bits == 4:
+            _scatter_codes(words, ubase + 512 + 32 * VG + vw, vb, blk.vcodes[sl] >> 2)
     return words.astype("<u4").tobytes()
 
 
@@ -477,14 +487,14 @@ def pack_extras(blk: Block, R, dense=False):
     return bytes(head) + words.astype("<u4").tobytes(), n16, n4
 
 
-def unpack_base(buf, R, G):
+def unpack_base(buf, R, G, v_bits=2):
     """Inverse of pack_base for the code planes and the metadata, element by element."""
     NG, U, VG = R // G, R // 32, D // G
     words = np.frombuffer(buf, dtype="<u4")
     halves = np.frombuffer(buf, dtype="<u2")
     ks = np.zeros((NG, D), np.float32)
     kz = np.zeros((NG, D), np.float32)
-    unit_bytes = 2048 + 128 * VG
+    unit_bytes = unit_bytes_of(G, v_bits)
     for kg in range(NG):
         for d in range(D):
             ks[kg, d] = u16_to_bf16(halves[(frag_meta_off(kg, G, unit_bytes) + d * 4) // 2])
@@ -502,6 +512,8 @@ def unpack_base(buf, R, G):
                 klow[j, d] = (int(words[(ubase + off) // 4]) >> bit) & 3
                 off, bit = _v_code_pos(jj, d)
                 vcodes[j, d] = (int(words[(ubase + 1024 + off) // 4]) >> bit) & 3
+                if v_bits == 4:
+                    vcodes[j, d] |= ((int(words[(ubase + 2048 + 128 * VG + off) // 4]) >> bit) & 3) << 2
             for vg in range(VG):
                 o = (ubase + 2048 + (jj * VG + vg) * 4) // 2
                 vs[j, vg] = u16_to_bf16(halves[o])
@@ -622,13 +634,13 @@ def pack_stream(st: OracleStream, layout=LAYOUT_FRAGMENT):
     base, table, extras = [], [], []
     used16 = 0
     tile = layout == LAYOUT_TILE
-    assert not tile or st.R == 128
+    assert not tile or (st.R == 128 and st.v_bits == 2)
     for blk in st.blocks:
         if tile:
             base.append(pack_base_tile(blk, st.G))
             ex, n16, n4 = pack_extras_tile(blk)
         else:
-            base.append(pack_base(blk, st.R, st.G))
+            base.append(pack_base(blk, st.R, st.G, st.v_bits))
             ex, n16, n4 = pack_extras(blk, st.R, dense_high_plane(st.tau_u4) and st.budget_bf16 + st.budget_u4 == 0)
         table.append(table_entry(used16, n16, n4))
         extras.append(ex)

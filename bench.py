@@ -202,13 +202,13 @@ def measured_traffic(kernel, source_file, group_size, tokens_packed, streams):
     return ent["dram_bytes_per_token_per_kv_head"] * tokens_packed * streams
 
 
-def algorithmic_bytes_per_layer(w, n16, n4, r, tokens_packed, n_partials):
+def algorithmic_bytes_per_layer(w, n16, n4, r, tokens_packed, n_partials, v_bits=2):
     """Bytes the method must move for one decode-attention launch (one layer): packed keys and values with
     their scales/zeros, promoted channels, residual window, q, o and the split partials."""
     G, R, D, g = w.group_size, w.residual_len, 128, w.g
     n2 = D - n16 - n4
     k_tok = 2 * n16 + n4 / 2 + n2 / 4 + 4 * (n4 + n2) / G + 160 / R
-    v_tok = D * 2 / 8 + 4 * D / G
+    v_tok = D * v_bits / 8 + 4 * D / G
     streams = w.batch * w.n_kv_heads
     per_stream = tokens_packed * (k_tok + v_tok) + 2 * r * D * 2 + g * D * 2 + g * D * 4
     return streams * per_stream + 2 * n_partials * g * (D + 2) * 4
@@ -233,7 +233,7 @@ def run_gpu(args, w):
     cfg = binding.make_config(w.n_layers, w.batch, w.n_q_heads, w.n_kv_heads, w.tokens + n_steps + 2 * w.residual_len,
                               residual_len=w.residual_len, group_size=w.group_size, tau_bf16=w.tau_bf16,
                               tau_u4=w.tau_u4, score_bits=w.score_bits, block_layout=args.layout,
-                              importance_mode=args.importance_mode, sink_len=args.sink_len,
+                              importance_mode=args.importance_mode, sink_len=args.sink_len, v_bits=args.v_bits,
                               extras_budget_bytes=((w.tokens + n_steps) // w.residual_len + 3) * 8192 if w.score_bits == 4 else 0)
     cache = binding.Cache(cfg, device=dev)
     prefill_ms = prefill(cache, w, dev)
@@ -354,7 +354,7 @@ def run_gpu(args, w):
     n_sms = torch.cuda.get_device_properties(dev).multi_processor_count
     n_part = min(2 * n_sms, units)
     n_part = n_part // streams * streams if n_part > streams else n_part + streams
-    alg = algorithmic_bytes_per_layer(w, n16, n4, d0.residual_tokens, tokens_packed, n_part)
+    alg = algorithmic_bytes_per_layer(w, n16, n4, d0.residual_tokens, tokens_packed, n_part, args.v_bits)
     peak, peak_src = measured_peaks()
     achieved = alg / (kern_ms * 1e-3) / 1e9
     line = {
@@ -373,7 +373,7 @@ def run_gpu(args, w):
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal_8TBs": achieved / 8000.0,
                      # the committed counters were taken on the two-tier mix (no UINT4 tier): other mixes have none
-                     "traffic": None if w.tau_u4 < w.tau_bf16 else measured_traffic(
+                     "traffic": None if (w.tau_u4 < w.tau_bf16 or args.v_bits != 2 or args.sink_len) else measured_traffic(
                          *(("attention_tc_kernel", "attention_tc.cu") if args.layout == 1 else
                            ("attention_mma_kernel", "attention_mma.cu")), w.group_size, tokens_packed,
                          w.batch * w.n_kv_heads),
@@ -406,6 +406,7 @@ def main():
     ap.add_argument("--importance-mode", type=int, default=0, choices=[0, 1, 2],
                     help="0: window importance (default), 1: cumulative, 2: error-only salience")
     ap.add_argument("--sink-len", type=int, default=0, help="sink tokens kept in bf16 (0, or a multiple of 32 up to 256)")
+    ap.add_argument("--v-bits", type=int, default=2, choices=[2, 4], help="value bit-width (4: fragment layout only)")
     ap.add_argument("--tokens", type=int, default=None)
     ap.add_argument("--layers", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

@@ -36,7 +36,7 @@ extern "C" {
 enum {
   MIXKVQ_OK = 0,
   MIXKVQ_E_INVALID_ARG = -1,          /* null pointer, bad dimension, layer out of range            */
-  MIXKVQ_E_UNSUPPORTED = -2,          /* head_dim != 128, v_bits != 2, unsupported R, G or layout    */
+  MIXKVQ_E_UNSUPPORTED = -2,          /* head_dim != 128, v_bits not 2 or 4, unsupported R, G or layout */
   MIXKVQ_E_ALIGNMENT = -3,            /* a device pointer is not 16-byte aligned                     */
   MIXKVQ_E_BUFFER_TOO_SMALL = -4,     /* cache memory or attention workspace smaller than required   */
   MIXKVQ_E_CAPACITY = -5,             /* append would exceed max_tokens                              */
@@ -62,7 +62,8 @@ typedef struct mixkvq_config {
   int32_t max_tokens;                 /* capacity per sequence                                       */
   int32_t residual_len;               /* R (Section 5.1: 128): multiple of 32, <= 256, multiple of G */
   int32_t group_size;                 /* G (Section 5.1: 32): 32, 64 or 128                          */
-  int32_t v_bits;                     /* value bit-width, must be 2 (Section 4.2)                    */
+  int32_t v_bits;                     /* value bit-width: 2 (Section 4.2), or 4 (fragment layout only; stored as
+                                         two 2-bit planes, the value scale must then stay below 2^7)  */
   int32_t score_bits;                 /* B of the sensitivity score S_d (Section 4.2), 2 or 4        */
   float tau_bf16;                     /* A_d >  tau_bf16            -> BF16                          */
   float tau_u4;                       /* tau_u4 < A_d <= tau_bf16   -> UINT4, else UINT2             */

@@ -106,8 +106,8 @@ def _ptr(t: torch.Tensor | None):
 
 def make_config(n_layers, batch, n_q_heads, n_kv_heads, max_tokens, residual_len=128, group_size=32,
                 tau_bf16=1e30, tau_u4=1e30, score_bits=2, importance_mode=0, extras_budget_bytes=0,
-                block_layout=0, budget_bf16=0, budget_u4=0, sink_len=0) -> Config:
-    return Config(n_layers, batch, n_q_heads, n_kv_heads, 128, max_tokens, residual_len, group_size, 2, score_bits,
+                block_layout=0, budget_bf16=0, budget_u4=0, sink_len=0, v_bits=2) -> Config:
+    return Config(n_layers, batch, n_q_heads, n_kv_heads, 128, max_tokens, residual_len, group_size, v_bits, score_bits,
                   tau_bf16, tau_u4, importance_mode, block_layout, extras_budget_bytes, budget_bf16, budget_u4,
                   sink_len, 0)
 

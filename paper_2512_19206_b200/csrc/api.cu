@@ -34,7 +34,8 @@ int check_config(const mixkvq_config* c) {
   if (c->n_layers < 1 || c->batch < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1 || c->max_tokens < 1)
     return MIXKVQ_E_INVALID_ARG;
   if (c->n_q_heads % c->n_kv_heads != 0) return MIXKVQ_E_INVALID_ARG;
-  if (c->head_dim != kD || c->v_bits != 2) return MIXKVQ_E_UNSUPPORTED;
+  if (c->head_dim != kD || (c->v_bits != 2 && c->v_bits != 4)) return MIXKVQ_E_UNSUPPORTED;
+  if (c->v_bits == 4 && c->block_layout != 0) return MIXKVQ_E_UNSUPPORTED;      // the tile layout holds 2-bit values only
   if (c->n_q_heads / c->n_kv_heads > 8) return MIXKVQ_E_UNSUPPORTED;
   if (c->group_size != 32 && c->group_size != 64 && c->group_size != 128) return MIXKVQ_E_UNSUPPORTED;
   if (c->residual_len < 32 || c->residual_len > 256 || c->residual_len % 32 != 0 ||
@@ -60,7 +61,7 @@ uint64_t plan(const mixkvq_config* c, mixkvq_cache* h) {
   h->NG = h->R / h->G;
   h->VG = kD / h->G;
   h->max_blocks = (c->max_tokens + h->R - 1) / h->R;
-  h->unit_bytes = 2048u + 128u * h->VG;
+  h->unit_bytes = 2048u + 128u * h->VG + (c->v_bits == 4 ? 1024u : 0u);
   h->tile = (c->block_layout == 1) ? 1 : 0;
   h->base_bytes = h->tile ? (uint32_t)h->NG * 512u + 8192u + 512u * (uint32_t)h->VG
                           : (uint32_t)h->NG * 512u + (uint32_t)h->U * h->unit_bytes;
@@ -95,6 +96,7 @@ LayerView view(const mixkvq_cache* h, int layer) {
   v.n_blocks = h->n_blocks[layer]; v.r = h->r[layer];
   v.tile = h->tile;
   v.budget_bf16 = h->cfg.budget_bf16; v.budget_u4 = h->cfg.budget_u4;
+  v.v_bits = h->cfg.v_bits;
   v.dense_hi = (h->cfg.tau_u4 < 0.0f && v.budget_bf16 + v.budget_u4 == 0) ? 1 : 0;
   v.base_bytes = h->base_bytes; v.unit_bytes = h->unit_bytes;
   v.extras_budget = h->extras_budget;

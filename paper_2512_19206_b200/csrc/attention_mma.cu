@@ -27,13 +27,14 @@ namespace {
 
 constexpr int kWarps = 6;
 constexpr int kStages = 3;
-constexpr int kStageBytes = 3072;            // one key-meta group (512 B) followed by the unit (<= 2560 B), as in the block
+// one ring stage: a key-meta group (512 B) followed by the unit (<= 2560 B; <= 3584 B with 4-bit values), as in the block
+__host__ __device__ constexpr int stage_bytes(bool v4) { return v4 ? 4096 : 3072; }
 constexpr int kKeyMetaOff = 0;
 constexpr int kUnitOff = 512;
 constexpr int kPrepBytes = 2560;             // kprep 576 | zprep 576 | svp 320 | zvp 1088
 constexpr int kBarBytes = 256;                 // mbarriers: a ring per warp and one more per warp for the residual window
 constexpr int kSharedTail = kBarBytes + 2048 + 2048 + 2 * kWarps * 32;
-constexpr int kSmemBytes = kWarps * (kStages * kStageBytes + kPrepBytes) + kSharedTail;
+__host__ __device__ constexpr int smem_bytes(bool v4) { return kWarps * (kStages * stage_bytes(v4) + kPrepBytes) + kSharedTail; }
 constexpr int kCtasPerSm = 2;
 constexpr int kCtasPerSmDense = 2;           // with a 4-bit base two key planes are in flight: more registers per thread, fewer CTAs
 static_assert((kWarps * kStages + kWarps) * 8 <= kBarBytes, "the mbarrier area at the start of the shared tail is too small");
@@ -133,12 +134,14 @@ __device__ __forceinline__ uint32_t key_shift(uint32_t w, int kt) { return kt < 
 
 // kU4: how the configuration can use the UINT4 tier: 0 = never (tau_u4 >= tau_bf16), 1 = some channels (high plane stored
 // per channel pair, gathered), 2 = 4-bit base (dense high plane)
-template <int G, int kU4>
+// kV4: 4-bit values (a second plane of 2-bit value codes per unit, scale 4 s_v)
+template <int G, int kU4, bool kV4>
 __global__ void __launch_bounds__(kWarps * 32, kU4 == 2 ? kCtasPerSmDense : kCtasPerSm)
 attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float scale_log2e, float* __restrict__ ws,
                      uint32_t four2) {
   constexpr int VG = kD / G;              // value groups per token
   constexpr int TPG = 8 / VG;             // 16-channel tiles per value group
+  constexpr int kStageBytes = stage_bytes(kV4);
   extern __shared__ __align__(128) unsigned char smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, r = lane >> 2, t = lane & 3;
 
@@ -178,7 +181,8 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
   const float pv_up = __uint_as_float((131u - 2u * (uint32_t)(lane >> 3)) << 23);          // 2^(4 - 2 * (2 ks + ch))
   const int pv_sv = ((((lane & 7) >> 1) * 20 + (lane >> 3)) * 2) + (lane & 1);             // svp half index of group 0
   const int pv_zv = (((lane >> 4) * 144 + ((lane & 7) >> 1) * 4 + 2 * ((lane >> 3) & 1)) * 2) + (lane & 1);   // zvp half index of group 0
-  constexpr uint32_t kUnitBytes = 2048u + 128u * (kD / G);   // codes of 32 tokens: keys 1024, values 1024, value scales
+  // codes of 32 tokens: keys 1024, values 1024, value scales (and the values' high plane 1024)
+  constexpr uint32_t kUnitBytes = 2048u + 128u * (kD / G) + (kV4 ? 1024u : 0u);
   constexpr int UPG = G / 32;                                 // units per key group
 
   const int S = lv.B * lv.Hkv, U = lv.U, g = lv.g;
@@ -618,6 +622,28 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
           }
         }
       }
+      // ---- 4-bit values: the high plane (codes >> 2, the low plane's bit order) with four times the scale
+      if constexpr (kV4) {
+        const uint4 vw0 = reinterpret_cast<const uint4*>(st + 2048 + 128 * VG)[lane];
+        const uint4 vw1 = reinterpret_cast<const uint4*>(st + 2048 + 128 * VG)[32 + lane];
+        const uint32_t vw[8] = {vw0.x, vw0.y, vw0.z, vw0.w, vw1.x, vw1.y, vw1.z, vw1.w};
+#pragma unroll
+        for (int vg = 0; vg < VG; ++vg) {
+          const uint4 sv = *reinterpret_cast<const uint4*>(&svp[t * 20 + vg * 4]);
+          const uint32_t Bp[2][2] = {{hmul2_u(hmul2_u(Pt[0][0], sv.x), four2), hmul2_u(hmul2_u(Pt[0][1], sv.y), four2)},
+                                     {hmul2_u(hmul2_u(Pt[1][0], sv.z), four2), hmul2_u(hmul2_u(Pt[1][1], sv.w), four2)}};
+#pragma unroll
+          for (int c = 0; c < TPG; ++c) {
+            const int ct = vg * TPG + c;
+            const uint32_t x0 = vw[ct], x1 = vw[ct] >> 8;
+#pragma unroll
+            for (int ks = 0; ks < 2; ++ks) {
+              const uint32_t mk0 = 0x00030003u << (4 * ks), mk1 = 0x00030003u << (4 * ks + 2);
+              mma_f16(O[ct], x0 & mk0, x1 & mk0, x0 & mk1, x1 & mk1, Bp[ks][0], Bp[ks][1]);
+            }
+          }
+        }
+      }
 
       // ---- release the stage and refill it, then move on to the next unit
       __syncwarp();
@@ -868,20 +894,25 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
   }
 }
 
-template <int G, int kU4>
-cudaError_t launch_one(const LayerView& lv, const __nv_bfloat16* qb, float sl, float* ws, int grid, cudaStream_t stream) {
+template <int G, int kU4, bool kV4>
+cudaError_t launch_v(const LayerView& lv, const __nv_bfloat16* qb, float sl, float* ws, int grid, cudaStream_t stream) {
   // launched with programmatic stream serialization: the kernel itself waits for its predecessor (griddepcontrol.wait)
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)grid);
   cfg.blockDim = dim3(kWarps * 32);
-  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.dynamicSmemBytes = smem_bytes(kV4);
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, attention_mma_kernel<G, kU4>, lv, qb, sl, ws, 0x44004400u);
+  return cudaLaunchKernelEx(&cfg, attention_mma_kernel<G, kU4, kV4>, lv, qb, sl, ws, 0x44004400u);
+}
+template <int G, int kU4>
+cudaError_t launch_one(const LayerView& lv, const __nv_bfloat16* qb, float sl, float* ws, int grid, cudaStream_t stream) {
+  return lv.v_bits == 4 ? launch_v<G, kU4, true>(lv, qb, sl, ws, grid, stream)
+                        : launch_v<G, kU4, false>(lv, qb, sl, ws, grid, stream);
 }
 
 template <int G>
@@ -896,14 +927,19 @@ cudaError_t launch_g(const LayerView& lv, const void* q, float scale, float* ws,
 
 }  // namespace
 
+template <int G, int kU4, bool kV4>
+static cudaError_t setup_v() {
+  cudaError_t e = cudaFuncSetAttribute(attention_mma_kernel<G, kU4, kV4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       smem_bytes(kV4));
+  if (e != cudaSuccess) return e;
+  // the CTAs of an SM only fit with the largest shared-memory carve-out; ask for it explicitly
+  return cudaFuncSetAttribute(attention_mma_kernel<G, kU4, kV4>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                              (int)cudaSharedmemCarveoutMaxShared);
+}
 template <int G, int kU4>
 static cudaError_t setup_one() {
-  cudaError_t e = cudaFuncSetAttribute(attention_mma_kernel<G, kU4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       kSmemBytes);
-  if (e != cudaSuccess) return e;
-  // kCtasPerSm CTAs only fit with the largest shared-memory carve-out; ask for it explicitly
-  return cudaFuncSetAttribute(attention_mma_kernel<G, kU4>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                              (int)cudaSharedmemCarveoutMaxShared);
+  cudaError_t e = setup_v<G, kU4, false>();
+  return e != cudaSuccess ? e : setup_v<G, kU4, true>();
 }
 template <int G>
 static cudaError_t setup_g() {

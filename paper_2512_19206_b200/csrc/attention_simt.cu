@@ -161,6 +161,8 @@ attention_simt_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float s
             int word, bit;
             v_code_pos(jj, c, &word, &bit);
             code = (vcodes[word] >> bit) & 3;
+            if (lv.v_bits == 4)      // the high plane follows the value scales
+              code |= ((reinterpret_cast<const uint32_t*>(ub_ptr + 2048 + 128 * lv.VG)[word] >> bit) & 3) << 2;
             mz = vmeta[jj * lv.VG + c / lv.G];
           }
           vv[i] = fmaf((float)code, bf16_bits_to_float(mz & 0xFFFF), bf16_bits_to_float(mz >> 16));

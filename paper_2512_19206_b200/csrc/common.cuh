@@ -32,6 +32,7 @@ struct LayerView {
   // method parameters
   int score_bits, importance_mode;
   float tau_bf16, tau_u4;
+  int v_bits;                 // 2, or 4: a second plane of 2-bit value codes follows the value scales in every unit
   int budget_bf16, budget_u4; // fixed-budget tiering when their sum is positive (the thresholds are then unused)
   // per-stream arrays (base pointer + stride in bytes)
   char* state;  uint64_t state_stride;

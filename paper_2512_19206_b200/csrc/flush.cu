@@ -443,11 +443,12 @@ flush_kernel(LayerView lv, BulkSrc src) {
         gmx = fmaxf(gmx, __shfl_xor_sync(0xffffffffu, gmx, off));
         gmn = fminf(gmn, __shfl_xor_sync(0xffffffffu, gmn, off));
       }
-      const float sc = stored_scale(gmx, gmn, 3.0f);
+      const int vmax = lv.v_bits == 4 ? 15 : 3;
+      const float sc = stored_scale(gmx, gmn, (float)vmax);
       const float rs = __frcp_rn(sc);
       uint32_t codes = 0;
 #pragma unroll
-      for (int k = 0; k < 4; ++k) codes |= (uint32_t)quant_code_fast(x[k], gmn, sc, rs, 3) << (8 * k);
+      for (int k = 0; k < 4; ++k) codes |= (uint32_t)quant_code_fast(x[k], gmn, sc, rs, vmax) << (8 * k);
       *reinterpret_cast<uint32_t*>(&cS[j * kD + 4 * lane]) = codes;
       if ((4 * lane) % G == 0)
         vmeta_of(j)[(4 * lane) / G] = float_to_bf16_bits_exact(sc) | (float_to_bf16_bits_exact(gmn) << 16);
@@ -482,9 +483,29 @@ flush_kernel(LayerView lv, BulkSrc src) {
             for (int e = 0; e < 2; ++e) {
               const int c = ct * 16 + rh * 8 + r;
               const int j = 32 * u + ks * 16 + ch * 8 + 2 * t + e;
-              w |= (uint32_t)cS[j * kD + c] << (16 * e + 2 * (4 * rh + 2 * ks + ch));
+              w |= (uint32_t)(cS[j * kD + c] & 3) << (16 * e + 2 * (4 * rh + 2 * ks + ch));
             }
       reinterpret_cast<uint32_t*>(blk + frag_unit_off(u, G, lv.unit_bytes) + 1024)[wi] = w;
+    }
+    // 4-bit values: the high plane (code >> 2) in the same bit order, after the unit's value scales
+    for (int i = tid; i < (lv.v_bits == 4 ? U * 256 : 0); i += 256) {
+      const int u = i >> 8, wi = i & 255;
+      const int ct = (wi >> 7) * 4 + (wi & 3), lane = (wi >> 2) & 31;
+      const int r = lane >> 2, t = lane & 3;
+      uint32_t w = 0;
+#pragma unroll
+      for (int rh = 0; rh < 2; ++rh)
+#pragma unroll
+        for (int ks = 0; ks < 2; ++ks)
+#pragma unroll
+          for (int ch = 0; ch < 2; ++ch)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              const int c = ct * 16 + rh * 8 + r;
+              const int j = 32 * u + ks * 16 + ch * 8 + 2 * t + e;
+              w |= (uint32_t)(cS[j * kD + c] >> 2) << (16 * e + 2 * (4 * rh + 2 * ks + ch));
+            }
+      reinterpret_cast<uint32_t*>(blk + frag_unit_off(u, G, lv.unit_bytes) + 2048 + 128 * VG)[wi] = w;
     }
   }
 

@@ -11,27 +11,27 @@ def f32(t):
 
 
 def make_cache(binding, w, max_tokens=None, importance_mode=0, extras_budget_bytes=0, layout=0, budget_bf16=0,
-               budget_u4=0, sink_len=0):
+               budget_u4=0, sink_len=0, v_bits=2):
     cfg = binding.make_config(w.n_layers, w.batch, w.n_q_heads, w.n_kv_heads, max_tokens or (w.tokens + 256),
                               residual_len=w.residual_len, group_size=w.group_size, tau_bf16=w.tau_bf16,
                               tau_u4=w.tau_u4, score_bits=w.score_bits, importance_mode=importance_mode,
                               extras_budget_bytes=extras_budget_bytes, block_layout=layout, budget_bf16=budget_bf16,
-                              budget_u4=budget_u4, sink_len=sink_len)
+                              budget_u4=budget_u4, sink_len=sink_len, v_bits=v_bits)
     return binding.Cache(cfg)
 
 
-def oracle_stream(w, importance_mode=0, budget_bf16=0, budget_u4=0, sink_len=0):
+def oracle_stream(w, importance_mode=0, budget_bf16=0, budget_u4=0, sink_len=0, v_bits=2):
     return O.OracleStream(g=w.g, R=w.residual_len, G=w.group_size, score_bits=w.score_bits, tau_bf16=w.tau_bf16,
                           tau_u4=w.tau_u4, importance_mode=importance_mode, budget_bf16=budget_bf16, budget_u4=budget_u4,
-                          sink_len=sink_len)
+                          sink_len=sink_len, v_bits=v_bits)
 
 
-def oracle_streams(w, layer, k, v, q, streams=None, importance_mode=0, budget_bf16=0, budget_u4=0, sink_len=0):
+def oracle_streams(w, layer, k, v, q, streams=None, importance_mode=0, budget_bf16=0, budget_u4=0, sink_len=0, v_bits=2):
     """Oracle caches of the requested (b, hk) streams after a bulk append of k, v, q (CPU bf16 tensors)."""
     out = {}
     kf, vf, qf = f32(k), f32(v), f32(q)
     for (b, hk) in streams or [(b, hk) for b in range(w.batch) for hk in range(w.n_kv_heads)]:
-        st = oracle_stream(w, importance_mode, budget_bf16, budget_u4, sink_len)
+        st = oracle_stream(w, importance_mode, budget_bf16, budget_u4, sink_len, v_bits)
         st.append_many(kf[b, hk], vf[b, hk], qf[b, hk * w.g:(hk + 1) * w.g])
         out[(b, hk)] = st
     return out

@@ -39,7 +39,7 @@ def test_cache_bytes_and_argument_validation(binding):
     assert nbytes > 2 * 4 * (8 * 12288 + 32768 + 65536)
     assert ws >= (148 * 8) * 8 * 130 * 4
     lib = binding.lib()
-    for field, bad, code in [("head_dim", 64, -2), ("v_bits", 4, -2), ("group_size", 48, -2), ("residual_len", 100, -2),
+    for field, bad, code in [("head_dim", 64, -2), ("v_bits", 3, -2), ("group_size", 48, -2), ("residual_len", 100, -2),
                              ("residual_len", 512, -2), ("n_q_heads", 7, -1), ("batch", 0, -1), ("score_bits", 3, -2),
                              ("n_q_heads", 32, -2)]:
         c = binding.make_config(2, 2, 8, 2, 1024)
@@ -49,6 +49,12 @@ def test_cache_bytes_and_argument_validation(binding):
     assert lib.mixkvq_cache_bytes(C.byref(c), None, None) == -2          # the tile layout needs R = 128
     c = binding.make_config(1, 1, 1, 1, 256, residual_len=64, group_size=128)
     assert lib.mixkvq_cache_bytes(C.byref(c), None, None) == -2          # R must be a multiple of G
+    c = binding.make_config(1, 1, 1, 1, 256, block_layout=1, v_bits=4)
+    assert lib.mixkvq_cache_bytes(C.byref(c), None, None) == -2          # 4-bit values: fragment layout only
+    for field, bad in [("sink_len", 48), ("sink_len", 512), ("budget_bf16", 100), ("reserved", 1)]:
+        c = binding.make_config(1, 1, 1, 1, 256, budget_u4=40)
+        setattr(c, field, bad)
+        assert lib.mixkvq_cache_bytes(C.byref(c), None, None) == -1, field
     assert lib.mixkvq_cache_bytes(None, None, None) == -1
     assert binding.status_string(-5) == "append exceeds max_tokens"
     assert binding.status_string(0) == "ok"

@@ -243,6 +243,40 @@ def test_decode_steps_through_the_sink(binding, kind):
     assert cache.status() == 0
 
 
+@pytest.mark.parametrize("kind", [0, 1])
+@pytest.mark.parametrize("R,G,preset", [(128, 32, "P24"), (128, 32, "P27"), (64, 64, "P24"), (128, 128, "P4BASE"), (256, 32, "P24")])
+def test_four_bit_values(binding, kind, R, G, preset):
+    # values at 4 bits per token group: two 2-bit planes per unit, bytes equal to the oracle's, attention within tolerance,
+    # and a few fused decode steps on top (one of them flushes a window when R = 64)
+    w = small("llama8b", batch=2, tokens=2 * R + 61, residual_len=R, group_size=G, **getattr(W, preset))
+    k, v, q = W.tokens(w, 0, 0, w.tokens + 6)
+    kc, vc, qc = k.cuda(), v.cuda(), q.cuda()
+    budget = 16 * 8192 if preset == "P4BASE" else 0
+    cache = U.make_cache(binding, w, v_bits=4, extras_budget_bytes=budget)
+    n = w.tokens
+    cache.quantize_append(0, kc[:, :, :n].contiguous(), vc[:, :, :n].contiguous(), qc[:, :, :n].contiguous())
+    cache.set_attention_kernel(kind)
+    orc = U.oracle_streams(w, 0, k[:, :, :n], v[:, :, :n], q[:, :, :n], v_bits=4)
+    U.compare_regions(cache, 0, w, orc)
+    qd = W.decode_query(w, 0, 0)
+    out = cache.decode_attention(0, qd.cuda(), W.softmax_scale())
+    assert U.max_abs_err(w, out, U.oracle_attention(w, orc, qd)) <= ATTN_TOL
+    for t in range(n, n + 6):
+        out = cache.decode_step(0, kc[:, :, t:t + 1].contiguous(), vc[:, :, t:t + 1].contiguous(),
+                                qc[:, :, t:t + 1].contiguous(), W.softmax_scale())
+        for (b, hk), st in orc.items():
+            st.append(U.f32(k[b, hk, t]), U.f32(v[b, hk, t]), U.f32(q[b, hk * w.g:(hk + 1) * w.g, t]))
+    assert U.max_abs_err(w, out, U.oracle_attention(w, orc, q[:, :, n + 5])) <= ATTN_TOL
+    U.compare_regions(cache, 0, w, orc)
+    assert cache.status() == 0
+
+
+def test_four_bit_values_need_the_fragment_layout(binding):
+    cfg = binding.make_config(1, 1, 4, 1, 1024, block_layout=1, v_bits=4)
+    with pytest.raises(binding.MixKVQError):
+        binding.cache_bytes(cfg)
+
+
 # ------------------------------------------------------------------------------------------- attention
 @pytest.mark.parametrize("kind,layout", [(0, 0), (1, 0), (0, 1), (1, 1)])
 @pytest.mark.parametrize("name,tokens,preset", [

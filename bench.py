@@ -234,6 +234,7 @@ def run_gpu(args, w):
                               residual_len=w.residual_len, group_size=w.group_size, tau_bf16=w.tau_bf16,
                               tau_u4=w.tau_u4, score_bits=w.score_bits, block_layout=args.layout,
                               importance_mode=args.importance_mode, sink_len=args.sink_len, v_bits=args.v_bits,
+                              budget_bf16=args.budget_bf16, budget_u4=args.budget_u4,
                               extras_budget_bytes=((w.tokens + n_steps) // w.residual_len + 3) * 8192 if w.score_bits == 4 else 0)
     cache = binding.Cache(cfg, device=dev)
     prefill_ms = prefill(cache, w, dev)
@@ -373,7 +374,8 @@ def run_gpu(args, w):
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal_8TBs": achieved / 8000.0,
                      # the committed counters were taken on the two-tier mix (no UINT4 tier): other mixes have none
-                     "traffic": None if (w.tau_u4 < w.tau_bf16 or args.v_bits != 2 or args.sink_len) else measured_traffic(
+                     "traffic": None if (w.tau_u4 < w.tau_bf16 or args.v_bits != 2 or args.sink_len or args.budget_bf16 +
+                                         args.budget_u4) else measured_traffic(
                          *(("attention_tc_kernel", "attention_tc.cu") if args.layout == 1 else
                            ("attention_mma_kernel", "attention_mma.cu")), w.group_size, tokens_packed,
                          w.batch * w.n_kv_heads),
@@ -407,6 +409,8 @@ def main():
                     help="0: window importance (default), 1: cumulative, 2: error-only salience")
     ap.add_argument("--sink-len", type=int, default=0, help="sink tokens kept in bf16 (0, or a multiple of 32 up to 256)")
     ap.add_argument("--v-bits", type=int, default=2, choices=[2, 4], help="value bit-width (4: fragment layout only)")
+    ap.add_argument("--budget-bf16", type=int, default=0, help="fixed-budget tiering: BF16 channels per window")
+    ap.add_argument("--budget-u4", type=int, default=0, help="fixed-budget tiering: UINT4 channels per window")
     ap.add_argument("--tokens", type=int, default=None)
     ap.add_argument("--layers", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

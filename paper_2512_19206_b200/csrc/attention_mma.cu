@@ -293,6 +293,9 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
     bool new_block = true;
     int n16 = 0, n4 = 0, n16p = 0;
     uint32_t xb0 = 0u, xb1 = 0u;          // B fragments of the block's first 16 promoted channels
+    // the block's first 32 UINT4 channels (two tiles of eight pairs): B fragments (gathered fp16 query pairs) and, per
+    // pair, where the two channels' scales sit in the scale table (half index, 0xFFFF: no channel)
+    uint32_t u4q[2][2] = {{0u, 0u}, {0u, 0u}}, u4s[2][2] = {{~0u, ~0u}, {~0u, ~0u}};
     const char* ex = nullptr;             // the block's extras
     const char* exu = nullptr;            // ... of the current unit
     uint32_t ex_unit = 0;
@@ -377,6 +380,29 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
           };
           xb0 = gather_q(t);
           xb1 = gather_q(t + 4);
+        }
+        if (kU4 == 1 && n4 > 0) {
+          const int n4pairs = (n4 + 1) >> 1;
+          const unsigned char* ids4 = reinterpret_cast<const unsigned char*>(ex) + 2 * n16p;
+#pragma unroll
+          for (int kk = 0; kk < 2; ++kk)
+#pragma unroll
+            for (int hp = 0; hp < 2; ++hp) {
+              const int p = 8 * kk + 4 * hp + t;
+              uint32_t c0 = 255u, c1 = 255u;
+              if (p < n4pairs) {
+                c0 = ids4[2 * p];
+                c1 = ids4[2 * p + 1];
+              }
+              auto scale_index = [&](uint32_t c) -> uint32_t {      // half index of channel c's scale in kprep
+                const int kt = c >> 4, col = c & 15;
+                return c < 128 ? (uint32_t)(((scale_word(kt) + ((col & 7) >> 1) * 2 + (col >> 3)) << 1) + (col & 1)) : 0xFFFFu;
+              };
+              const uint32_t q0 = c0 < 128 ? (uint32_t)__half_as_ushort(qf16[r * kD + c0]) : 0u;
+              const uint32_t q1 = c1 < 128 ? (uint32_t)__half_as_ushort(qf16[r * kD + c1]) : 0u;
+              u4q[kk][hp] = q0 | (q1 << 16);
+              u4s[kk][hp] = scale_index(c0) | (scale_index(c1) << 16);
+            }
         }
         new_block = false;
         xa_loaded = false;
@@ -516,47 +542,57 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
           for (int mt = 0; mt < 2; ++mt) mma_bf16(Sx[mt], a[mt][0], a[mt][1], a[mt][2], a[mt][3], b0, b1);
         }
       }
-      // ---- UINT4 high plane: c_hi * 4s, gathered q in fp16
+      // ---- UINT4 high plane: c_hi * 4s, gathered q in fp16.  The first two tiles (32 channels) use the block's gathered
+      // query pairs and scale positions; further tiles look their channels up per unit.
       if (kU4 == 1 && n4 > 0) {
         const int n4pairs = (n4 + 1) >> 1;
         const uint32_t* hw = reinterpret_cast<const uint32_t*>(exu + 128 * n16p);
         const unsigned char* ids4 = reinterpret_cast<const unsigned char*>(ex) + 2 * n16p;
-        const __half* kph = reinterpret_cast<const __half*>(kprep);
-        for (int kk = 0; kk * 8 < n4pairs; ++kk) {
-          uint32_t a[2][4], b[2];
+        const unsigned short* kph = reinterpret_cast<const unsigned short*>(kprep);
+        auto plane_tile = [&](int kk, const uint32_t (&sidx)[2], const uint32_t (&qb)[2]) {
+          uint32_t a[2][4];
 #pragma unroll
           for (int hp = 0; hp < 2; ++hp) {
             const int p = 8 * kk + 4 * hp + t;
-            uint32_t w = 0, sc = 0;
-            b[hp] = 0;
-            if (p < n4pairs) {
-              w = hw[p * 4 + (r & 3)] >> (8 * (r >> 2));
-              const uint32_t c0 = ids4[2 * p], c1 = ids4[2 * p + 1];
-              auto scale_of = [&](uint32_t c) -> __half {
-                // fp16 scale of channel c in kprep: [(kt*4 + t')*4 + ch*2] half2, element e
-                const int kt = c >> 4, col = c & 15;
-                return kph[((scale_word(kt) + ((col & 7) >> 1) * 2 + (col >> 3)) << 1) + (col & 1)];
-              };
-              const __half zero = __float2half_rn(0.f);
-              const __half s0 = (c0 < 128) ? scale_of(c0) : zero, s1 = (c1 < 128) ? scale_of(c1) : zero;
-              const __half q0 = (c0 < 128) ? qf16[r * kD + c0] : zero, q1 = (c1 < 128) ? qf16[r * kD + c1] : zero;
-              __half2 s2 = __halves2half2(s0, s1), q2 = __halves2half2(q0, q1);
-              sc = *reinterpret_cast<uint32_t*>(&s2);
-              b[hp] = *reinterpret_cast<uint32_t*>(&q2);
-            }
-            const uint32_t m4 = hmul2_u(sc, 0x44004400u);          // 4s
+            const uint32_t w = p < n4pairs ? hw[p * 4 + (r & 3)] >> (8 * (r >> 2)) : 0u;
+            const uint32_t i0 = sidx[hp] & 0xFFFFu, i1 = sidx[hp] >> 16;
+            const uint32_t sc = (i0 != 0xFFFFu ? (uint32_t)kph[i0] : 0u) | ((i1 != 0xFFFFu ? (uint32_t)kph[i1] : 0u) << 16);
+            const uint32_t m4 = hmul2_u(sc, four2);                // 4s
             const uint32_t o4 = hmul2_u(sc, 0xCC00CC00u);          // -16s
 #pragma unroll
             for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
               for (int rh = 0; rh < 2; ++rh) {
                 const int f = 2 * mt + rh;
-                const uint32_t code = ((w << (8 - 2 * f)) & 0x03000300u) | 0x44004400u;   // 4 + c_hi
+                const uint32_t code = ((w << (8 - 2 * f)) & 0x03000300u) | four2;          // 4 + c_hi
                 a[mt][2 * hp + rh] = hfma2_u(code, m4, o4);                                // c_hi * 4s
               }
           }
 #pragma unroll
-          for (int mt = 0; mt < 2; ++mt) mma_f16(Sx[mt], a[mt][0], a[mt][1], a[mt][2], a[mt][3], b[0], b[1]);
+          for (int mt = 0; mt < 2; ++mt) mma_f16(Sx[mt], a[mt][0], a[mt][1], a[mt][2], a[mt][3], qb[0], qb[1]);
+        };
+        plane_tile(0, u4s[0], u4q[0]);
+        if (n4pairs > 8) plane_tile(1, u4s[1], u4q[1]);
+        for (int kk = 2; kk * 8 < n4pairs; ++kk) {
+          uint32_t sidx[2], qb[2];
+#pragma unroll
+          for (int hp = 0; hp < 2; ++hp) {
+            const int p = 8 * kk + 4 * hp + t;
+            uint32_t c0 = 255u, c1 = 255u;
+            if (p < n4pairs) {
+              c0 = ids4[2 * p];
+              c1 = ids4[2 * p + 1];
+            }
+            auto scale_index = [&](uint32_t c) -> uint32_t {
+              const int kt = c >> 4, col = c & 15;
+              return c < 128 ? (uint32_t)(((scale_word(kt) + ((col & 7) >> 1) * 2 + (col >> 3)) << 1) + (col & 1)) : 0xFFFFu;
+            };
+            const uint32_t q0 = c0 < 128 ? (uint32_t)__half_as_ushort(qf16[r * kD + c0]) : 0u;
+            const uint32_t q1 = c1 < 128 ? (uint32_t)__half_as_ushort(qf16[r * kD + c1]) : 0u;
+            qb[hp] = q0 | (q1 << 16);
+            sidx[hp] = scale_index(c0) | (scale_index(c1) << 16);
+          }
+          plane_tile(kk, sidx, qb);
         }
       }
 

@@ -418,6 +418,19 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
       // ---- extras of this unit (BF16 pairs of the first 16 promoted channels), unless the previous unit already
       // requested them
       if (n16 > 0 && !xa_loaded) load_xa(exu);
+      // the UINT4 high-plane words of the first two tiles of this unit are requested early as well
+      uint32_t u4w[2][2] = {{0u, 0u}, {0u, 0u}};
+      if (kU4 == 1 && n4 > 0) {
+        const int n4pairs = (n4 + 1) >> 1;
+        const uint32_t* hw = reinterpret_cast<const uint32_t*>(exu + 128 * n16p);
+#pragma unroll
+        for (int kk = 0; kk < 2; ++kk)
+#pragma unroll
+          for (int hp = 0; hp < 2; ++hp) {
+            const int p = 8 * kk + 4 * hp + t;
+            if (p < n4pairs) u4w[kk][hp] = hw[p * 4 + (r & 3)];
+          }
+      }
       // the key codes: two 16-byte loads per lane are the A fragments of all sixteen key tiles (with a 4-bit base the
       // first plane to run is the high plane, which lies with the block's extras in global memory)
       const uint4* kplane = (kU4 == 2) ? reinterpret_cast<const uint4*>(exu + 128 * n16p) : reinterpret_cast<const uint4*>(st);
@@ -549,12 +562,11 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
         const uint32_t* hw = reinterpret_cast<const uint32_t*>(exu + 128 * n16p);
         const unsigned char* ids4 = reinterpret_cast<const unsigned char*>(ex) + 2 * n16p;
         const unsigned short* kph = reinterpret_cast<const unsigned short*>(kprep);
-        auto plane_tile = [&](int kk, const uint32_t (&sidx)[2], const uint32_t (&qb)[2]) {
+        auto plane_tile = [&](const uint32_t (&words)[2], const uint32_t (&sidx)[2], const uint32_t (&qb)[2]) {
           uint32_t a[2][4];
 #pragma unroll
           for (int hp = 0; hp < 2; ++hp) {
-            const int p = 8 * kk + 4 * hp + t;
-            const uint32_t w = p < n4pairs ? hw[p * 4 + (r & 3)] >> (8 * (r >> 2)) : 0u;
+            const uint32_t w = words[hp] >> (8 * (r >> 2));
             const uint32_t i0 = sidx[hp] & 0xFFFFu, i1 = sidx[hp] >> 16;
             const uint32_t sc = (i0 != 0xFFFFu ? (uint32_t)kph[i0] : 0u) | ((i1 != 0xFFFFu ? (uint32_t)kph[i1] : 0u) << 16);
             const uint32_t m4 = hmul2_u(sc, four2);                // 4s
@@ -571,10 +583,10 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
 #pragma unroll
           for (int mt = 0; mt < 2; ++mt) mma_f16(Sx[mt], a[mt][0], a[mt][1], a[mt][2], a[mt][3], qb[0], qb[1]);
         };
-        plane_tile(0, u4s[0], u4q[0]);
-        if (n4pairs > 8) plane_tile(1, u4s[1], u4q[1]);
+        plane_tile(u4w[0], u4s[0], u4q[0]);
+        if (n4pairs > 8) plane_tile(u4w[1], u4s[1], u4q[1]);
         for (int kk = 2; kk * 8 < n4pairs; ++kk) {
-          uint32_t sidx[2], qb[2];
+          uint32_t sidx[2], qb[2], words[2] = {0u, 0u};
 #pragma unroll
           for (int hp = 0; hp < 2; ++hp) {
             const int p = 8 * kk + 4 * hp + t;
@@ -582,6 +594,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
             if (p < n4pairs) {
               c0 = ids4[2 * p];
               c1 = ids4[2 * p + 1];
+              words[hp] = hw[p * 4 + (r & 3)];
             }
             auto scale_index = [&](uint32_t c) -> uint32_t {
               const int kt = c >> 4, col = c & 15;
@@ -592,7 +605,7 @@ attention_mma_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sc
             qb[hp] = q0 | (q1 << 16);
             sidx[hp] = scale_index(c0) | (scale_index(c1) << 16);
           }
-          plane_tile(kk, sidx, qb);
+          plane_tile(words, sidx, qb);
         }
       }
 

@@ -277,6 +277,31 @@ def test_four_bit_values_need_the_fragment_layout(binding):
         binding.cache_bytes(cfg)
 
 
+def test_stream_order_around_the_early_started_kernels(binding):
+    # the attention and combine kernels may start before their predecessor in the stream has finished and wait for it on
+    # the device: a query rewritten by an ordinary kernel right before the call, and an output copied right after it,
+    # must behave as in plain stream order, call after call without host synchronization
+    w = small("qwen7b", batch=2, tokens=6 * 128 + 50, **W.P24)
+    k, v, q = W.tokens(w, 0, 0, w.tokens)
+    cache = U.make_cache(binding, w)
+    cache.quantize_append(0, k.cuda(), v.cuda(), q.cuda())
+    queries = [W.decode_query(w, 0, i).cuda() for i in range(6)]
+    want = [cache.decode_attention(0, qi, W.softmax_scale()).clone() for qi in queries]
+    torch.cuda.synchronize()
+    q_dev = torch.empty_like(queries[0])
+    out = torch.empty_like(want[0])
+    got = []
+    for rep in range(3):
+        for qi in queries:
+            q_dev.copy_(qi)                                   # ordinary kernel writes the input
+            cache.decode_attention(0, q_dev, W.softmax_scale(), out=out)
+            got.append(out.clone())                           # ordinary kernel reads the output
+    torch.cuda.synchronize()
+    for i, g in enumerate(got):
+        assert torch.equal(g, want[i % len(queries)]), i
+    assert cache.status() == 0
+
+
 # ------------------------------------------------------------------------------------------- attention
 @pytest.mark.parametrize("kind,layout", [(0, 0), (1, 0), (0, 1), (1, 1)])
 @pytest.mark.parametrize("name,tokens,preset", [

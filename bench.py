@@ -377,10 +377,10 @@ def run_gpu(args, w):
                      "traffic": None if (w.tau_u4 < w.tau_bf16 or args.v_bits != 2 or args.sink_len or args.budget_bf16 +
                                          args.budget_u4) else measured_traffic(
                          *(("attention_tc_kernel", "attention_tc.cu") if args.layout == 1 else
-                           ("attention_mma_kernel", "attention_mma.cu")), w.group_size, tokens_packed,
+                           ("attention_ws_kernel", "attention_ws.cu")), w.group_size, tokens_packed,
                          w.batch * w.n_kv_heads),
                      "peak_source": peak_src,
-                     "kernel": "attention_tc_kernel" if args.layout == 1 else "attention_mma_kernel", "kernel_us": kern_ms * 1e3, "algorithmic_bytes": alg},
+                     "kernel": "attention_tc_kernel" if args.layout == 1 else "attention_ws_kernel", "kernel_us": kern_ms * 1e3, "algorithmic_bytes": alg},
         "e2e": {"value": e2e_us, "unit": "us/step", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": n_e2e},
         "gpu_launches": int(launches),

@@ -1,39 +1,62 @@
-"""Builds libmixkvq.so (sm_100a) in-tree with nvcc.  Usable as `python -m paper_2512_19206_b200.build`."""
+"""Builds libmixkvq.so (sm_100a) in-tree with nvcc.  Usable as `python -m paper_2512_19206_b200.build`.
+
+Every source file is compiled to an object of its own (in parallel, only when it or a header changed) and the
+objects are linked into the shared library.
+"""
 from __future__ import annotations
 
 import os
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
+OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libmixkvq.so")
-SOURCES = ["api.cu", "append.cu", "select.cu", "flush.cu", "combine.cu", "attention_simt.cu", "attention_mma.cu",
+SOURCES = ["api.cu", "append.cu", "select.cu", "flush.cu", "combine.cu", "attention_simt.cu", "attention_ws.cu",
            "attention_tc.cu"]
+FLAGS = ["-Xcompiler", "-fPIC", "-O3", "-std=c++17", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
+         "--fmad=true"]
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB):
-        return True
-    t = os.path.getmtime(LIB)
-    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(HERE, "..", "include", "mixkvq.h")]
-    return any(os.path.getmtime(d) > t for d in deps)
+def _headers() -> list[str]:
+    return [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cuh", ".h"))] + [
+        os.path.join(HERE, "..", "include", "mixkvq.h")]
+
+
+def _newer(path: str, than: float) -> bool:
+    return os.path.getmtime(path) > than
+
+
+def _compile(nvcc: str, src: str, obj: str, verbose: bool) -> str:
+    cmd = [nvcc, "-c"] + FLAGS + (["-Xptxas=-v"] if verbose else []) + ["-o", obj, src]
+    res = subprocess.run(cmd, capture_output=True, text=True)
+    if res.returncode != 0:
+        raise RuntimeError("nvcc failed on " + src + ":\n" + res.stdout + res.stderr)
+    return res.stderr
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not _stale():
-        return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cmd = [nvcc, "-shared", "-Xcompiler", "-fPIC", "-O3", "-std=c++17", "-lineinfo",
-           "-gencode", "arch=compute_100a,code=sm_100a", "--fmad=true",
-           "-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES]
+    os.makedirs(OBJ, exist_ok=True)
+    hdr_time = max(os.path.getmtime(h) for h in _headers())
+    jobs = []
+    for s in SOURCES:
+        src, obj = os.path.join(CSRC, s), os.path.join(OBJ, s[:-3] + ".o")
+        if force or not os.path.exists(obj) or _newer(src, os.path.getmtime(obj)) or hdr_time > os.path.getmtime(obj):
+            jobs.append((src, obj))
+    with ThreadPoolExecutor(max_workers=min(8, max(1, len(jobs)))) as pool:
+        logs = list(pool.map(lambda j: _compile(nvcc, j[0], j[1], verbose), jobs))
     if verbose:
-        cmd.insert(1, "-Xptxas=-v")
-    res = subprocess.run(cmd, capture_output=True, text=True)
-    if res.returncode != 0:
-        raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
-    if verbose:
-        print(res.stderr)
+        for log in logs:
+            print(log)
+    objs = [os.path.join(OBJ, s[:-3] + ".o") for s in SOURCES]
+    if jobs or not os.path.exists(LIB) or any(_newer(o, os.path.getmtime(LIB)) for o in objs):
+        res = subprocess.run([nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB] + objs,
+                             capture_output=True, text=True)
+        if res.returncode != 0:
+            raise RuntimeError("link failed:\n" + res.stdout + res.stderr)
     return LIB
 
 

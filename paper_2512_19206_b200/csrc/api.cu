@@ -139,7 +139,7 @@ int run_attention(mixkvq_cache* h, int layer, const void* q, float* out, float s
   else if (h->tile)
     e = launch_attention_tc(lv, q, h->attn_kind == 2 ? nullptr : out, scale, ws, h->n_sms, st, &launches);
   else
-    e = launch_attention_mma(lv, q, h->attn_kind == 2 ? nullptr : out, scale, ws, h->n_sms, st, &launches);
+    e = launch_attention_ws(lv, q, h->attn_kind == 2 ? nullptr : out, scale, ws, h->n_sms, st, &launches);
   h->launches += launches;
   return e == cudaSuccess ? MIXKVQ_OK : MIXKVQ_E_CUDA;
 }
@@ -184,7 +184,7 @@ int mixkvq_cache_init(const mixkvq_config* cfg, void* cache_dev, size_t bytes, v
   if (cudaMemsetAsync(h->mem, 0, kHeaderBytes, st) != cudaSuccess) { delete h; return MIXKVQ_E_CUDA; }
   for (int l = 0; l < cfg->n_layers; ++l)
     if (zero_layer_state(h, l, st) != MIXKVQ_OK) { delete h; return MIXKVQ_E_CUDA; }
-  if (attention_mma_setup() != cudaSuccess || attention_tc_setup() != cudaSuccess) { delete h; return MIXKVQ_E_CUDA; }
+  if (attention_ws_setup() != cudaSuccess || attention_tc_setup() != cudaSuccess) { delete h; return MIXKVQ_E_CUDA; }
   *out = h;
   return MIXKVQ_OK;
 }

@@ -21,8 +21,8 @@ namespace mixkvq {
 
 cudaError_t launch_combine2(const float* ws, float* out, int g, int Hkv, int Hq, int S, int n1, long long units1,
                             int slot2, int n2, long long units2, cudaStream_t stream);
-int attention_mma_grid(const LayerView& lv, int n_sms);
-long long attention_mma_positions(const LayerView& lv);
+int attention_ws_grid(const LayerView& lv, int n_sms);
+long long attention_ws_positions(const LayerView& lv);
 
 namespace {
 
@@ -729,7 +729,7 @@ cudaError_t attention_tc_setup() {
 cudaError_t launch_attention_tc(const LayerView& lv, const void* q, float* out, float scale, float* ws, int n_sms,
                                 cudaStream_t stream, int* launches) {
   *launches = 0;
-  if (lv.n_blocks == 0) return launch_attention_mma(lv, q, out, scale, ws, n_sms, stream, launches);
+  if (lv.n_blocks == 0) return launch_attention_ws(lv, q, out, scale, ws, n_sms, stream, launches);
   const int S = lv.B * lv.Hkv;
   const long long total = (long long)S * lv.n_blocks;
   int grid = (int)min((long long)min(n_sms, kMaxCtas / (2 * kWG)), (total + kWG - 1) / kWG);
@@ -745,11 +745,11 @@ cudaError_t launch_attention_tc(const LayerView& lv, const void* q, float* out, 
   const int n1 = (int)min((long long)grid * kWG, total);      // worker groups that own packed blocks
   const int slot2 = n1 + S;
   int l2 = 0;
-  e = launch_attention_mma(res, q, nullptr, scale, ws + (size_t)slot2 * kPartialFloats, n_sms, stream, &l2);
+  e = launch_attention_ws(res, q, nullptr, scale, ws + (size_t)slot2 * kPartialFloats, n_sms, stream, &l2);
   *launches += l2;
   if (e != cudaSuccess) return e;
-  e = launch_combine2(ws, out, lv.g, lv.Hkv, lv.Hq, S, n1, lv.n_blocks, slot2, attention_mma_grid(res, n_sms),
-                      attention_mma_positions(res), stream);
+  e = launch_combine2(ws, out, lv.g, lv.Hkv, lv.Hq, S, n1, lv.n_blocks, slot2, attention_ws_grid(res, n_sms),
+                      attention_ws_positions(res), stream);
   *launches += 1;
   return e;
 }

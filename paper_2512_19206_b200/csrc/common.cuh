@@ -48,6 +48,11 @@ struct LayerView {
   // The attention kernel then stores them at residual slot r - 1 and adds |q| to the importance accumulator itself.
   const uint16_t* new_k;
   const uint16_t* new_v;
+  // waits on staged copies and on hand-overs between warps give up after this many polls (0: the kernel's default)
+  uint32_t wait_polls;
+  // test hook for the give-up path: the barrier of every warp pair's first staged copy is armed for this many bytes
+  // more than are copied, so that it never completes (0 in normal use)
+  uint32_t debug_extra_tx;
 };
 
 __host__ __device__ inline uint32_t extras_header_bytes(int n16, int n4) {
@@ -185,9 +190,9 @@ cudaError_t launch_select_raw(const void* q, const void* k, int B, int Hq, int H
 // decode attention: writes split partials to `ws`, then the combine kernel writes `out`; returns launches made
 cudaError_t launch_attention_simt(const LayerView& lv, const void* q, float* out, float scale, float* ws,
                                   int n_sms, cudaStream_t stream, int* launches);
-cudaError_t launch_attention_mma(const LayerView& lv, const void* q, float* out, float scale, float* ws,
-                                 int n_sms, cudaStream_t stream, int* launches);
-cudaError_t attention_mma_setup();
+cudaError_t launch_attention_ws(const LayerView& lv, const void* q, float* out, float scale, float* ws,
+                                int n_sms, cudaStream_t stream, int* launches);
+cudaError_t attention_ws_setup();
 // tile layout (R == 128): tcgen05 kernel
 cudaError_t launch_attention_tc(const LayerView& lv, const void* q, float* out, float scale, float* ws,
                                 int n_sms, cudaStream_t stream, int* launches);

@@ -12,7 +12,7 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libmixkvq.so")
+LIB_PATH = os.environ.get("MIXKVQ_LIB") or os.path.join(_HERE, "libmixkvq.so")
 
 EXPORTS = [
     "mixkvq_cache_bytes", "mixkvq_cache_init", "mixkvq_cache_destroy", "mixkvq_cache_reset",

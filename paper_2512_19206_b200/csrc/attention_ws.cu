@@ -52,8 +52,7 @@ __host__ __device__ constexpr int pair_bytes(bool v4) {
 constexpr int kBarsPerPair = 2 * kStages + 2;
 constexpr int kQS = 136;                     // halves per row of the query tables (272 bytes: rows fall on different banks)
 constexpr int kBarBytes = ((kPairs * kBarsPerPair * 8 + 127) / 128) * 128;
-constexpr int kBqBytes = 8 * 32 * 8;           // B fragments of q for the base key tiles: [8 k-tiles][32 lanes] 8 bytes
-constexpr int kSharedTail = kBarBytes + 2 * 8 * kQS * 2 + kBqBytes + 2 * kPairs * 32;
+constexpr int kSharedTail = kBarBytes + 2 * 8 * kQS * 2 + 2 * kPairs * 32;
 __host__ __device__ constexpr int smem_bytes(bool v4) { return kPairs * pair_bytes(v4) + kSharedTail; }
 constexpr int kResidualWeight = 3;           // an unquantized 32-token unit counts as this many packed units in the split
 constexpr int kMergeStride = 132;            // floats per head row of a pair's output in the merge
@@ -259,12 +258,11 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
   const uint32_t rfull_u32 = bar_u32 + 2 * kStages * 8, rempty_u32 = rfull_u32 + 8;
   const uint32_t qb16_u32 = tail_u32 + kBarBytes;                           // [8][kQS] q, bf16 bits (0 for heads >= g)
   const uint32_t qf16_u32 = qb16_u32 + 8 * kQS * 2;                         // [8][kQS] q, fp16
-  const uint32_t bq_u32 = qf16_u32 + 8 * kQS * 2;                           // [8 kt][32 lanes]{channels 2t.., channels 8 + 2t..} fp16 q * mult(kt)
-  float* mS = reinterpret_cast<float*>(smem + kPairs * kPairBytes + kBarBytes + 2 * 8 * kQS * 2 + kBqBytes);    // [kPairs][8]
+  float* mS = reinterpret_cast<float*>(smem + kPairs * kPairBytes + kBarBytes + 2 * 8 * kQS * 2);    // [kPairs][8]
   float* lS = mS + kPairs * 8;                                                                       // [kPairs][8]
 
-  if (threadIdx.x == 0) {
-    for (int i = 0; i < kPairs * kBarsPerPair; ++i) mbar_init(tail_u32 + 8 * i, 1);
+  if (threadIdx.x < kPairs * kBarsPerPair) {
+    mbar_init(tail_u32 + 8 * threadIdx.x, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (!logits_role) {
@@ -380,25 +378,12 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
       uint4 q_regs = make_uint4(0u, 0u, 0u, 0u);      // thread (h, c) of the first 128: head h, channels 8c .. 8c+7
       const int b = s / lv.Hkv, hk = s % lv.Hkv, h = threadIdx.x >> 4, c = threadIdx.x & 15;
       if (h < g) q_regs = *reinterpret_cast<const uint4*>(q + ((size_t)b * lv.Hq + hk * g + h) * kD + 8 * c);
-      // B fragments of q for the base key tiles, as lane (r, t) of a logits warp needs them for k-tile kt: head r, channels
-      // 16kt + {2t, 2t+1} and {2t+8, 2t+9}, times mult(kt) = 2^(8 - position of the k-tile's code field)
-      uint32_t bq_lo = 0u, bq_hi = 0u;
-      if (threadIdx.x < 256) {
-        const int kt = threadIdx.x >> 5;
-        if (r < g) {
-          const uint32_t* qw = reinterpret_cast<const uint32_t*>(q + ((size_t)b * lv.Hq + hk * g + r) * kD + 16 * kt + 2 * t);
-          const float mult = __uint_as_float((uint32_t)(127 + 8 - ((0x86486464u >> (4 * kt)) & 0xF)) << 23);
-          const uint32_t w0 = qw[0], w1 = qw[4];
-          bq_lo = pack_half2(bf_lo(w0) * mult, bf_hi(w0) * mult);
-          bq_hi = pack_half2(bf_lo(w1) * mult, bf_hi(w1) * mult);
-        }
-      }
       __syncthreads();          // the previous segment's readers of the tables are done
-      if (threadIdx.x < 256) sts64(bq_u32 + threadIdx.x * 8, bq_lo, bq_hi);
       if (h < 8) {
         sts128(qb16_u32 + (h * kQS + 8 * c) * 2, q_regs.x, q_regs.y, q_regs.z, q_regs.w);
-        sts128(qf16_u32 + (h * kQS + 8 * c) * 2, bf16x2_to_f16x2(q_regs.x), bf16x2_to_f16x2(q_regs.y),
-               bf16x2_to_f16x2(q_regs.z), bf16x2_to_f16x2(q_regs.w));
+        if (kU4 == 1)      // the fp16 table is for the gathered UINT4 channels
+          sts128(qf16_u32 + (h * kQS + 8 * c) * 2, bf16x2_to_f16x2(q_regs.x), bf16x2_to_f16x2(q_regs.y),
+                 bf16x2_to_f16x2(q_regs.z), bf16x2_to_f16x2(q_regs.w));
       }
       __syncthreads();
     }
@@ -481,7 +466,17 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
         u = wb - bi * U;
         pf_entry = table[bi];
       }
-      const uint32_t bq_rd = bq_u32 + lane * 8;          // this lane's B fragments of q for the base key tiles, 256 bytes per k-tile
+      // B fragments of q for the base key tiles: head r, channels 16kt + {2t, 2t+1} and {2t+8, 2t+9}, times mult(kt)
+      uint32_t bq[8][2];
+#pragma unroll
+      for (int kt = 0; kt < 8; ++kt) {
+        const float mult = (float)(1 << (8 - key_pos(kt)));
+#pragma unroll
+        for (int hch = 0; hch < 2; ++hch) {
+          const uint32_t w = lds32(qrow_u32 + (16 * kt + 8 * hch + 2 * t) * 2);
+          bq[kt][hch] = pack_half2(bf_lo(w) * mult, bf_hi(w) * mult);
+        }
+      }
       // per-lane constants of the key-group preparation: the lane converts channels 4*lane .. 4*lane+3 (k-tile lane / 4)
       const float pk_zs = __uint_as_float((119u + (uint32_t)key_pos(lane >> 2)) << 23);        // 2^(pos - 8)
       // zero-point tiles: [8 kt][4 t]{z ch0, z ch0, z ch1, z ch1} half2 z / mult; the lane's first pair
@@ -606,9 +601,8 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
 #pragma unroll
             for (int kt2 = 0; kt2 < 8; ++kt2) {
               const uint4 zz = lds128(zp_rd + 4 * zprep_word(kt2));
-              const uint2 bq = lds64(bq_rd + 256 * kt2);
-              if (kt2 == 0) mma_f16_to(zc, zz.x, zz.y, zz.z, zz.w, bq.x, bq.y, 0.f, 0.f, 0.f, 0.f);
-              else mma_f16(zc, zz.x, zz.y, zz.z, zz.w, bq.x, bq.y);
+              if (kt2 == 0) mma_f16_to(zc, zz.x, zz.y, zz.z, zz.w, bq[0][0], bq[0][1], 0.f, 0.f, 0.f, 0.f);
+              else mma_f16(zc, zz.x, zz.y, zz.z, zz.w, bq[kt2][0], bq[kt2][1]);
             }
           }
 
@@ -621,7 +615,6 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
             for (int kt = 0; kt < 8; ++kt) {
               // scales of the lane's channel pairs (16kt + 2t, +1) and (16kt + 8 + 2t, +1); code bias 4 -> offset -4 s
               uint4 kp = lds128(kp_rd + kprep_off(kt, 0));
-              const uint2 bq = lds64(bq_rd + 256 * kt);
               if (high) kp = make_uint4(hmul2_u(kp.x, four2), hmul2_u(kp.y, four2), hmul2_u(kp.z, four2), hmul2_u(kp.w, four2));
               const uint32_t mask = 0x00030003u << key_pos(kt);
 #pragma unroll
@@ -632,8 +625,8 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
                   const uint32_t code = (key_shift(kw[mt][j], kt) & mask) | four2;           // 4 + c * 2^(pos-8)
                   a[j] = hfma2_u(code, j < 2 ? kp.x : kp.z, j < 2 ? kp.y : kp.w);            // c * s * 2^(pos-8)
                 }
-                if (first && kt == 0) mma_f16_to(Sx[mt], a[0], a[1], a[2], a[3], bq.x, bq.y, zc[0], zc[1], zc[2], zc[3]);
-                else mma_f16(Sx[mt], a[0], a[1], a[2], a[3], bq.x, bq.y);
+                if (first && kt == 0) mma_f16_to(Sx[mt], a[0], a[1], a[2], a[3], bq[0][0], bq[0][1], zc[0], zc[1], zc[2], zc[3]);
+                else mma_f16(Sx[mt], a[0], a[1], a[2], a[3], bq[kt][0], bq[kt][1]);
               }
             }
           };
@@ -915,6 +908,8 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
             sts16(zv_wr + 64 * vg, __half_as_ushort(__float2half_rn(bf_hi(mzv[vg]))));
           }
         }
+        const uint4 vw0 = lds128(st + 1024);
+        const uint4 vw1 = lds128(st + 1536);
         __syncwarp();      // the tables written above are read by other lanes below
         wait_or_give_up(lfull_u32 + ring_stage * 8u, ring_parity);
         const uint32_t lb = lane32 + ring_stage * kLBufBytes;
@@ -945,8 +940,6 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
         }
         // ---- P.V: codes as fp16 subnormals, scales folded into P
         {
-          const uint4 vw0 = lds128(st + 1024);
-          const uint4 vw1 = lds128(st + 1536);
           const uint32_t vw[8] = {vw0.x, vw0.y, vw0.z, vw0.w, vw1.x, vw1.y, vw1.z, vw1.w};
 #pragma unroll
           for (int vg = 0; vg < VG; ++vg) {

@@ -21,11 +21,16 @@ struct mixkvq_cache {
   int n_sms;
   int attn_kind;
   uint64_t launches;
+  // What the library enqueued last on this handle: kNoPackedWrite if it did not write packed blocks, a layer index if
+  // it wrote that layer's packed blocks (a flush), kAllPacked after initialisation, a reset or a write from outside.
+  // The next decode attention on such a layer waits for all earlier work before it reads anything.
+  int last_packed_writer;
 };
 
 namespace {
 
 constexpr uint64_t kHeaderBytes = 256;   // device status word lives at offset 0
+constexpr int kNoPackedWrite = -1, kAllPacked = -2;
 
 uint64_t align_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 
@@ -123,6 +128,7 @@ int zero_layer_state(mixkvq_cache* h, int layer, cudaStream_t st) {
   h->n_blocks[layer] = 0;
   h->r[layer] = 0;
   h->n_sink[layer] = 0;
+  h->last_packed_writer = kAllPacked;
   return MIXKVQ_OK;
 }
 
@@ -132,6 +138,9 @@ int run_attention(mixkvq_cache* h, int layer, const void* q, float* out, float s
   LayerView lv = view(h, layer);
   lv.new_k = static_cast<const uint16_t*>(new_k);
   lv.new_v = static_cast<const uint16_t*>(new_v);
+  lv.stage_early = (h->last_packed_writer == kNoPackedWrite ||
+                    (h->last_packed_writer >= 0 && h->last_packed_writer != layer)) ? 1 : 0;
+  h->last_packed_writer = kNoPackedWrite;
   int launches = 0;
   cudaError_t e;
   if (h->attn_kind == 1)
@@ -174,6 +183,7 @@ int mixkvq_cache_init(const mixkvq_config* cfg, void* cache_dev, size_t bytes, v
   h->n_sink.assign(cfg->n_layers, 0);
   h->attn_kind = 0;
   h->launches = 0;
+  h->last_packed_writer = kAllPacked;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&h->n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
@@ -198,6 +208,7 @@ int mixkvq_cache_reset(mixkvq_cache* cache, int layer, void* stream) {
   if (!cache || layer >= cache->cfg.n_layers) return MIXKVQ_E_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (layer >= 0) return zero_layer_state(cache, layer, st);
+  cache->last_packed_writer = kAllPacked;
   if (cudaMemsetAsync(cache->mem, 0, kHeaderBytes, st) != cudaSuccess) return MIXKVQ_E_CUDA;
   for (int l = 0; l < cache->cfg.n_layers; ++l)
     if (zero_layer_state(cache, l, st) != MIXKVQ_OK) return MIXKVQ_E_CUDA;
@@ -209,6 +220,7 @@ int mixkvq_select_channels(mixkvq_cache* cache, int layer, uint8_t* tiers_dev, d
   if (cache->r[layer] == 0) return MIXKVQ_E_EMPTY;
   LayerView lv = view(cache, layer);
   cache->launches += 1;
+  cache->last_packed_writer = kNoPackedWrite;
   return launch_select_window(lv, tiers_dev, salience_dev, static_cast<cudaStream_t>(stream)) == cudaSuccess
              ? MIXKVQ_OK : MIXKVQ_E_CUDA;
 }
@@ -242,6 +254,7 @@ int mixkvq_quantize_append(mixkvq_cache* cache, int layer, const void* k_dev, co
       LayerView lv = view(cache, layer);
       if (launch_sink_append(lv, k_dev, v_dev, n_tokens, t, m, st) != cudaSuccess) return MIXKVQ_E_CUDA;
       cache->launches += 1;
+      cache->last_packed_writer = kNoPackedWrite;
       cache->n_sink[layer] += m;
       t += m;
       continue;
@@ -250,6 +263,7 @@ int mixkvq_quantize_append(mixkvq_cache* cache, int layer, const void* k_dev, co
       LayerView lv = view(cache, layer);
       if (launch_flush(lv, st) != cudaSuccess) return MIXKVQ_E_CUDA;
       cache->launches += 1;
+      cache->last_packed_writer = layer;
       cache->n_blocks[layer] += 1;
       cache->r[layer] = 0;
     }
@@ -261,6 +275,7 @@ int mixkvq_quantize_append(mixkvq_cache* cache, int layer, const void* k_dev, co
       LayerView lv = view(cache, layer);
       if (launch_flush_bulk(lv, k_dev, v_dev, q_dev, n_tokens, t, nb, st) != cudaSuccess) return MIXKVQ_E_CUDA;
       cache->launches += cache->cfg.importance_mode == 1 ? 4 : 3;
+      cache->last_packed_writer = layer;
       cache->n_blocks[layer] += nb;
       t += nb * cache->R;
       continue;
@@ -269,6 +284,7 @@ int mixkvq_quantize_append(mixkvq_cache* cache, int layer, const void* k_dev, co
     LayerView lv = view(cache, layer);
     if (launch_append(lv, k_dev, v_dev, q_dev, n_tokens, t, m, st) != cudaSuccess) return MIXKVQ_E_CUDA;
     cache->launches += 1;
+    cache->last_packed_writer = kNoPackedWrite;
     cache->r[layer] += m;
     t += m;
   }
@@ -308,6 +324,7 @@ int mixkvq_decode_step(mixkvq_cache* cache, int layer, const void* k_dev, const 
     LayerView lv = view(cache, layer);
     if (launch_flush(lv, st) != cudaSuccess) return MIXKVQ_E_CUDA;
     cache->launches += 1;
+    cache->last_packed_writer = layer;
     cache->n_blocks[layer] += 1;
     cache->r[layer] = 0;
   }
@@ -341,6 +358,12 @@ int mixkvq_decode_attention_noalloc(mixkvq_cache* cache, int layer, const void* 
   }
   return run_attention(cache, layer, q_dev, out_dev, softmax_scale, static_cast<float*>(g_builtin_scratch_addr[dev]),
                        static_cast<cudaStream_t>(stream));
+}
+
+int mixkvq_cache_written_externally(mixkvq_cache* cache) {
+  if (!cache) return MIXKVQ_E_INVALID_ARG;
+  cache->last_packed_writer = kAllPacked;
+  return MIXKVQ_OK;
 }
 
 int mixkvq_set_attention_kernel(mixkvq_cache* cache, int kind) {

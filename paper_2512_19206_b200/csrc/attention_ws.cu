@@ -288,10 +288,20 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
   const long long cb = split_begin(total, gridDim.x, blockIdx.x), ce = split_begin(total, gridDim.x, blockIdx.x + 1);
 
   // Programmatic dependent launch: the grid may have been started while the kernel before it in the stream was still
-  // running.  Nothing above touches global memory; everything below does, so wait here for that kernel's results,
-  // and let the kernel after this one be started early in the same way.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // running.  Nothing above touches global memory.  dep_wait() waits for that kernel's results and lets the kernel after
+  // this one be started early in the same way; every thread calls it before its first access to global memory, with one
+  // exception: when the host knows that the kernel before this one did not write this layer's packed blocks
+  // (stage_early), the first staged copies of the packed units go out before the wait.  That is safe because a kernel
+  // of this library triggers its successor only after its own wait, so that everything two launches back is complete.
+  bool dep_waited = false;
+  auto dep_wait = [&]() {
+    if (!dep_waited) {
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+      asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+      dep_waited = true;
+    }
+  };
+  if (!lv.stage_early) dep_wait();
 
   uint32_t ring_stage = 0;        // ring stage of the next packed unit this pair consumes
   uint32_t ring_parity = 0;       // phase parity of that stage's barriers
@@ -368,10 +378,20 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
       issued += (int)enabled;
     };
     const uint32_t stage0 = ring_stage, parity0 = ring_parity;
+    // the logits warp's first block: its table entry and the head of its extras (the lists of promoted channels) are a
+    // chain of two dependent loads; they go out here, with the first copies
+    const char* extras = lv.extras + (size_t)s * lv.extras_stride;
+    const uint2* table = reinterpret_cast<const uint2*>(lv.table + (size_t)s * lv.table_stride);
+    uint2 pf_entry = make_uint2(0u, 0u);
+    uint4 pf_head = make_uint4(~0u, ~0u, ~0u, ~0u);
     if (!logits_role) {
 #pragma unroll 1
       for (int i = 0; i < kStages; ++i) issue((ring_stage + i) & (kStages - 1), i == 0);
+    } else if (n_pack > 0 && lv.stage_early) {
+      pf_entry = table[wb / U];
+      if (pf_entry.y & 0xFFFFu) pf_head = *reinterpret_cast<const uint4*>(extras + (size_t)pf_entry.x * 16);
     }
+    dep_wait();
 
     // ---- query of this stream: bf16 and fp16 tables (heads >= g are zero rows)
     {
@@ -457,14 +477,14 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
       }
 
       // ---- packed units
-      const char* extras = lv.extras + (size_t)s * lv.extras_stride;
-      const uint2* table = reinterpret_cast<const uint2*>(lv.table + (size_t)s * lv.table_stride);
       int bi = 0, u = 0;                     // block and unit inside it of the next unit to consume
-      uint2 pf_entry = make_uint2(0, 0);
       if (n_pack > 0) {
         bi = wb / U;
         u = wb - bi * U;
-        pf_entry = table[bi];
+        if (!lv.stage_early) {
+          pf_entry = table[bi];
+          if (pf_entry.y & 0xFFFFu) pf_head = *reinterpret_cast<const uint4*>(extras + (size_t)pf_entry.x * 16);
+        }
       }
       // B fragments of q for the base key tiles: head r, channels 16kt + {2t, 2t+1} and {2t+8, 2t+9}, times mult(kt)
       uint32_t bq[8][2];
@@ -496,6 +516,7 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
       while (done < n_pack) {
         // ---- a block: its table entry, its promoted channels' query entries
         const uint2 entry = pf_entry;
+        const uint4 head = pf_head;              // the first 16 bytes of the block's extras: up to 8 pairs of promoted channels
         if (bi + 1 < lv.n_blocks) pf_entry = table[bi + 1];
         const int n16 = entry.y & 0xFF, n4 = (entry.y >> 8) & 0xFF, n16p = (n16 + 1) >> 1;
         const char* ex = extras + (size_t)entry.x * 16;                       // the block's extras
@@ -519,15 +540,15 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
         };
         if (n16 > 0) {
           load_xa(exu);
-          auto gather_q = [&](int p) -> uint32_t {
+          auto gather_q = [&](int p, uint32_t word) -> uint32_t {       // pair p < 8: its two channel numbers are in `word`
             if (p >= n16p) return 0u;
-            const uint32_t ids = *reinterpret_cast<const uint16_t*>(ex + 2 * p);
+            const uint32_t ids = word >> (16 * (p & 1));
             const uint32_t c0 = ids & 0xFF, c1 = (ids >> 8) & 0xFF;
             const uint32_t lo = (c0 < 128) ? lds16(qrow_u32 + 2 * c0) : 0u, hi = (c1 < 128) ? lds16(qrow_u32 + 2 * c1) : 0u;
             return lo | (hi << 16);
           };
-          xb0 = gather_q(t);
-          xb1 = gather_q(t + 4);
+          xb0 = gather_q(t, (t & 2) ? head.y : head.x);
+          xb1 = gather_q(t + 4, (t & 2) ? head.w : head.z);
         }
         // the block's first 32 UINT4 channels (two tiles of eight pairs): B fragments (gathered fp16 query pairs) and, per
         // pair, where the two channels' scales sit in the scale table (byte offset of the half, 0xFFFF: no channel)
@@ -743,6 +764,8 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
         done += nu;
         u = 0;
         ++bi;
+        // the next block's channel lists (its table entry has arrived by now)
+        if (bi < lv.n_blocks && (pf_entry.y & 0xFFFFu)) pf_head = *reinterpret_cast<const uint4*>(extras + (size_t)pf_entry.x * 16);
       }
       if (gave_up && lane == 0) atomicOr(lv.status, (uint32_t)MIXKVQ_DEV_COPY_TIMEOUT);
     } else {
@@ -1033,31 +1056,24 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
     // ---- merge the pairs of the CTA, write the partial of (CTA, stream): the 16 threads that own a head add the pairs'
     // rows with the factors 2^(m_p - M).
     __syncthreads();
-    if (threadIdx.x < 128) {
-      const int h = threadIdx.x >> 4, c0 = threadIdx.x & 15;
+    for (int idx = threadIdx.x; idx < 256; idx += kThreads) {
+      const int h = idx >> 5, c = 4 * (idx & 31);          // head, first of the thread's four channels
       float M = -INFINITY, L = 0.f, f[kPairs];
 #pragma unroll
       for (int w = 0; w < kPairs; ++w) M = fmaxf(M, mS[w * 8 + h]);
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
       for (int w = 0; w < kPairs; ++w) {
         const float mw = mS[w * 8 + h];
-        f[w] = (mw == -INFINITY) ? 0.f : exp2f(mw - M);
+        f[w] = (mw == -INFINITY) ? 0.f : ex2_approx(mw - M);
         L += f[w] * lS[w * 8 + h];
+        const float4 o = *reinterpret_cast<const float4*>(smem + w * kPairBytes + (h * kMergeStride + c) * 4);
+        acc.x += f[w] * o.x; acc.y += f[w] * o.y; acc.z += f[w] * o.z; acc.w += f[w] * o.w;
       }
       float* part = ws + (size_t)(blockIdx.x + s) * kPartialFloats + h * 130;
-#pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        const int c = c0 + 16 * k;
-        float acc = 0.f;
-#pragma unroll
-        for (int w = 0; w < kPairs; ++w)
-          acc += f[w] * reinterpret_cast<const float*>(smem + w * kPairBytes)[h * kMergeStride + c];
-        part[2 + c] = acc;
-      }
-      if (c0 == 0) {
-        part[0] = M;
-        part[1] = L;
-      }
+      *reinterpret_cast<float2*>(part + 2 + c) = make_float2(acc.x, acc.y);
+      *reinterpret_cast<float2*>(part + 4 + c) = make_float2(acc.z, acc.w);
+      if (c == 0) *reinterpret_cast<float2*>(part) = make_float2(M, L);
     }
     if (seg < ce) {
       // another segment follows: its copies are staged into the rings that were just read

@@ -48,6 +48,9 @@ struct LayerView {
   // The attention kernel then stores them at residual slot r - 1 and adds |q| to the importance accumulator itself.
   const uint16_t* new_k;
   const uint16_t* new_v;
+  // decode attention may stage its first packed units before it waits for the kernel launched before it: set by the
+  // host when that kernel did not write this layer's packed blocks
+  int stage_early;
   // waits on staged copies and on hand-overs between warps give up after this many polls (0: the kernel's default)
   uint32_t wait_polls;
   // test hook for the give-up path: the barrier of every warp pair's first staged copy is armed for this many bytes

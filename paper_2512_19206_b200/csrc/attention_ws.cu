@@ -43,8 +43,9 @@ constexpr int kKeyMetaOff = 0;
 constexpr int kUnitOff = 512;
 // per-pair tables: key scales {s, -4s} (576) | key zero-point tiles (576) | value scales (320) | value zero-point tile (1088)
 constexpr int kKprepOff = 0, kZprepOff = 576, kSvpOff = 1152, kZvpOff = 1472, kPrepBytes = 2560;
-// hand-over of a unit's logits: 32 bytes per lane; one buffer per ring stage and one for unquantized units
-constexpr int kLBufBytes = 1024;
+// hand-over of a unit's logits: 32 bytes per lane, then 8 bytes per lane with the zero-point term of the unit's key
+// group; one buffer per ring stage and one for unquantized units
+constexpr int kLBufBytes = 1280, kLBufZeroOff = 1024;
 __host__ __device__ constexpr int pair_bytes(bool v4) {
   return kStages * stage_bytes(v4) + kPrepBytes + (kStages + 1) * kLBufBytes;
 }
@@ -505,6 +506,7 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
       const uint32_t kp_rd = ring_u32 + kPrepBase + kKprepOff + 16 * t;
       const uint32_t zp_rd = ring_u32 + kPrepBase + kZprepOff + 16 * t;
       const uint32_t lane16 = ring_u32 + lane * 16, lane32 = ring_u32 + kLBufBase + lane * 32;
+      const uint32_t lane8 = ring_u32 + kLBufBase + kLBufZeroOff + lane * 8;
       // byte offset inside the scale table of channel c's scale (half)
       auto scale_byte = [&](uint32_t c) -> uint32_t {
         const int kt = c >> 4, col = c & 15;
@@ -618,7 +620,7 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
             sts64(zp_wr + 16, zb, zb);
             __syncwarp();      // the tables written above are read by other lanes below
             // the zero-point term q . z of the group: a tile chain of its own (the tile's rows are equal, so are the rows
-            // of the result); it is the initial value of the unit's logit accumulators
+            // of the result), independent of the key tiles below; the partner adds it to the logits
 #pragma unroll
             for (int kt2 = 0; kt2 < 8; ++kt2) {
               const uint4 zz = lds128(zp_rd + 4 * zprep_word(kt2));
@@ -646,7 +648,7 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
                   const uint32_t code = (key_shift(kw[mt][j], kt) & mask) | four2;           // 4 + c * 2^(pos-8)
                   a[j] = hfma2_u(code, j < 2 ? kp.x : kp.z, j < 2 ? kp.y : kp.w);            // c * s * 2^(pos-8)
                 }
-                if (first && kt == 0) mma_f16_to(Sx[mt], a[0], a[1], a[2], a[3], bq[0][0], bq[0][1], zc[0], zc[1], zc[2], zc[3]);
+                if (first && kt == 0) mma_f16_to(Sx[mt], a[0], a[1], a[2], a[3], bq[0][0], bq[0][1], 0.f, 0.f, 0.f, 0.f);
                 else mma_f16(Sx[mt], a[0], a[1], a[2], a[3], bq[kt][0], bq[kt][1]);
               }
             }
@@ -755,6 +757,7 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
             const uint32_t lb = lane32 + ring_stage * kLBufBytes;
             sts128(lb, __float_as_uint(Sx[0][0]), __float_as_uint(Sx[0][1]), __float_as_uint(Sx[0][2]), __float_as_uint(Sx[0][3]));
             sts128(lb + 16, __float_as_uint(Sx[1][0]), __float_as_uint(Sx[1][1]), __float_as_uint(Sx[1][2]), __float_as_uint(Sx[1][3]));
+            sts64(lane8 + ring_stage * kLBufBytes, __float_as_uint(zc[0]), __float_as_uint(zc[1]));
             __syncwarp();
             mbar_arrive_one(lfull_u32 + ring_stage * 8u);
           }
@@ -906,6 +909,7 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
                              2 * ((((lane >> 4) * 144 + ((lane & 7) >> 1) * 4 + 2 * ((lane >> 3) & 1)) * 2) + (lane & 1));
       const uint32_t sv_rd = ring_u32 + kPrepBase + kSvpOff + t * 80;
       const uint32_t lane16 = ring_u32 + lane * 16, lane32 = ring_u32 + kLBufBase + lane * 32;
+      const uint32_t lane8 = ring_u32 + kLBufBase + kLBufZeroOff + lane * 8;
       const uint32_t vm_rd = ring_u32 + kUnitOff + 2048 + lane * (4 * VG);
 #pragma unroll 1
       for (int done = 0; done < n_pack; ++done) {
@@ -937,17 +941,20 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
         wait_or_give_up(lfull_u32 + ring_stage * 8u, ring_parity);
         const uint32_t lb = lane32 + ring_stage * kLBufBytes;
         const uint4 s0 = lds128(lb), s1 = lds128(lb + 16);
+        const uint2 zq = lds64(lane8 + ring_stage * kLBufBytes);
         const float sx[2][4] = {{__uint_as_float(s0.x), __uint_as_float(s0.y), __uint_as_float(s0.z), __uint_as_float(s0.w)},
                                 {__uint_as_float(s1.x), __uint_as_float(s1.y), __uint_as_float(s1.z), __uint_as_float(s1.w)}};
+        // logit = (sx + q . z) * scale: the zero-point term of the key group is the same for every token of the unit
+        const float zl0 = __uint_as_float(zq.x) * scale_log2e, zl1 = __uint_as_float(zq.y) * scale_log2e;
         // ---- online softmax (log2 domain); heads 2t, 2t+1; tokens r, r+8 of each m-tile.
         // The reference maximum only has to keep the probabilities inside the fp16 range: it is raised (to the true
         // maximum so far, with the accumulators rescaled) when a logit of this unit exceeds it by more than kMaxSlack.
         {
-          const float u0 = fmaxf(fmaxf(sx[0][0], sx[0][2]), fmaxf(sx[1][0], sx[1][2])) * scale_log2e;
-          const float u1 = fmaxf(fmaxf(sx[0][1], sx[0][3]), fmaxf(sx[1][1], sx[1][3])) * scale_log2e;
+          const float u0 = fmaf(fmaxf(fmaxf(sx[0][0], sx[0][2]), fmaxf(sx[1][0], sx[1][2])), scale_log2e, zl0);
+          const float u1 = fmaf(fmaxf(fmaxf(sx[0][1], sx[0][3]), fmaxf(sx[1][1], sx[1][3])), scale_log2e, zl1);
           if (__any_sync(0xffffffffu, (u0 > m0 + kMaxSlack) || (u1 > m1 + kMaxSlack))) raise_reference(u0, u1);
         }
-        const float c0 = -m0, c1 = -m1;
+        const float c0 = zl0 - m0, c1 = zl1 - m1;
         // P^T B fragments: [k-step][tokens 2t.. / 2t+8..], head r
         uint32_t Pt[2][2];
 #pragma unroll

@@ -50,7 +50,9 @@ enum {
 enum {
   MIXKVQ_DEV_EXTRAS_FULL = 1,         /* a block's promoted channels did not fit the extras arena: that
                                          block was not written and the layer's cache is invalid      */
-  MIXKVQ_DEV_COPY_TIMEOUT = 2         /* a bounded wait for a staged bulk copy gave up               */
+  MIXKVQ_DEV_COPY_TIMEOUT = 2         /* a bounded wait (for a staged bulk copy, or for the partner warp of a pair) ran out:
+                                         the warps concerned contributed nothing to that call's output, which is
+                                         therefore wrong (0 where no warp contributed); later calls are unaffected    */
 };
 
 typedef struct mixkvq_config {
@@ -146,7 +148,14 @@ int mixkvq_quantize_append(mixkvq_cache* cache, int layer, const void* k_dev, co
  * Numeric range: the tensor-core operands are fp16, so |q| must stay below 4094, a stored key scale below 2^11 and a
  * stored value scale below 2^9 (value ranges up to about 1500); beyond that the output overflows to inf or NaN.
  * The kernels are launched with programmatic stream serialization and wait on the device for all earlier work of
- * the stream before they touch global memory, so stream order holds as for any other launch. */
+ * the stream before they read q_dev or write anything, so stream order holds as for any other launch.  One access comes
+ * before that wait: the first packed blocks of the layer are requested early unless the call this library enqueued last
+ * on this handle wrote packed blocks of this layer (a flush; initialisation and reset count for all layers).  Cache
+ * memory is written through this library only; a caller that writes it by other means (restoring saved cache bytes with
+ * a kernel of its own, say) calls mixkvq_cache_written_externally before the next attention call.
+ * No wait inside the kernels is unbounded: a staged copy or a hand-over between two warps that has not arrived after
+ * 2^21 polls (each poll suspends the thread for up to about a microsecond: two seconds at most, milliseconds if the
+ * polls return at once) sets MIXKVQ_DEV_COPY_TIMEOUT and the call returns. */
 int mixkvq_decode_attention(mixkvq_cache* cache, int layer, const void* q_dev, float* out_dev, float softmax_scale,
                             void* workspace_dev, size_t workspace_bytes, void* stream);
 
@@ -169,8 +178,10 @@ int mixkvq_decode_step(mixkvq_cache* cache, int layer, const void* k_dev, const 
  *   - batch * n_kv_heads of the cache must be <= MIXKVQ_NOALLOC_MAX_STREAMS, else
  *     MIXKVQ_E_BUILTIN_SCRATCH is returned and nothing is launched.
  *   - The first call on each device looks up the device address of the scratch array (with that device
- *     current, which must be the device that owns the cache memory).  Make that first call before any
- *     stream capture begins.
+ *     current, which must be the device that owns the cache memory: MIXKVQ_E_INVALID_ARG otherwise).  Make
+ *     that first call before any stream capture begins, and from one thread: the look-up is not guarded
+ *     against concurrent first calls.  The address is kept for the life of the process; it does not
+ *     survive a cudaDeviceReset.
  *   - All calls on a device share the one array.  Nothing in it has to start at zero (every partial a
  *     call reads was written by that same call), so stale contents of earlier calls are harmless; but
  *     two calls whose kernels overlap on the GPU (different streams, no ordering between them) race on
@@ -178,6 +189,17 @@ int mixkvq_decode_step(mixkvq_cache* cache, int layer, const void* k_dev, const 
 #define MIXKVQ_NOALLOC_MAX_STREAMS 256
 int mixkvq_decode_attention_noalloc(mixkvq_cache* cache, int layer, const void* q_dev, float* out_dev,
                                     float softmax_scale, void* stream);
+
+/* Tells the library that cache memory was written by other means than its own calls since the last call on this
+ * handle: the next decode attention of every layer then waits for all earlier work of the stream before its first read. */
+int mixkvq_cache_written_externally(mixkvq_cache* cache);
+
+/* Test hook for the give-up path of the decode-attention kernel (fragment layout).  While extra_bytes > 0 (a multiple
+ * of 16), the barrier of the first staged copy of every warp pair is armed for extra_bytes more than the copy delivers,
+ * so it never completes, and every wait gives up after max_polls polls (0: the default): the call returns, the device
+ * status word carries MIXKVQ_DEV_COPY_TIMEOUT and the output rows are zero.  Nothing faults or hangs: the copies
+ * themselves are the normal ones.  (0, 0) restores normal operation. */
+int mixkvq_test_arm_copy_timeout(mixkvq_cache* cache, uint32_t extra_bytes, uint32_t max_polls);
 
 /* Selects the decode-attention kernel: 0 = tensor-core kernel (default), 1 = plain-ALU kernel
  * (kept for comparison; same results within tolerance, much slower), 2 = the tensor-core split kernel

@@ -12,13 +12,14 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.environ.get("MIXKVQ_LIB") or os.path.join(_HERE, "libmixkvq.so")
+LIB_PATH = os.path.join(_HERE, "libmixkvq.so")
 
 EXPORTS = [
     "mixkvq_cache_bytes", "mixkvq_cache_init", "mixkvq_cache_destroy", "mixkvq_cache_reset",
     "mixkvq_select_channels", "mixkvq_select_channels_raw", "mixkvq_quantize_append",
     "mixkvq_decode_attention", "mixkvq_decode_attention_noalloc", "mixkvq_decode_step", "mixkvq_set_attention_kernel", "mixkvq_query_status",
     "mixkvq_cache_describe", "mixkvq_launch_count", "mixkvq_status_string",
+    "mixkvq_cache_written_externally", "mixkvq_test_arm_copy_timeout",
 ]
 
 DEV_EXTRAS_FULL, DEV_COPY_TIMEOUT = 1, 2
@@ -71,6 +72,8 @@ def lib():
         L.mixkvq_decode_attention_noalloc.argtypes = [vp, i32, vp, vp, f32, vp]
         L.mixkvq_decode_step.argtypes = [vp, i32, vp, vp, vp, vp, f32, vp, C.c_size_t, vp]
         L.mixkvq_set_attention_kernel.argtypes = [vp, i32]
+        L.mixkvq_cache_written_externally.argtypes = [vp]
+        L.mixkvq_test_arm_copy_timeout.argtypes = [vp, C.c_uint32, C.c_uint32]
         L.mixkvq_query_status.argtypes = [vp, C.POINTER(i32), vp]
         L.mixkvq_cache_describe.argtypes = [vp, i32, C.POINTER(LayoutDesc)]
         L.mixkvq_launch_count.argtypes = [vp]
@@ -197,6 +200,12 @@ class Cache:
         _check(lib().mixkvq_select_channels(self.handle, layer, _ptr(tiers), _ptr(sal), _stream()),
                "mixkvq_select_channels")
         return tiers, sal
+
+    def written_externally(self):
+        _check(lib().mixkvq_cache_written_externally(self.handle), "mixkvq_cache_written_externally")
+
+    def test_arm_copy_timeout(self, extra_bytes: int, max_polls: int):
+        _check(lib().mixkvq_test_arm_copy_timeout(self.handle, extra_bytes, max_polls), "mixkvq_test_arm_copy_timeout")
 
     def set_attention_kernel(self, kind: int):
         _check(lib().mixkvq_set_attention_kernel(self.handle, kind), "mixkvq_set_attention_kernel")

@@ -25,6 +25,7 @@ struct mixkvq_cache {
   // it wrote that layer's packed blocks (a flush), kAllPacked after initialisation, a reset or a write from outside.
   // The next decode attention on such a layer waits for all earlier work before it reads anything.
   int last_packed_writer;
+  uint32_t test_extra_tx, test_wait_polls;   // mixkvq_test_arm_copy_timeout
 };
 
 namespace {
@@ -117,6 +118,8 @@ LayerView view(const mixkvq_cache* h, int layer) {
   v.sink = L + h->sink_off;     v.sink_stride = h->sink_stride;
   v.sink_len = h->cfg.sink_len; v.n_sink = h->n_sink[layer];
   v.status = reinterpret_cast<uint32_t*>(h->mem);
+  v.debug_extra_tx = h->test_extra_tx;
+  v.wait_polls = h->test_wait_polls;
   return v;
 }
 
@@ -184,6 +187,7 @@ int mixkvq_cache_init(const mixkvq_config* cfg, void* cache_dev, size_t bytes, v
   h->attn_kind = 0;
   h->launches = 0;
   h->last_packed_writer = kAllPacked;
+  h->test_extra_tx = h->test_wait_polls = 0;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&h->n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
@@ -329,7 +333,9 @@ int mixkvq_decode_step(mixkvq_cache* cache, int layer, const void* k_dev, const 
     cache->r[layer] = 0;
   }
   cache->r[layer] += 1;        // the attention kernel stores the token at slot r - 1 and accumulates |q|
-  return run_attention(cache, layer, q_dev, out_dev, softmax_scale, static_cast<float*>(workspace_dev), st, k_dev, v_dev);
+  const int rc = run_attention(cache, layer, q_dev, out_dev, softmax_scale, static_cast<float*>(workspace_dev), st, k_dev, v_dev);
+  if (rc != MIXKVQ_OK) cache->r[layer] -= 1;      // nothing was enqueued: the token is not part of the layer
+  return rc;
 }
 
 // ---- decode attention with the split partials in storage compiled into the library (no allocation)
@@ -350,6 +356,10 @@ int mixkvq_decode_attention_noalloc(mixkvq_cache* cache, int layer, const void* 
   if (cache->n_blocks[layer] == 0 && cache->r[layer] == 0 && cache->n_sink[layer] == 0) return MIXKVQ_E_EMPTY;
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MIXKVQ_E_CUDA;
+  // the scratch array of the CURRENT device is used: it must be the device that holds the cache memory
+  cudaPointerAttributes attr;
+  if (cudaPointerGetAttributes(&attr, cache->mem) != cudaSuccess) return MIXKVQ_E_CUDA;
+  if (attr.type != cudaMemoryTypeDevice || attr.device != dev) return MIXKVQ_E_INVALID_ARG;
   if (!g_builtin_scratch_addr[dev]) {
     // once per device, with that device current: resolve the array's address on this device
     void* p = nullptr;
@@ -363,6 +373,13 @@ int mixkvq_decode_attention_noalloc(mixkvq_cache* cache, int layer, const void* 
 int mixkvq_cache_written_externally(mixkvq_cache* cache) {
   if (!cache) return MIXKVQ_E_INVALID_ARG;
   cache->last_packed_writer = kAllPacked;
+  return MIXKVQ_OK;
+}
+
+int mixkvq_test_arm_copy_timeout(mixkvq_cache* cache, uint32_t extra_bytes, uint32_t max_polls) {
+  if (!cache || (extra_bytes & 15u)) return MIXKVQ_E_INVALID_ARG;
+  cache->test_extra_tx = extra_bytes;
+  cache->test_wait_polls = max_polls;
   return MIXKVQ_OK;
 }
 

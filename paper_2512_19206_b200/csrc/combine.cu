@@ -54,7 +54,8 @@ combine_kernel(const float* __restrict__ ws, float* __restrict__ out, int g, int
     }
     M = Mn;
   }
-  out[((size_t)b * Hq + hk * g + h) * kD + c] = o / l;
+  // l == 0 only when every split gave up (its partial is then m = -inf, l = 0, o = 0 and the status word says so)
+  out[((size_t)b * Hq + hk * g + h) * kD + c] = l > 0.f ? o / l : 0.f;
 }
 
 cudaError_t launch_combine(const float* ws, float* out, int g, int Hkv, int Hq, int mode, int n,
@@ -106,7 +107,7 @@ combine2_kernel(const float* __restrict__ ws, float* __restrict__ out, int g, in
     l += f * p[1];
     o += f * p[2 + c];
   }
-  out[((size_t)b * Hq + hk * g + h) * kD + c] = o / l;
+  out[((size_t)b * Hq + hk * g + h) * kD + c] = l > 0.f ? o / l : 0.f;
 }
 
 cudaError_t launch_combine2(const float* ws, float* out, int g, int Hkv, int Hq, int S, int n1, long long units1,

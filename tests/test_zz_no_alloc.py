@@ -5,8 +5,9 @@ is sized once at start-up, or a host program whose language binding has no devic
 library offers one entry point that keeps the split partials of decode attention in a scratch array
 compiled into the library.  This test calls it through the C ABI twice in a row (the second call on a
 different, shorter cache, so stale partials of the first call are still lying in the array) and checks each
-result against the ordinary entry point within the attention tolerance of the other GPU tests.  It runs last
-so that a failure here cannot hide another test's result.
+result against the ordinary entry point: both run the same kernels on the same grid, so the outputs must be equal
+bit for bit (and within the attention tolerance of the other GPU tests, which follows).  It runs last so that a
+failure here cannot hide another test's result.
 """
 import ctypes as C
 
@@ -51,7 +52,19 @@ def test_noalloc_entry_matches_workspace_entry_on_two_calls_in_a_row(binding):
         torch.cuda.synchronize()
         assert torch.isfinite(got).all()
         assert float((got - want).abs().max()) <= ATTN_TOL
+        assert torch.equal(got, want)
         assert cache.status() == 0
+
+
+def test_noalloc_entry_with_the_plain_alu_kernel(binding):
+    # the comparison kernel lays its partials out differently in the same array
+    w, cache = _filled_cache(binding, "qwen7b", 2, 3 * 128 + 50, W.P24)
+    cache.set_attention_kernel(1)
+    qd = W.decode_query(w, 0, 0).cuda()
+    want = cache.decode_attention(0, qd, W.softmax_scale())
+    got = cache.decode_attention_noalloc(0, qd, W.softmax_scale())
+    assert torch.equal(got, want)
+    assert cache.status() == 0
 
 
 def test_noalloc_entry_rejects_more_streams_than_its_scratch_holds(binding):

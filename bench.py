@@ -2,11 +2,17 @@
 """Benchmark of the MixKVQ decode hot path on B200.
 
 A step is one decode step of the whole path over all layers: for every layer `mixkvq_decode_step`, i.e. the
-append of the new token (with the scoring + quantize + pack flush once per R steps) fused with decode attention.  The cache is pre-filled to the configured context with seeded synthetic
-tensors; all timed inputs are resident in HBM.  Prints one JSON line (rank 0).
+append of the new token (with the scoring + quantize + pack flush once per R steps) fused with decode attention.
+The cache is pre-filled to the configured context with seeded synthetic tensors; all timed inputs are resident
+in HBM.  Prints one JSON line (rank 0).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config qwen7b|llama8b|tiny|...] [--impl reference]
 
+The line leads with the qwen2.5-7b shape (batch 8, 32768 cached tokens, 28 layers).  It also carries the separate
+timings of the step's parts (attention, append, the step that flushes, the amortised step) and, under `configs`,
+the decode-attention kernel on the other workload shapes (a few layers each).
+`--gpus N` without launcher variables starts N ranks itself (one per GPU, independent replicas; only the measured
+times are reduced, with MAX); under torchrun it takes rank and world size from the environment.
 `--impl reference` times the CPU oracle (as it stands) on a bounded sample of the same workload.
 """
 from __future__ import annotations
@@ -25,10 +31,12 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 from paper_2512_19206_b200 import workloads as W  # noqa: E402
-from paper_2512_19206_b200.replicas import dist_env, max_over_ranks, job_tokens_per_s  # noqa: E402
+from paper_2512_19206_b200.replicas import dist_env, max_over_ranks, job_tokens_per_s, spawn_local_ranks  # noqa: E402
 
 METRIC = "decode-attn us/step (all layers) over mixed-precision KV"
 PREFILL_CHUNK = 4096
+SPLIT_KERNEL = ("attention_ws_kernel", "attention_ws.cu")
+TILE_KERNEL = ("attention_tc_kernel", "attention_tc.cu")
 
 
 def measured_peaks():
@@ -40,18 +48,21 @@ def measured_peaks():
 
 
 # ---------------------------------------------------------------------------------------------- CPU oracle leg
+def oracle_stream(w):
+    from oracle import mixkvq_oracle as O
+    return O.OracleStream(g=w.g, R=w.residual_len, G=w.group_size, score_bits=w.score_bits, tau_bf16=w.tau_bf16,
+                          tau_u4=w.tau_u4)
+
+
 def oracle_sample(w, n_streams=2, reps=3):
     """Times the oracle's attention on `n_streams` (layer, b, hk) streams at the full context.
 
     Returns (seconds per stream-step, description).  Inputs come from the same generator (CPU)."""
-    from oracle import mixkvq_oracle as O
-    import numpy as np
     secs = []
     for i in range(n_streams):
         layer, hk = i % w.n_layers, i % w.n_kv_heads
         one = W.small(w, batch=1)
-        st = O.OracleStream(g=w.g, R=w.residual_len, G=w.group_size, score_bits=w.score_bits, tau_bf16=w.tau_bf16,
-                            tau_u4=w.tau_u4)
+        st = oracle_stream(w)
         t = 0
         while t < w.tokens:
             n = min(PREFILL_CHUNK, w.tokens - t)
@@ -68,6 +79,23 @@ def oracle_sample(w, n_streams=2, reps=3):
     return statistics.mean(secs), (f"oracle attention on {n_streams} of {w.n_layers * w.batch * w.n_kv_heads} "
                                    f"(layer, batch, kv-head) streams at T={w.tokens}, {reps} repetitions each, "
                                    "scaled linearly to all streams")
+
+
+def oracle_flush_ms(w, n_blocks=6):
+    """Mean time of one oracle flush (scoring, tiering, quantization of one R-token window of one stream)."""
+    one = W.small(w, batch=1)
+    st = oracle_stream(w)
+    R = w.residual_len
+    k, v, q = W.tokens(one, 0, 0, (n_blocks + 1) * R)
+    kf, vf, qf = k[0, 0].float().numpy(), v[0, 0].float().numpy(), q[0, :w.g].float().numpy()
+    st.append_many(kf[:R], vf[:R], qf[:, :R])                      # the window is full now
+    secs = []
+    for b in range(1, n_blocks + 1):
+        t0 = time.perf_counter()
+        st.append_many(kf[b * R:b * R + 1], vf[b * R:b * R + 1], qf[:, b * R:b * R + 1])   # flushes the full window first
+        secs.append(time.perf_counter() - t0)
+        st.append_many(kf[b * R + 1:(b + 1) * R], vf[b * R + 1:(b + 1) * R], qf[:, b * R + 1:(b + 1) * R])
+    return statistics.mean(secs) * 1e3
 
 
 def oracle_threads():
@@ -94,11 +122,12 @@ def run_reference(args, w):
     n_streams = w.n_layers * w.batch * w.n_kv_heads
     us = per_stream * n_streams * 1e6
     line = {
-        "impl": "reference", "metric": METRIC, "value": us, "unit": "us/step", "n_gpus": args.gpus,
+        "impl": "reference", "metric": METRIC, "value": us, "unit": "us/step", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": workload_config(w, args.importance_mode),
-        "cpu_baseline": {"value": us, "unit": "us/step", "cores": oracle_threads(), "kind": "oracle", "sample": desc},
+        "cpu_baseline": {"value": us, "unit": "us/step", "cores": oracle_threads(), "kind": "oracle",
+                         "impl": f"numpy, {oracle_threads()} BLAS threads", "sample": desc},
         "e2e": {"value": us, "unit": "us/step", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "tokens_per_s": w.batch / (us * 1e-6),
     }
@@ -125,7 +154,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                                          "-lms", "50", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+                                          "-lms", "20", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
         except Exception:
             self.proc = None
 
@@ -153,15 +182,27 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
-def prefill(cache, w, dev):
-    """Fills every layer to the configured context; returns the device time (ms) spent inside the bulk
+def make_cache(binding, w, args, dev, extra_tokens):
+    cfg = binding.make_config(w.n_layers, w.batch, w.n_q_heads, w.n_kv_heads, w.tokens + extra_tokens,
+                              residual_len=w.residual_len, group_size=w.group_size, tau_bf16=w.tau_bf16,
+                              tau_u4=w.tau_u4, score_bits=w.score_bits, block_layout=args.layout,
+                              importance_mode=args.importance_mode, sink_len=args.sink_len, v_bits=args.v_bits,
+                              budget_bf16=args.budget_bf16, budget_u4=args.budget_u4,
+                              extras_budget_bytes=((w.tokens + extra_tokens) // w.residual_len + 3) * 8192
+                              if w.score_bits == 4 else 0)
+    return binding.Cache(cfg, device=dev)
+
+
+def prefill(cache, w, dev, t_from=0, t_to=None):
+    """Appends tokens [t_from, t_to) to every layer in chunks; returns the device time (ms) spent inside the bulk
     mixkvq_quantize_append calls alone (input generation excluded)."""
+    t_to = w.tokens if t_to is None else t_to
     ms = 0.0
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for layer in range(w.n_layers):
-        t = 0
-        while t < w.tokens:
-            n = min(PREFILL_CHUNK, w.tokens - t)
+        t = t_from
+        while t < t_to:
+            n = min(PREFILL_CHUNK, t_to - t)
             k, v, q = W.tokens(w, layer, t, n, device=dev)
             e0.record()
             cache.quantize_append(layer, k, v, q)
@@ -175,7 +216,6 @@ def prefill(cache, w, dev):
 
 def tier_mix(cache, w):
     """Mean (n16, n4) per block over all layers/streams, from the block tables."""
-    import numpy as np
     n16 = n4 = nb = 0
     for layer in range(w.n_layers):
         d = cache.describe(layer)
@@ -214,6 +254,79 @@ def algorithmic_bytes_per_layer(w, n16, n4, r, tokens_packed, n_partials, v_bits
     return streams * per_stream + 2 * n_partials * g * (D + 2) * 4
 
 
+def n_split_partials(w, d0, dev):
+    """Partials written per launch = CTAs of the split kernel: two per SM, a multiple of the stream count when there
+    are fewer streams than CTA slots (the library's grid rule), each CTA one partial per stream it touches."""
+    streams = w.batch * w.n_kv_heads
+    units = (d0.n_blocks * w.residual_len // 32 + (d0.residual_tokens + 31) // 32) * streams
+    n_sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    n_part = min(2 * n_sms, units)
+    return n_part // streams * streams if n_part > streams else n_part + streams
+
+
+def time_loop(fn, reps):
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(reps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def attention_timings(cache, w, qs, out, scale):
+    """(split kernel ms per launch, attention + combine us per layer) at the cache's current state."""
+    def all_layers():
+        for layer in range(w.n_layers):
+            cache.decode_attention(layer, qs[layer], scale, out=out[layer])
+    reps = max(3, min(20, int(200 / max(1, w.n_layers))))
+    cache.set_attention_kernel(2)
+    all_layers()
+    kern_ms = time_loop(all_layers, reps) / w.n_layers
+    cache.set_attention_kernel(0)
+    all_layers()
+    attn_us = time_loop(all_layers, reps) / w.n_layers * 1e3
+    return kern_ms, attn_us
+
+
+def roofline_entry(cache, w, dev, args, kern_ms):
+    d0 = cache.describe(0)
+    n16, n4 = tier_mix(cache, w)
+    tokens_packed = d0.n_blocks * w.residual_len
+    alg = algorithmic_bytes_per_layer(w, n16, n4, d0.residual_tokens, tokens_packed, n_split_partials(w, d0, dev), args.v_bits)
+    peak, peak_src = measured_peaks()
+    achieved = alg / (kern_ms * 1e-3) / 1e9
+    return n16, n4, tokens_packed, alg, achieved, peak, peak_src
+
+
+def other_config(binding, dev, args, name, w, label, contexts=None):
+    """The decode-attention kernel on another workload shape, a few layers of it: one entry per context length."""
+    entries = []
+    contexts = contexts or [w.tokens]
+    cache = make_cache(binding, W.small(w, tokens=max(contexts)), args, dev, 2 * w.residual_len + 8)
+    scale = W.softmax_scale()
+    out = torch.empty((w.n_layers, w.batch, w.n_q_heads, 128), dtype=torch.float32, device=dev)
+    done = 0
+    for T in contexts:
+        prefill(cache, w, dev, done, T)
+        done = T
+        qs = [W.decode_query(w, layer, 0, device=dev) for layer in range(w.n_layers)]
+        kern_ms, attn_us = attention_timings(cache, w, qs, out, scale)
+        n16, n4, tokens_packed, alg, achieved, peak, _ = roofline_entry(cache, w, dev, args, kern_ms)
+        entries.append({
+            "workload": label, "shape": f"B={w.batch} Hq={w.n_q_heads} Hkv={w.n_kv_heads} T={T} G={w.group_size}",
+            "layers_measured": w.n_layers, "layers_of_model": W.CONFIGS[name].n_layers,
+            "kernel_us": kern_ms * 1e3, "algorithmic_bytes": alg, "achieved_gbs": achieved, "frac": achieved / peak,
+            "attention_us_per_layer": attn_us,
+            "attention_us_per_step_all_layers": attn_us * W.CONFIGS[name].n_layers,
+            "tier_mix_mean": {"n16": n16, "n4": n4}, "device_status": cache.status()})
+    cache.close()
+    del cache
+    torch.cuda.empty_cache()
+    return entries
+
+
 def run_gpu(args, w):
     rank, world, local = dist_env()
     torch.cuda.set_device(local)
@@ -228,25 +341,20 @@ def run_gpu(args, w):
         dist.barrier()
     binding.lib()
 
-    K, Wm = args.steps, args.warmup
+    K, Wm, R = args.steps, args.warmup, w.residual_len
     n_steps = Wm + K + 4
-    cfg = binding.make_config(w.n_layers, w.batch, w.n_q_heads, w.n_kv_heads, w.tokens + n_steps + 2 * w.residual_len,
-                              residual_len=w.residual_len, group_size=w.group_size, tau_bf16=w.tau_bf16,
-                              tau_u4=w.tau_u4, score_bits=w.score_bits, block_layout=args.layout,
-                              importance_mode=args.importance_mode, sink_len=args.sink_len, v_bits=args.v_bits,
-                              budget_bf16=args.budget_bf16, budget_u4=args.budget_u4,
-                              extras_budget_bytes=((w.tokens + n_steps) // w.residual_len + 3) * 8192 if w.score_bits == 4 else 0)
-    cache = binding.Cache(cfg, device=dev)
+    cache = make_cache(binding, w, args, dev, n_steps + 4 * R + 64)
     prefill_ms = prefill(cache, w, dev)
     assert cache.status() == 0
     scale = W.softmax_scale()
 
     # decode-step inputs, resident in HBM: [layer][step] -> (k, v, q) of one token
+    n_in = n_steps + 2 * R + 40
     steps_in = []
     for layer in range(w.n_layers):
-        k, v, q = W.tokens(w, layer, w.tokens, n_steps, device=dev)
+        k, v, q = W.tokens(w, layer, w.tokens, n_in, device=dev)
         steps_in.append([(k[:, :, i:i + 1].contiguous(), v[:, :, i:i + 1].contiguous(), q[:, :, i:i + 1].contiguous())
-                         for i in range(n_steps)])
+                         for i in range(n_in)])
     out = torch.empty((w.n_layers, w.batch, w.n_q_heads, 128), dtype=torch.float32, device=dev)
 
     def step(i):
@@ -277,25 +385,13 @@ def run_gpu(args, w):
     torch.cuda.profiler.stop()
     ms = e0.elapsed_time(e1)
     launches = cache.launch_count() - launches0
-    flushes = sum(1 for i in range(Wm, Wm + K) if (w.tokens + i) % w.residual_len == 0) * w.n_layers
+    flushes = sum(1 for i in range(Wm, Wm + K) if (w.tokens + i) % R == 0) * w.n_layers
 
-    # ---- dominant kernel alone (split kernel, no combine), same state: average launch duration
-    d0 = cache.describe(0)
-    cache.set_attention_kernel(2)
-    qs = [steps_in[layer][Wm + K][2].view(w.batch, w.n_q_heads, 128) for layer in range(w.n_layers)]
+    # ---- dominant kernel alone (split kernel, no combine), and attention + combine, same state
+    nxt = Wm + K                                    # next unused decode-step input
+    qs = [steps_in[layer][nxt][2].view(w.batch, w.n_q_heads, 128) for layer in range(w.n_layers)]
+    kern_ms, attn_us_layer = attention_timings(cache, w, qs, out, scale)
     reps = max(3, min(20, int(200 / max(1, w.n_layers))))
-    for layer in range(w.n_layers):
-        cache.decode_attention(layer, qs[layer], scale, out=out[layer])
-    torch.cuda.synchronize()
-    k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    k0.record()
-    for _ in range(reps):
-        for layer in range(w.n_layers):
-            cache.decode_attention(layer, qs[layer], scale, out=out[layer])
-    k1.record()
-    torch.cuda.synchronize()
-    kern_ms = k0.elapsed_time(k1) / (reps * w.n_layers)
-    cache.set_attention_kernel(0)
     # ---- attention + combine for all layers from one CUDA graph (fixed state): launch gaps removed
     g = torch.cuda.CUDAGraph()
     s = torch.cuda.Stream()
@@ -309,21 +405,42 @@ def run_gpu(args, w):
                 cache.decode_attention(layer, qs[layer], scale, out=out[layer])
     torch.cuda.synchronize()
     g.replay()
-    torch.cuda.synchronize()
-    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    g0.record()
-    for _ in range(reps):
-        g.replay()
-    g1.record()
-    torch.cuda.synchronize()
-    graph_us = g0.elapsed_time(g1) / reps * 1e3
+    graph_us = time_loop(g.replay, reps) * 1e3
     clocks = sampler.stop() if rank == 0 else None
+    n16, n4, tokens_packed, alg, achieved, peak, peak_src = roofline_entry(cache, w, dev, args, kern_ms)
+
+    # ---- the parts of the step on their own: the plain append of one token (no flush), and the step on which the
+    # residual window is full, so that the append first scores, quantizes and packs it (once every R steps)
+    def append_all(i):
+        for layer in range(w.n_layers):
+            k, v, q = steps_in[layer][i]
+            cache.quantize_append(layer, k, v, q)
+
+    def window_fill():
+        return cache.describe(0).residual_tokens
+
+    plain = []
+    while window_fill() != R and len(plain) < 4:      # a few plain appends, timed one step at a time
+        i = nxt
+        plain.append(time_loop(lambda: append_all(i), 1) * 1e3)
+        nxt += 1
+    while window_fill() != R:                         # advance (untimed) until the window is full
+        append_all(nxt)
+        nxt += 1
+    i = nxt
+    flush_step_us = time_loop(lambda: append_all(i), 1) * 1e3      # flush + append on every layer
+    nxt += 1
+    while len(plain) < 4:
+        i = nxt
+        plain.append(time_loop(lambda: append_all(i), 1) * 1e3)
+        nxt += 1
+    append_us = statistics.median(plain)
 
     # ---- end to end through the C ABI with host buffers: H2D of the step's inputs, D2H of its outputs
     n_e2e = min(K, 16)
-    hk = torch.stack([torch.stack([steps_in[l][Wm + i][0] for l in range(w.n_layers)]) for i in range(n_e2e)]).cpu().pin_memory()
-    hv = torch.stack([torch.stack([steps_in[l][Wm + i][1] for l in range(w.n_layers)]) for i in range(n_e2e)]).cpu().pin_memory()
-    hq = torch.stack([torch.stack([steps_in[l][Wm + i][2] for l in range(w.n_layers)]) for i in range(n_e2e)]).cpu().pin_memory()
+    hk = torch.stack([torch.stack([steps_in[l][nxt + i][0] for l in range(w.n_layers)]) for i in range(n_e2e)]).cpu().pin_memory()
+    hv = torch.stack([torch.stack([steps_in[l][nxt + i][1] for l in range(w.n_layers)]) for i in range(n_e2e)]).cpu().pin_memory()
+    hq = torch.stack([torch.stack([steps_in[l][nxt + i][2] for l in range(w.n_layers)]) for i in range(n_e2e)]).cpu().pin_memory()
     hout = torch.empty(out.shape, dtype=torch.float32).pin_memory()
     dk, dv, dq = [torch.empty(x.shape[1:], dtype=x.dtype, device=dev) for x in (hk, hv, hq)]
     barrier()
@@ -346,18 +463,8 @@ def run_gpu(args, w):
             dist.destroy_process_group()
         return
 
-    n16, n4 = tier_mix(cache, w)
-    tokens_packed = d0.n_blocks * w.residual_len
-    units = (tokens_packed // 32 + (d0.residual_tokens + 31) // 32) * w.batch * w.n_kv_heads
-    # partials written per launch = CTAs of the split kernel: two per SM, a multiple of the stream count when there are
-    # fewer streams than CTA slots (the library's grid rule), each CTA one partial per stream it touches
-    streams = w.batch * w.n_kv_heads
-    n_sms = torch.cuda.get_device_properties(dev).multi_processor_count
-    n_part = min(2 * n_sms, units)
-    n_part = n_part // streams * streams if n_part > streams else n_part + streams
-    alg = algorithmic_bytes_per_layer(w, n16, n4, d0.residual_tokens, tokens_packed, n_part, args.v_bits)
-    peak, peak_src = measured_peaks()
     achieved = alg / (kern_ms * 1e-3) / 1e9
+    attn_us = attn_us_layer * w.n_layers
     line = {
         "metric": METRIC, "value": us, "unit": "us/step", "n_gpus": world, "steps": K, "warmup": Wm,
         "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
@@ -365,6 +472,13 @@ def run_gpu(args, w):
         "arithmetic": "2/4-bit codes and bf16 metadata expanded to fp16 tensor-core operands, fp32 accumulate and softmax",
         "config": workload_config(w, args.importance_mode),
         "tokens_per_s": job_tokens_per_s(w.batch, world, us),
+        "step_parts": {
+            "note": "all layers; `value` is the fused call (append inside the attention kernel) on steps without a flush",
+            "attention_us": attn_us, "attention_graph_us": graph_us,
+            "append_us": append_us, "flush_step_us": flush_step_us,
+            "amortised_us_per_step": attn_us + append_us + (flush_step_us - append_us) / R,
+            "fused_amortised_us_per_step": us + (flush_step_us - append_us) / R,
+            "flush_every_steps": R},
         "attention_graph_us_per_step": graph_us,
         "prefill_quantize": {"ms": prefill_ms, "tokens_per_s": w.n_layers * w.batch * w.tokens / (prefill_ms * 1e-3),
                              "input_gb_per_s": w.n_layers * w.batch * w.tokens * 256 * (2 * w.n_kv_heads + w.n_q_heads)
@@ -376,22 +490,42 @@ def run_gpu(args, w):
                      # the committed counters were taken on the two-tier mix (no UINT4 tier): other mixes have none
                      "traffic": None if (w.tau_u4 < w.tau_bf16 or args.v_bits != 2 or args.sink_len or args.budget_bf16 +
                                          args.budget_u4) else measured_traffic(
-                         *(("attention_tc_kernel", "attention_tc.cu") if args.layout == 1 else
-                           ("attention_ws_kernel", "attention_ws.cu")), w.group_size, tokens_packed,
+                         *(TILE_KERNEL if args.layout == 1 else SPLIT_KERNEL), w.group_size, tokens_packed,
                          w.batch * w.n_kv_heads),
                      "peak_source": peak_src,
-                     "kernel": "attention_tc_kernel" if args.layout == 1 else "attention_ws_kernel", "kernel_us": kern_ms * 1e3, "algorithmic_bytes": alg},
+                     "kernel": (TILE_KERNEL if args.layout == 1 else SPLIT_KERNEL)[0], "kernel_us": kern_ms * 1e3,
+                     "kernel_us_note": "mean over back-to-back launches of the split kernel alone (one per layer); each "
+                                       "launch starts behind its predecessor with programmatic dependent launch, so set-up "
+                                       "and the first requests of a launch overlap the tail of the one before",
+                     "algorithmic_bytes": alg},
         "e2e": {"value": e2e_us, "unit": "us/step", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "steps": n_e2e},
         "gpu_launches": int(launches),
         "device_status": status,
         "clocks": clocks,
     }
+    cache.close()
+    del cache, steps_in
+    torch.cuda.empty_cache()
+    if world == 1 and not args.no_configs and args.config == "qwen7b" and not args.tokens and not args.layers:
+        cfgs = []
+        cfgs += other_config(binding, dev, args, "tiny", W.CONFIGS["tiny"], "config 1: tiny (L2-resident)")
+        l8 = W.small(W.CONFIGS["llama8b"], n_layers=4)
+        cfgs += other_config(binding, dev, args, "llama8b", W.small(l8, **W.P24), "config 3: llama-3.1-8b, 2-bit base")
+        cfgs += other_config(binding, dev, args, "llama8b", W.small(l8, **W.P4BASE), "config 3: llama-3.1-8b, 4-bit base")
+        cfgs += other_config(binding, dev, args, "qwen32b", W.small(W.CONFIGS["qwen32b"], n_layers=3),
+                             "config 4: qwen2.5-32b (3 distinct layers of 64)")
+        cfgs += other_config(binding, dev, args, "longcot", W.small(W.CONFIGS["longcot"], n_layers=4),
+                             "config 5: long-CoT stream", contexts=[8192, 32768, 65536, 131072])
+        line["configs"] = cfgs
     if world == 1 and not args.no_cpu_baseline:
         sec, desc = oracle_sample(w, n_streams=8, reps=5)
         n_streams = w.n_layers * w.batch * w.n_kv_heads
         line["cpu_baseline"] = {"value": sec * n_streams * 1e6, "unit": "us/step", "cores": oracle_threads(),
-                                "kind": "oracle", "sample": desc}
+                                "kind": "oracle", "impl": f"numpy, {oracle_threads()} BLAS threads", "sample": desc,
+                                "flush_ms_per_block": oracle_flush_ms(w),
+                                "flush_note": "one stream's window of R tokens: scoring, tiering, quantization (oracle); "
+                                              "the GPU's flush_step_us covers all layers x streams"}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -400,7 +534,7 @@ def run_gpu(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=128)
+    ap.add_argument("--steps", type=int, default=64)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", default="qwen7b", choices=sorted(W.CONFIGS))
     ap.add_argument("--group-size", type=int, default=None)
@@ -415,11 +549,18 @@ def main():
     ap.add_argument("--layers", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-configs", action="store_true", help="skip the other workload shapes")
     ap.add_argument("--preset", default=None, choices=["P24", "P27", "P4BASE"],
                     help="threshold preset: two tiers (default), three tiers, or 4-bit base precision")
     ap.add_argument("--layout", type=int, default=0, choices=[0, 1],
                     help="0: fragment layout + mma.sync attention (default), 1: tile layout + tcgen05 attention")
     args = ap.parse_args()
+    launched = "RANK" in os.environ and "WORLD_SIZE" in os.environ
+    if args.impl == "ours" and args.gpus > 1 and not launched:
+        # no launcher: start the ranks here, one per GPU (independent replicas of the workload)
+        sys.exit(spawn_local_ranks(args.gpus, [sys.executable, os.path.abspath(__file__)] + sys.argv[1:]))
+    if launched and args.impl == "ours" and int(os.environ["WORLD_SIZE"]) != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but the launcher started {os.environ['WORLD_SIZE']} ranks")
     w = W.CONFIGS[args.config]
     over = {}
     if args.group_size:

@@ -30,3 +30,41 @@ def max_over_ranks(values, device="cpu"):
 def job_tokens_per_s(batch_per_replica: int, world: int, us_per_step: float) -> float:
     """Whole-job decode throughput: every replica emits one token per sequence per step."""
     return world * batch_per_replica / (us_per_step * 1e-6)
+
+
+def free_port() -> int:
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def spawn_local_ranks(n: int, argv, env=None, timeout=None) -> int:
+    """Starts `argv` n times on this node, rank i with RANK = LOCAL_RANK = i, WORLD_SIZE = n and a rendezvous on
+    127.0.0.1, waits for all of them and returns the largest exit code.  The children inherit stdout and stderr, so
+    the one line rank 0 prints is the job's line.  If a rank fails, the others are stopped."""
+    import subprocess
+    import time
+    port = free_port()
+    procs = []
+    for rank in range(n):
+        e = dict(os.environ if env is None else env)
+        e.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen(list(argv), env=e))
+    t0, rc = time.monotonic(), 0
+    live = list(procs)
+    while live:
+        for p in list(live):
+            code = p.poll()
+            if code is not None:
+                live.remove(p)
+                rc = max(rc, abs(code))
+                if code != 0:
+                    for other in live:
+                        other.terminate()
+        if timeout is not None and time.monotonic() - t0 > timeout:
+            for other in live:
+                other.kill()
+            return max(rc, 124)
+        time.sleep(0.05)
+    return rc

@@ -40,3 +40,27 @@ def test_two_gloo_replicas_report_the_slowest_rank():
 def test_single_process_is_the_identity():
     assert replicas.dist_env()[1] >= 1
     assert replicas.max_over_ranks([3.0, 4.5]) == [3.0, 4.5]
+
+
+def test_the_benchmark_launcher_starts_one_rank_per_gpu(tmp_path):
+    """`bench.py --gpus N` without launcher variables starts its N ranks with replicas.spawn_local_ranks; here the same
+    function starts two gloo ranks of a stub step on CPU: one line comes back, from rank 0, with the slowest rank's time."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    stub = os.path.join(root, "tests", "replica_stub.py")
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    env["PYTHONPATH"] = root + os.pathsep + env.get("PYTHONPATH", "")
+    code = ("import sys; from paper_2512_19206_b200 import replicas; "
+            f"sys.exit(replicas.spawn_local_ranks(2, [sys.executable, {stub!r}] + sys.argv[1:], timeout=120))")
+    res = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, timeout=180)
+    assert res.returncode == 0, res.stderr
+    lines = [ln for ln in res.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["us_per_step"] == 150.0 and line["kernel_us"] == 7.0
+    assert line["tokens_per_s"] == 2 * 8 / 150e-6
+    # a failing rank makes the job fail
+    res = subprocess.run([sys.executable, "-c", code, "3"], env=env, capture_output=True, text=True, timeout=180)
+    assert res.returncode == 3

@@ -19,6 +19,9 @@ What each function follows:
 * ``pack_*``                              the storage layout (Appendix D "Storage Layout" gives
                                           the three stores; the bit positions are this repository's).
 * ``effective_bits`` / ``fp16_cache_bytes``  B_eff of Appendix C; the footprint example of Section 1.
+* ``rope``                                the rotary embedding that Appendix D puts before the scores ("saliency
+                                          evaluation is performed post-transformation"): keys and queries are
+                                          rotated, then appended.
 
 Precision: scores and attention in fp64.  The quantizer runs the fixed IEEE fp32 sequence
 (subtract, divide by the stored bf16 scale, round half to even, clamp) because its integer result
@@ -314,6 +317,29 @@ class OracleStream:
         if return_probs:
             return o.astype(np.float32), p
         return o.astype(np.float32)
+
+
+def rope(x, cos, sin):
+    """Rotary position embedding of bf16-valued rows x [..., n, D] at the n positions whose table rows are
+    cos, sin [n, D/2] (float32, supplied by the caller: the oracle takes no trigonometric function).
+
+    Pairing of the channels: (i, i + D/2), the "rotate-half" convention of the Llama and Qwen families.  With
+    c = cos[p, i], s = sin[p, i]:   y[i] = x[i] c - x[i + D/2] s,   y[i + D/2] = x[i + D/2] c + x[i] s.
+    Arithmetic: every product and the one sum are single IEEE fp32 operations (round to nearest, no fused
+    multiply-add); the result is rounded to bf16 (nearest, ties to even).  Returned as float32 holding bf16 values.
+    Appendix D fixes only that scores and keys are taken after this rotation; the order of the operations is this
+    repository's, stated here so that the rotated bf16 bits are reproducible."""
+    x = np.asarray(x, np.float32)
+    cos = np.asarray(cos, np.float32)
+    sin = np.asarray(sin, np.float32)
+    h = x.shape[-1] // 2
+    x1, x2 = x[..., :h], x[..., h:]
+    a = (x1 * cos).astype(np.float32)
+    b = (x2 * sin).astype(np.float32)
+    c = (x2 * cos).astype(np.float32)
+    d = (x1 * sin).astype(np.float32)
+    y = np.concatenate([(a - b).astype(np.float32), (c + d).astype(np.float32)], axis=-1)
+    return bf16_rne(y)
 
 
 def unquantized_attention(q, K, V, scale):

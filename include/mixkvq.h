@@ -167,6 +167,24 @@ int mixkvq_decode_attention(mixkvq_cache* cache, int layer, const void* q_dev, f
 int mixkvq_decode_step(mixkvq_cache* cache, int layer, const void* k_dev, const void* v_dev, const void* q_dev,
                        float* out_dev, float softmax_scale, void* workspace_dev, size_t workspace_bytes, void* stream);
 
+/* Appendix D ("saliency evaluation is performed post-transformation"): for models with rotary position embeddings the
+ * scores, the stored keys and the attention all use rotated queries and keys.  These two calls rotate before they
+ * append.  k_dev [B, Hkv, n_tokens, 128] and q_dev [B, Hq, n_tokens, 128] (bf16) are rotated IN PLACE: afterwards q_dev
+ * holds the rotated queries that mixkvq_decode_attention takes, k_dev the keys that were stored.  v_dev is not touched.
+ *   cos_dev, sin_dev: float tables [n_positions, 64] of the caller's angles (row p = position p, entry i the angle of
+ *   channel pair (i, i + 64): the "rotate-half" pairing); token j of the call uses row pos0 + j.  The caller owns them.
+ *   Arithmetic: y[i] = x[i] c - x[i+64] s, y[i+64] = x[i+64] c + x[i] s, every product and the sum one fp32 operation
+ *   rounded to nearest, the result rounded to bf16 (ties to even).  The cache then equals, byte for byte, that of
+ *   mixkvq_quantize_append on tensors rotated in this way.
+ * Errors as for mixkvq_quantize_append / mixkvq_decode_step; on MIXKVQ_E_CAPACITY nothing was rotated. */
+int mixkvq_rope_append(mixkvq_cache* cache, int layer, void* k_dev, const void* v_dev, void* q_dev, const float* cos_dev,
+                       const float* sin_dev, int pos0, int n_tokens, void* stream);
+/* The same for one decode step: rotates the step's k_dev [B, Hkv, 1, 128] and q_dev [B, Hq, 1, 128] with table row `pos`,
+ * then does what mixkvq_decode_step does. */
+int mixkvq_rope_decode_step(mixkvq_cache* cache, int layer, void* k_dev, const void* v_dev, void* q_dev,
+                            const float* cos_dev, const float* sin_dev, int pos, float* out_dev, float softmax_scale,
+                            void* workspace_dev, size_t workspace_bytes, void* stream);
+
 /* (The paper has no counterpart of this entry point; it exists for integration reasons only.)
  * Same computation and same results as mixkvq_decode_attention, for callers that have no way to hand
  * over a workspace: code that runs inside a serving engine's pre-sized memory pool, a plugin that may

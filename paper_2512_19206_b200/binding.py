@@ -19,7 +19,7 @@ EXPORTS = [
     "mixkvq_select_channels", "mixkvq_select_channels_raw", "mixkvq_quantize_append",
     "mixkvq_decode_attention", "mixkvq_decode_attention_noalloc", "mixkvq_decode_step", "mixkvq_set_attention_kernel", "mixkvq_query_status",
     "mixkvq_cache_describe", "mixkvq_launch_count", "mixkvq_status_string",
-    "mixkvq_cache_written_externally", "mixkvq_test_arm_copy_timeout",
+    "mixkvq_cache_written_externally", "mixkvq_test_arm_copy_timeout", "mixkvq_rope_append", "mixkvq_rope_decode_step",
 ]
 
 DEV_EXTRAS_FULL, DEV_COPY_TIMEOUT = 1, 2
@@ -72,6 +72,8 @@ def lib():
         L.mixkvq_decode_attention_noalloc.argtypes = [vp, i32, vp, vp, f32, vp]
         L.mixkvq_decode_step.argtypes = [vp, i32, vp, vp, vp, vp, f32, vp, C.c_size_t, vp]
         L.mixkvq_set_attention_kernel.argtypes = [vp, i32]
+        L.mixkvq_rope_append.argtypes = [vp, i32, vp, vp, vp, vp, vp, i32, i32, vp]
+        L.mixkvq_rope_decode_step.argtypes = [vp, i32, vp, vp, vp, vp, vp, i32, vp, f32, vp, C.c_size_t, vp]
         L.mixkvq_cache_written_externally.argtypes = [vp]
         L.mixkvq_test_arm_copy_timeout.argtypes = [vp, C.c_uint32, C.c_uint32]
         L.mixkvq_query_status.argtypes = [vp, C.POINTER(i32), vp]
@@ -180,6 +182,22 @@ class Cache:
             out = torch.empty((q.shape[0], q.shape[1], 128), dtype=torch.float32, device=q.device)
         _check(lib().mixkvq_decode_step(self.handle, layer, _ptr(k), _ptr(v), _ptr(q), _ptr(out), float(scale),
                                         _ptr(self.workspace), self.workspace.numel(), _stream()), "mixkvq_decode_step")
+        return out
+
+    def rope_append(self, layer, k, v, q, cos, sin, pos0):
+        """Rotates k [B,Hkv,n,128] and q [B,Hq,n,128] (bf16) IN PLACE with rows pos0.. of the float32 tables cos, sin
+        [n_positions, 64], then appends them as quantize_append does."""
+        assert cos.dtype == torch.float32 and sin.dtype == torch.float32
+        _check(lib().mixkvq_rope_append(self.handle, layer, _ptr(k), _ptr(v), _ptr(q), _ptr(cos), _ptr(sin), int(pos0),
+                                        k.shape[2], _stream()), "mixkvq_rope_append")
+
+    def rope_decode_step(self, layer, k, v, q, cos, sin, pos, scale, out=None):
+        """One decode step with the rotation of k and q (in place) in front: see decode_step."""
+        if out is None:
+            out = torch.empty((q.shape[0], q.shape[1], 128), dtype=torch.float32, device=q.device)
+        _check(lib().mixkvq_rope_decode_step(self.handle, layer, _ptr(k), _ptr(v), _ptr(q), _ptr(cos), _ptr(sin), int(pos),
+                                             _ptr(out), float(scale), _ptr(self.workspace), self.workspace.numel(),
+                                             _stream()), "mixkvq_rope_decode_step")
         return out
 
     def decode_attention_noalloc(self, layer, q, scale, out=None):

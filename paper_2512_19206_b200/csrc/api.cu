@@ -338,6 +338,44 @@ int mixkvq_decode_step(mixkvq_cache* cache, int layer, const void* k_dev, const 
   return rc;
 }
 
+int mixkvq_rope_append(mixkvq_cache* cache, int layer, void* k_dev, const void* v_dev, void* q_dev, const float* cos_dev,
+                       const float* sin_dev, int pos0, int n_tokens, void* stream) {
+  if (!cache || !k_dev || !v_dev || !q_dev || !cos_dev || !sin_dev || layer < 0 || layer >= cache->cfg.n_layers ||
+      n_tokens < 1 || pos0 < 0)
+    return MIXKVQ_E_INVALID_ARG;
+  if (!aligned16(k_dev) || !aligned16(v_dev) || !aligned16(q_dev) || !aligned16(cos_dev) || !aligned16(sin_dev))
+    return MIXKVQ_E_ALIGNMENT;
+  const long long have = (long long)cache->n_sink[layer] + (long long)cache->n_blocks[layer] * cache->R + cache->r[layer];
+  if (have + n_tokens > cache->cfg.max_tokens) return MIXKVQ_E_CAPACITY;      // nothing is rotated either
+  if (launch_rope(k_dev, q_dev, cos_dev, sin_dev, cache->cfg.batch, cache->cfg.n_kv_heads, cache->cfg.n_q_heads, n_tokens,
+                  pos0, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return MIXKVQ_E_CUDA;
+  cache->launches += 1;
+  cache->last_packed_writer = kNoPackedWrite;
+  return mixkvq_quantize_append(cache, layer, k_dev, v_dev, q_dev, n_tokens, stream);
+}
+
+int mixkvq_rope_decode_step(mixkvq_cache* cache, int layer, void* k_dev, const void* v_dev, void* q_dev,
+                            const float* cos_dev, const float* sin_dev, int pos, float* out_dev, float softmax_scale,
+                            void* workspace_dev, size_t workspace_bytes_given, void* stream) {
+  if (!cache || !k_dev || !v_dev || !q_dev || !cos_dev || !sin_dev || !out_dev || !workspace_dev || layer < 0 ||
+      layer >= cache->cfg.n_layers || pos < 0)
+    return MIXKVQ_E_INVALID_ARG;
+  if (!aligned16(k_dev) || !aligned16(v_dev) || !aligned16(q_dev) || !aligned16(cos_dev) || !aligned16(sin_dev) ||
+      !aligned16(out_dev) || !aligned16(workspace_dev))
+    return MIXKVQ_E_ALIGNMENT;
+  if (workspace_bytes_given < workspace_bytes(cache->S)) return MIXKVQ_E_BUFFER_TOO_SMALL;
+  const long long have = (long long)cache->n_sink[layer] + (long long)cache->n_blocks[layer] * cache->R + cache->r[layer];
+  if (have + 1 > cache->cfg.max_tokens) return MIXKVQ_E_CAPACITY;
+  if (launch_rope(k_dev, q_dev, cos_dev, sin_dev, cache->cfg.batch, cache->cfg.n_kv_heads, cache->cfg.n_q_heads, 1, pos,
+                  static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return MIXKVQ_E_CUDA;
+  cache->launches += 1;
+  cache->last_packed_writer = kNoPackedWrite;
+  return mixkvq_decode_step(cache, layer, k_dev, v_dev, q_dev, out_dev, softmax_scale, workspace_dev, workspace_bytes_given,
+                            stream);
+}
+
 // ---- decode attention with the split partials in storage compiled into the library (no allocation)
 namespace {
 constexpr size_t kBuiltinScratchBytes =

@@ -184,6 +184,8 @@ cudaError_t launch_append(const LayerView& lv, const void* k, const void* v, con
                           int m, cudaStream_t stream);
 cudaError_t launch_sink_append(const LayerView& lv, const void* k, const void* v, int n_tokens, int t0, int m,
                                cudaStream_t stream);
+cudaError_t launch_rope(void* k, void* q, const float* cos_t, const float* sin_t, int B, int Hkv, int Hq, int n_tokens,
+                        int pos0, cudaStream_t stream);
 cudaError_t launch_flush(const LayerView& lv, cudaStream_t stream);
 cudaError_t launch_flush_bulk(const LayerView& lv, const void* k, const void* v, const void* q, int n_tokens, int t0,
                               int nb, cudaStream_t stream);

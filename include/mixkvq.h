@@ -48,8 +48,12 @@ enum {
 
 /* bits of the sticky device status word */
 enum {
-  MIXKVQ_DEV_EXTRAS_FULL = 1,         /* a block's promoted channels did not fit the extras arena: that
-                                         block was not written and the layer's cache is invalid      */
+  MIXKVQ_DEV_EXTRAS_FULL = 1,         /* a block's promoted channels did not fit the stream's extras arena.  The
+                                         block's base part is written as usual, but nothing goes to the arena and the
+                                         block's table entry records no promoted channel (n16 = n4 = 0): its BF16-tier
+                                         channels then read as 0 and its UINT4 channels lose their high plane, so the
+                                         layer's attention is wrong from that block on, until the cache is reset
+                                         (with a larger extras_budget_bytes).  Earlier blocks are unaffected            */
   MIXKVQ_DEV_COPY_TIMEOUT = 2         /* a bounded wait (for a staged bulk copy, or for the partner warp of a pair) ran out:
                                          the warps concerned contributed nothing to that call's output, which is
                                          therefore wrong (0 where no warp contributed); later calls are unaffected    */

@@ -24,8 +24,9 @@ __host__ __device__ inline uint32_t flush_extras_bytes(const LayerView& lv, int 
 }
 
 // Bulk append, between the two passes: one thread per stream walks the new blocks in order, gives each its offset in
-// the promoted-channel arena and advances the arena pointer; a block that no longer fits loses its promotions and
-// the status word says so (the same rule as for a single flush).
+// the promoted-channel arena and advances the arena pointer.  A block that no longer fits gets nothing in the arena and
+// a table entry without promoted channels (its base part is still written; its BF16-tier channels then read as 0 and
+// its UINT4 channels lose their high plane), and the status word says so: the same rule as for a single flush.
 __global__ void bulk_prefix_kernel(LayerView lv, int nb) {
   const int s = blockIdx.x * blockDim.x + threadIdx.x;
   if (s >= lv.B * lv.Hkv) return;
@@ -299,7 +300,7 @@ flush_kernel(LayerView lv, BulkSrc src) {
       if ((uint64_t)off16 * 16 + need > lv.extras_budget) {
         atomicOr(lv.status, (uint32_t)MIXKVQ_DEV_EXTRAS_FULL);
         n16 = 0;
-        n4 = 0;      // nothing is written to the arena; the block is invalid and the status says so
+        n4 = 0;      // nothing goes to the arena and the entry records no promoted channel; the status word says so
       } else {
         *used = off16 + need / 16;
       }

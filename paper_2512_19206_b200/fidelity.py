@@ -44,7 +44,9 @@ def tier_counts(cache: "B.Cache", layer: int):
 
 
 def reference_attention(k: torch.Tensor, v: torch.Tensor, q: torch.Tensor, scale: float) -> torch.Tensor:
-    """Unquantized decode attention in fp32: k, v [B, Hkv, T, D] bf16, q [B, Hq, D] bf16 -> [B, Hq, D] fp32."""
+    """Unquantized decode attention in fp32: k, v [B, Hkv, T, D] bf16, q [B, Hq, D] bf16 -> [B, Hq, D] fp32.
+    A yardstick for this tool's error columns only (plain PyTorch, no part of the decode path); the tests tie it and
+    the tool's rows to the CPU oracle."""
     b, hkv, t, d = k.shape
     g = q.shape[1] // hkv
     qf = q.float().view(b, hkv, g, d)
@@ -120,12 +122,14 @@ def default_pairs():
     inf = 1e30
     pairs = [("uniform 2-bit keys", inf, inf, 2, 0)]
     pairs += [(f"two tiers, tau_bf16 = {t:g}", t, inf, 2, 0) for t in (13.0, 6.5, 3.25)]
-    pairs += [("three tiers (6.5, 4.0)", 6.5, 4.0, 2, 0), ("three tiers (6.5, 2.0)", 6.5, 2.0, 2, 0)]
+    pairs += [(f"three tiers ({W.P27['tau_bf16']:g}, {W.P27['tau_u4']:g})", W.P27["tau_bf16"], W.P27["tau_u4"], 2, 0),
+              ("three tiers (6.5, 2.0)", 6.5, 2.0, 2, 0)]
     pairs += [("error-only salience, tau_bf16 = 6.5", 6.5, inf, 2, 2)]
     pairs += [("fixed budget: 4 BF16", inf, inf, 2, 0, {"budget_bf16": 4}),
               ("fixed budget: 4 BF16 + 24 UINT4", inf, inf, 2, 0, {"budget_bf16": 4, "budget_u4": 24}),
               ("two tiers (6.5) + 32 sink tokens", 6.5, inf, 2, 0, {"sink_len": 32})]
-    pairs += [("4-bit base (2.17)", W.P4BASE["tau_bf16"], -1.0, 4, 0), ("all keys bf16 (values 2-bit)", -1.0, -1.0, 2, 0)]
+    pairs += [(f"4-bit base ({W.P4BASE['tau_bf16']:g})", W.P4BASE["tau_bf16"], -1.0, 4, 0),
+              ("all keys bf16 (values 2-bit)", -1.0, -1.0, 2, 0)]
     return pairs
 
 

@@ -43,3 +43,37 @@ def test_more_key_bits_mean_less_attention_error():
     assert all_bf16[0] == 16.0
     # rms error of the attention output: promoting the salient channels helps, unquantized keys help more
     assert uniform[4] > two_tier[4] > all_bf16[4] > 0.0
+
+
+@pytest.mark.gpu
+def test_a_sweep_row_equals_the_oracles_numbers():
+    """One setting of the sweep (three tiers) on a small workload: the tier counts and the key bit-width equal the
+    oracle's exactly, the error columns equal the oracle's own (its quantized attention against its unquantized
+    attention, both fp64) within twice the attention tolerance."""
+    import numpy as np
+    import gpu_util as U
+    from oracle import mixkvq_oracle as O
+    from paper_2512_19206_b200 import build, binding
+    build.build()
+    binding.lib()
+    w = W.small(W.CONFIGS["qwen7b"], n_layers=1, batch=1, tokens=1024 + 77, **W.P27)
+    n_queries = 3
+    beff, n16, n4, worst, rms = F.measure(w, w.tau_bf16, w.tau_u4, n_queries=n_queries)
+    k, v, q = [x.cpu() for x in W.tokens(w, 0, 0, w.tokens, device="cuda")]      # the tool draws its inputs on the GPU
+    orc = U.oracle_streams(w, 0, k, v, q)
+    blocks = [b for st in orc.values() for b in st.blocks]
+    o16 = float(np.mean([(b.tiers == O.TIER_BF16).sum() for b in blocks]))
+    o4 = float(np.mean([(b.tiers == O.TIER_U4).sum() for b in blocks]))
+    assert (n16, n4) == (o16, o4)
+    assert beff == pytest.approx(O.effective_bits(o16, o4, 128 - o16 - o4))
+    errs = []
+    for i in range(n_queries):
+        qd = U.f32(W.decode_query(w, 0, i, device="cuda"))
+        for (b, hk), st in orc.items():
+            qh = qd[b, hk * w.g:(hk + 1) * w.g]
+            quant = st.attention(qh, W.softmax_scale())
+            exact = O.unquantized_attention(qh, U.f32(k[b, hk]), U.f32(v[b, hk]), W.softmax_scale())
+            errs.append(np.abs(np.asarray(quant, np.float64) - np.asarray(exact, np.float64)))
+    errs = np.stack(errs)
+    assert abs(worst - float(errs.max())) <= 4e-3
+    assert abs(rms - float(np.sqrt((errs ** 2).mean()))) <= 4e-3

@@ -117,3 +117,38 @@ def test_long_cot_stream_checkpoints(binding):
     lists = {tuple(np.flatnonzero(b.tiers == O.TIER_BF16)) for b in orc[streams[0]].blocks}
     assert len(lists) > 4
     assert cache.status() == 0
+
+
+def test_long_cot_streamed_decode_steps(binding):
+    """The long chain-of-thought stream as it is produced: from 32K cached tokens, 2100 fused decode steps (one token
+    per step through mixkvq_decode_step, 16 flushes with drifting outlier channels).  Two sampled streams follow on the
+    CPU oracle token by token: attention at 16 seeded steps within the tolerance, all their bytes equal at the end."""
+    w = W.small(W.CONFIGS["longcot"], n_layers=1, batch=2, tokens=32768, **W.P24)
+    n_steps = 2100
+    streams = [(0, 3), (1, 0)]
+    cache = U.make_cache(binding, w, max_tokens=w.tokens + n_steps + 256)
+    orc = {s: U.oracle_stream(w) for s in streams}
+    t = 0
+    while t < w.tokens:
+        k, v, q = W.tokens(w, 0, t, CHUNK, device="cuda")
+        cache.quantize_append(0, k, v, q)
+        for (b, hk), st in orc.items():
+            st.append_many(U.f32(k[b, hk]), U.f32(v[b, hk]), U.f32(q[b, hk * w.g:(hk + 1) * w.g]))
+        t += CHUNK
+    checked = set(np.random.default_rng(0x5EED).choice(n_steps, size=16, replace=False).tolist()) | {n_steps - 1}
+    k, v, q = W.tokens(w, 0, w.tokens, n_steps, device="cuda")
+    kc, vc, qc = U.f32(k), U.f32(v), U.f32(q)
+    flushes0 = {s: st.n_flushes for s, st in orc.items()}
+    scale = W.softmax_scale()
+    worst = 0.0
+    for i in range(n_steps):
+        out = cache.decode_step(0, k[:, :, i:i + 1].contiguous(), v[:, :, i:i + 1].contiguous(), q[:, :, i:i + 1].contiguous(), scale)
+        for (b, hk), st in orc.items():
+            st.append(kc[b, hk, i], vc[b, hk, i], qc[b, hk * w.g:(hk + 1) * w.g, i])
+        if i in checked:
+            ref = {(b, hk): st.attention(qc[b, hk * w.g:(hk + 1) * w.g, i], scale) for (b, hk), st in orc.items()}
+            worst = max(worst, U.max_abs_err(w, out, ref))
+    assert worst <= ATTN_TOL, worst
+    assert all(st.n_flushes - flushes0[s] >= 16 for s, st in orc.items())
+    U.compare_regions(cache, 0, w, orc)
+    assert cache.status() == 0

@@ -404,6 +404,24 @@ def test_extras_arena_exhaustion_sets_status(binding):
     cache = U.make_cache(binding, w, extras_budget_bytes=2048)     # room for about one block's promoted channels
     cache.quantize_append(0, k.cuda(), v.cuda(), q.cuda())
     assert cache.status() & binding.DEV_EXTRAS_FULL
+    # the stated behaviour: blocks that fitted equal the oracle's; a block that did not fit has a table entry without
+    # promoted channels, nothing of it in the arena, and its base part written as usual
+    oracle = U.oracle_streams(w, 0, k, v, q)
+    st = oracle[(0, 0)]
+    got = cache.stream_regions(0, 0)
+    want = O.pack_stream(st)
+    assert got["base"] == want["base"]
+    fitted = 0
+    for i in range(len(st.blocks)):
+        entry = got["table"][8 * i:8 * i + 8]
+        if entry == want["table"][8 * i:8 * i + 8] and fitted == i:
+            fitted += 1
+        else:
+            assert entry[4] == 0 and entry[5] == 0                 # n16 = n4 = 0
+    assert 1 <= fitted < len(st.blocks)
+    used = 16 * int.from_bytes(got["state"][1028:1032], "little")      # the arena holds the fitted blocks only
+    assert 0 < used <= 2048 and used < len(want["extras"])
+    assert got["extras"] == want["extras"][:used]
     cache.reset()
     assert cache.status() == 0 and cache.describe(0).n_blocks == 0
 

@@ -19,6 +19,8 @@ What each function follows:
 * ``pack_*``                              the storage layout (Appendix D "Storage Layout" gives
                                           the three stores; the bit positions are this repository's).
 * ``effective_bits`` / ``fp16_cache_bytes``  B_eff of Appendix C; the footprint example of Section 1.
+* ``causal_attention``                    Eq. 1 for the prompt (the prefill phase of Section 4.2): every position attends
+                                          to itself and the positions before it, full precision, fp64.
 * ``rope``                                the rotary embedding that Appendix D puts before the scores ("saliency
                                           evaluation is performed post-transformation"): keys and queries are
                                           rotated, then appended.
@@ -349,6 +351,25 @@ def unquantized_attention(q, K, V, scale):
     p = np.exp(logits)
     p /= p.sum(axis=1, keepdims=True)
     return p @ np.asarray(V, np.float64)
+
+
+def causal_attention(q, K, V, scale):
+    """Eq. 1 over a prompt, position by position: q [g, L, D], K, V [L, D] (bf16-valued) -> [g, L, D] float64.
+    Position i sees keys and values 0..i: the plain definition, one softmax per row, nothing blocked or reused.
+    The prompt's keys and values are attended in full precision (Section 4.2: quantization happens after the
+    prefill computation; the cache the prompt leaves behind is that of append_many)."""
+    q = np.asarray(q, np.float64)
+    K = np.asarray(K, np.float64)
+    V = np.asarray(V, np.float64)
+    g, L, _ = q.shape
+    out = np.zeros((g, L, V.shape[1]), np.float64)
+    for i in range(L):
+        logits = (q[:, i] @ K[:i + 1].T) * float(scale)
+        logits -= logits.max(axis=1, keepdims=True)
+        p = np.exp(logits)
+        p /= p.sum(axis=1, keepdims=True)
+        out[:, i] = p @ V[:i + 1]
+    return out
 
 
 # --------------------------------------------------------------------------------------------

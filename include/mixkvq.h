@@ -171,6 +171,17 @@ int mixkvq_decode_attention(mixkvq_cache* cache, int layer, const void* q_dev, f
 int mixkvq_decode_step(mixkvq_cache* cache, int layer, const void* k_dev, const void* v_dev, const void* q_dev,
                        float* out_dev, float softmax_scale, void* workspace_dev, size_t workspace_bytes, void* stream);
 
+/* The prefill phase of Section 4.2 for one layer: causal attention of the prompt over itself in full precision (Eq. 1,
+ * position i sees positions 0..i), then the prompt's keys and values go into the cache exactly as
+ * mixkvq_quantize_append(n_tokens) would put them (complete windows quantized, the last 1..R tokens in the residual
+ * window).  The layer must be empty (MIXKVQ_E_UNSUPPORTED otherwise: a later chunk would have to attend to a
+ * dequantized cache).
+ *   k_dev, v_dev [B, Hkv, n_tokens, 128], q_dev [B, Hq, n_tokens, 128] bf16 (post-RoPE)  ->  out_dev [B, Hq, n_tokens, 128] float
+ * The attention runs on the tcgen05 tensor cores (bf16 products for the logits, fp16 probabilities and values for the
+ * output, fp32 accumulation in tensor memory); values must stay inside the fp16 range. */
+int mixkvq_prefill(mixkvq_cache* cache, int layer, const void* k_dev, const void* v_dev, const void* q_dev, int n_tokens,
+                   float* out_dev, float softmax_scale, void* stream);
+
 /* Appendix D ("saliency evaluation is performed post-transformation"): for models with rotary position embeddings the
  * scores, the stored keys and the attention all use rotated queries and keys.  These two calls rotate before they
  * append.  k_dev [B, Hkv, n_tokens, 128] and q_dev [B, Hq, n_tokens, 128] (bf16) are rotated IN PLACE: afterwards q_dev

@@ -14,7 +14,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libmixkvq.so")
-SOURCES = ["api.cu", "append.cu", "rope.cu", "select.cu", "flush.cu", "combine.cu", "attention_simt.cu", "attention_ws.cu",
+SOURCES = ["api.cu", "append.cu", "rope.cu", "prefill.cu", "select.cu", "flush.cu", "combine.cu", "attention_simt.cu", "attention_ws.cu",
            "attention_tc.cu"]
 FLAGS = ["-Xcompiler", "-fPIC", "-O3", "-std=c++17", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
          "--fmad=true"]

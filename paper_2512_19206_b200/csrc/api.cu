@@ -198,7 +198,7 @@ int mixkvq_cache_init(const mixkvq_config* cfg, void* cache_dev, size_t bytes, v
   if (cudaMemsetAsync(h->mem, 0, kHeaderBytes, st) != cudaSuccess) { delete h; return MIXKVQ_E_CUDA; }
   for (int l = 0; l < cfg->n_layers; ++l)
     if (zero_layer_state(h, l, st) != MIXKVQ_OK) { delete h; return MIXKVQ_E_CUDA; }
-  if (attention_ws_setup() != cudaSuccess || attention_tc_setup() != cudaSuccess) { delete h; return MIXKVQ_E_CUDA; }
+  if (attention_ws_setup() != cudaSuccess || attention_tc_setup() != cudaSuccess || prefill_attention_setup() != cudaSuccess) { delete h; return MIXKVQ_E_CUDA; }
   *out = h;
   return MIXKVQ_OK;
 }
@@ -336,6 +336,23 @@ int mixkvq_decode_step(mixkvq_cache* cache, int layer, const void* k_dev, const 
   const int rc = run_attention(cache, layer, q_dev, out_dev, softmax_scale, static_cast<float*>(workspace_dev), st, k_dev, v_dev);
   if (rc != MIXKVQ_OK) cache->r[layer] -= 1;      // nothing was enqueued: the token is not part of the layer
   return rc;
+}
+
+int mixkvq_prefill(mixkvq_cache* cache, int layer, const void* k_dev, const void* v_dev, const void* q_dev, int n_tokens,
+                   float* out_dev, float softmax_scale, void* stream) {
+  if (!cache || !k_dev || !v_dev || !q_dev || !out_dev || layer < 0 || layer >= cache->cfg.n_layers || n_tokens < 1)
+    return MIXKVQ_E_INVALID_ARG;
+  if (!aligned16(k_dev) || !aligned16(v_dev) || !aligned16(q_dev) || !aligned16(out_dev)) return MIXKVQ_E_ALIGNMENT;
+  // the prompt attends to itself only: the layer must be empty
+  if (cache->n_blocks[layer] != 0 || cache->r[layer] != 0 || cache->n_sink[layer] != 0) return MIXKVQ_E_UNSUPPORTED;
+  if (n_tokens > cache->cfg.max_tokens) return MIXKVQ_E_CAPACITY;
+  if (launch_prefill_attention(q_dev, k_dev, v_dev, out_dev, cache->cfg.batch, cache->cfg.n_q_heads, cache->cfg.n_kv_heads,
+                               n_tokens, softmax_scale, reinterpret_cast<uint32_t*>(cache->mem), cache->test_wait_polls,
+                               static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return MIXKVQ_E_CUDA;
+  cache->launches += 1;
+  cache->last_packed_writer = kNoPackedWrite;
+  return mixkvq_quantize_append(cache, layer, k_dev, v_dev, q_dev, n_tokens, stream);
 }
 
 int mixkvq_rope_append(mixkvq_cache* cache, int layer, void* k_dev, const void* v_dev, void* q_dev, const float* cos_dev,

@@ -41,7 +41,7 @@ def free_port() -> int:
 
 def spawn_local_ranks(n: int, argv, env=None, timeout=None) -> int:
     """Starts `argv` n times on this node, rank i with RANK = LOCAL_RANK = i, WORLD_SIZE = n and a rendezvous on
-    127.0.0.1, waits for all of them and returns the largest exit code.  The children inherit stdout and stderr, so
+    127.0.0.1, waits for all of them and returns 0 if all ended with 0, else the exit code of the first rank seen failing.  The children inherit stdout and stderr, so
     the one line rank 0 prints is the job's line.  If a rank fails, the others are stopped."""
     import subprocess
     import time
@@ -53,18 +53,20 @@ def spawn_local_ranks(n: int, argv, env=None, timeout=None) -> int:
         procs.append(subprocess.Popen(list(argv), env=e))
     t0, rc = time.monotonic(), 0
     live = list(procs)
+    stopped = set()
     while live:
         for p in list(live):
             code = p.poll()
             if code is not None:
                 live.remove(p)
-                rc = max(rc, abs(code))
-                if code != 0:
+                if code != 0 and rc == 0 and p.pid not in stopped:
+                    rc = abs(code)
                     for other in live:
+                        stopped.add(other.pid)
                         other.terminate()
         if timeout is not None and time.monotonic() - t0 > timeout:
             for other in live:
                 other.kill()
-            return max(rc, 124)
+            return rc or 124
         time.sleep(0.05)
     return rc

@@ -177,10 +177,16 @@ int mixkvq_decode_step(mixkvq_cache* cache, int layer, const void* k_dev, const 
  * window).  The layer must be empty (MIXKVQ_E_UNSUPPORTED otherwise: a later chunk would have to attend to a
  * dequantized cache).
  *   k_dev, v_dev [B, Hkv, n_tokens, 128], q_dev [B, Hq, n_tokens, 128] bf16 (post-RoPE)  ->  out_dev [B, Hq, n_tokens, 128] float
+ *   scratch_dev: device memory of at least mixkvq_prefill_scratch_bytes(cfg, n_tokens) bytes, 16-byte aligned, owned by
+ *   the caller and free for reuse once the work enqueued by this call has run (it holds K and V of the prompt
+ *   rearranged into the tensor core's tile layout); too small -> MIXKVQ_E_CAPACITY.
  * The attention runs on the tcgen05 tensor cores (bf16 products for the logits, fp16 probabilities and values for the
- * output, fp32 accumulation in tensor memory); values must stay inside the fp16 range. */
+ * output, fp32 accumulation in tensor memory); values must stay inside the fp16 range.  softmax_scale > 0.  A barrier
+ * wait that runs out sets MIXKVQ_DEV_COPY_TIMEOUT in the status word and leaves the affected output rows unwritten.
+ * Nothing is allocated and nothing synchronises with the host. */
+size_t mixkvq_prefill_scratch_bytes(const mixkvq_config* cfg, int n_tokens);
 int mixkvq_prefill(mixkvq_cache* cache, int layer, const void* k_dev, const void* v_dev, const void* q_dev, int n_tokens,
-                   float* out_dev, float softmax_scale, void* stream);
+                   float* out_dev, float softmax_scale, void* scratch_dev, size_t scratch_bytes, void* stream);
 
 /* Appendix D ("saliency evaluation is performed post-transformation"): for models with rotary position embeddings the
  * scores, the stored keys and the attention all use rotated queries and keys.  These two calls rotate before they

@@ -19,7 +19,7 @@ EXPORTS = [
     "mixkvq_select_channels", "mixkvq_select_channels_raw", "mixkvq_quantize_append",
     "mixkvq_decode_attention", "mixkvq_decode_attention_noalloc", "mixkvq_decode_step", "mixkvq_set_attention_kernel", "mixkvq_query_status",
     "mixkvq_cache_describe", "mixkvq_launch_count", "mixkvq_status_string",
-    "mixkvq_cache_written_externally", "mixkvq_test_arm_copy_timeout", "mixkvq_rope_append", "mixkvq_rope_decode_step", "mixkvq_prefill",
+    "mixkvq_cache_written_externally", "mixkvq_test_arm_copy_timeout", "mixkvq_rope_append", "mixkvq_rope_decode_step", "mixkvq_prefill", "mixkvq_prefill_scratch_bytes",
 ]
 
 DEV_EXTRAS_FULL, DEV_COPY_TIMEOUT = 1, 2
@@ -72,7 +72,9 @@ def lib():
         L.mixkvq_decode_attention_noalloc.argtypes = [vp, i32, vp, vp, f32, vp]
         L.mixkvq_decode_step.argtypes = [vp, i32, vp, vp, vp, vp, f32, vp, C.c_size_t, vp]
         L.mixkvq_set_attention_kernel.argtypes = [vp, i32]
-        L.mixkvq_prefill.argtypes = [vp, i32, vp, vp, vp, i32, vp, f32, vp]
+        L.mixkvq_prefill.argtypes = [vp, i32, vp, vp, vp, i32, vp, f32, vp, C.c_size_t, vp]
+        L.mixkvq_prefill_scratch_bytes.argtypes = [C.POINTER(Config), i32]
+        L.mixkvq_prefill_scratch_bytes.restype = C.c_size_t
         L.mixkvq_rope_append.argtypes = [vp, i32, vp, vp, vp, vp, vp, i32, i32, vp]
         L.mixkvq_rope_decode_step.argtypes = [vp, i32, vp, vp, vp, vp, vp, i32, vp, f32, vp, C.c_size_t, vp]
         L.mixkvq_cache_written_externally.argtypes = [vp]
@@ -185,14 +187,21 @@ class Cache:
                                         _ptr(self.workspace), self.workspace.numel(), _stream()), "mixkvq_decode_step")
         return out
 
-    def prefill(self, layer, k, v, q, scale, out=None):
+    def prefill(self, layer, k, v, q, scale, out=None, scratch=None):
         """Causal attention of the prompt over itself (k, v [B,Hkv,n,128], q [B,Hq,n,128] bf16 -> [B,Hq,n,128] float32),
-        then the prompt goes into the (empty) layer as quantize_append would put it."""
+        then the prompt goes into the (empty) layer as quantize_append would put it.  `scratch`: a uint8 device
+        tensor of at least prefill_scratch_bytes(n) bytes (allocated here when absent)."""
+        n = k.shape[2]
         if out is None:
             out = torch.empty(q.shape, dtype=torch.float32, device=q.device)
-        _check(lib().mixkvq_prefill(self.handle, layer, _ptr(k), _ptr(v), _ptr(q), k.shape[2], _ptr(out), float(scale),
-                                    _stream()), "mixkvq_prefill")
+        if scratch is None:
+            scratch = torch.empty(self.prefill_scratch_bytes(n), dtype=torch.uint8, device=q.device)
+        _check(lib().mixkvq_prefill(self.handle, layer, _ptr(k), _ptr(v), _ptr(q), n, _ptr(out), float(scale),
+                                    _ptr(scratch), scratch.numel(), _stream()), "mixkvq_prefill")
         return out
+
+    def prefill_scratch_bytes(self, n_tokens):
+        return int(lib().mixkvq_prefill_scratch_bytes(C.byref(self.cfg), int(n_tokens)))
 
     def rope_append(self, layer, k, v, q, cos, sin, pos0):
         """Rotates k [B,Hkv,n,128] and q [B,Hq,n,128] (bf16) IN PLACE with rows pos0.. of the float32 tables cos, sin

@@ -338,19 +338,28 @@ int mixkvq_decode_step(mixkvq_cache* cache, int layer, const void* k_dev, const 
   return rc;
 }
 
+size_t mixkvq_prefill_scratch_bytes(const mixkvq_config* cfg, int n_tokens) {
+  if (check_config(cfg) != MIXKVQ_OK || n_tokens < 1) return 0;
+  return prefill_scratch_bytes(cfg->batch, cfg->n_kv_heads, n_tokens);
+}
+
 int mixkvq_prefill(mixkvq_cache* cache, int layer, const void* k_dev, const void* v_dev, const void* q_dev, int n_tokens,
-                   float* out_dev, float softmax_scale, void* stream) {
-  if (!cache || !k_dev || !v_dev || !q_dev || !out_dev || layer < 0 || layer >= cache->cfg.n_layers || n_tokens < 1)
+                   float* out_dev, float softmax_scale, void* scratch_dev, size_t scratch_bytes, void* stream) {
+  if (!cache || !k_dev || !v_dev || !q_dev || !out_dev || !scratch_dev || layer < 0 || layer >= cache->cfg.n_layers ||
+      n_tokens < 1 || !(softmax_scale > 0.f))
     return MIXKVQ_E_INVALID_ARG;
-  if (!aligned16(k_dev) || !aligned16(v_dev) || !aligned16(q_dev) || !aligned16(out_dev)) return MIXKVQ_E_ALIGNMENT;
+  if (!aligned16(k_dev) || !aligned16(v_dev) || !aligned16(q_dev) || !aligned16(out_dev) || !aligned16(scratch_dev))
+    return MIXKVQ_E_ALIGNMENT;
   // the prompt attends to itself only: the layer must be empty
   if (cache->n_blocks[layer] != 0 || cache->r[layer] != 0 || cache->n_sink[layer] != 0) return MIXKVQ_E_UNSUPPORTED;
-  if (n_tokens > cache->cfg.max_tokens) return MIXKVQ_E_CAPACITY;
-  if (launch_prefill_attention(q_dev, k_dev, v_dev, out_dev, cache->cfg.batch, cache->cfg.n_q_heads, cache->cfg.n_kv_heads,
-                               n_tokens, softmax_scale, reinterpret_cast<uint32_t*>(cache->mem), cache->test_wait_polls,
-                               static_cast<cudaStream_t>(stream)) != cudaSuccess)
+  if (n_tokens > cache->cfg.max_tokens ||
+      scratch_bytes < prefill_scratch_bytes(cache->cfg.batch, cache->cfg.n_kv_heads, n_tokens))
+    return MIXKVQ_E_CAPACITY;
+  if (launch_prefill_attention(q_dev, k_dev, v_dev, out_dev, scratch_dev, cache->cfg.batch, cache->cfg.n_q_heads,
+                               cache->cfg.n_kv_heads, n_tokens, softmax_scale, reinterpret_cast<uint32_t*>(cache->mem),
+                               cache->test_wait_polls, static_cast<cudaStream_t>(stream)) != cudaSuccess)
     return MIXKVQ_E_CUDA;
-  cache->launches += 1;
+  cache->launches += 2;
   cache->last_packed_writer = kNoPackedWrite;
   return mixkvq_quantize_append(cache, layer, k_dev, v_dev, q_dev, n_tokens, stream);
 }

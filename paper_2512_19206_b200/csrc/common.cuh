@@ -185,8 +185,9 @@ cudaError_t launch_append(const LayerView& lv, const void* k, const void* v, con
 cudaError_t launch_sink_append(const LayerView& lv, const void* k, const void* v, int n_tokens, int t0, int m,
                                cudaStream_t stream);
 // causal full-precision attention over a prompt (tcgen05)
-cudaError_t launch_prefill_attention(const void* q, const void* k, const void* v, float* out, int B, int Hq, int Hkv, int L,
-                                     float scale, uint32_t* status, uint32_t max_polls, cudaStream_t stream);
+cudaError_t launch_prefill_attention(const void* q, const void* k, const void* v, float* out, void* scratch, int B, int Hq,
+                                     int Hkv, int L, float scale, uint32_t* status, uint32_t max_polls, cudaStream_t stream);
+size_t prefill_scratch_bytes(int B, int Hkv, int L);
 cudaError_t prefill_attention_setup();
 cudaError_t launch_rope(void* k, void* q, const float* cos_t, const float* sin_t, int B, int Hkv, int Hq, int n_tokens,
                         int pos0, cudaStream_t stream);

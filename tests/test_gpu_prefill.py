@@ -53,3 +53,8 @@ def test_prefill_large_magnitudes_and_errors(binding):
     with pytest.raises(binding.MixKVQError) as e:                      # the layer is no longer empty
         cache.prefill(0, k.cuda(), v.cuda(), q.cuda(), W.softmax_scale())
     assert e.value.code == -2
+    cache.reset()
+    small = torch.empty(cache.prefill_scratch_bytes(300) - 16, dtype=torch.uint8, device="cuda")
+    with pytest.raises(binding.MixKVQError):                           # the scratch buffer is too small
+        cache.prefill(0, k.cuda(), v.cuda(), q.cuda(), W.softmax_scale(), scratch=small)
+    assert cache.prefill_scratch_bytes(300) == 2 * w.n_kv_heads * 3 * 32768

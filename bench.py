@@ -327,6 +327,61 @@ def other_config(binding, dev, args, name, w, label, contexts=None):
     return entries
 
 
+def tensor_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["bf16_tflops"]), float(d["bf16_tflops_sustained"]), "measured (MEASURED_PEAKS.json)"
+    return 1590.0, 1400.0, "fallback (1.59 PFLOP/s burst, 1.4 sustained, no MEASURED_PEAKS.json)"
+
+
+def prefill_attention_entries(binding, dev, args, contexts=(8192, 32768)):
+    """The prefill call (causal full-precision attention of the prompt on the tensor cores, then the bulk quantizing
+    append) on one layer of the headline model shape, one sequence: a tensor-bound path, reported against the
+    measured bf16 GEMM peaks.  The flops are those of the causal definition: 4 D L (L + 1) / 2 per query head."""
+    entries = []
+    burst, sustained, src = tensor_peaks()
+    for L in contexts:
+        w = W.small(W.CONFIGS["qwen7b"], n_layers=1, batch=1, tokens=L)
+        cache = make_cache(binding, w, args, dev, 0)
+        k, v, q = W.tokens(w, 0, 0, L, device=dev)
+        out = torch.empty(q.shape, dtype=torch.float32, device=dev)
+        scratch = torch.empty(cache.prefill_scratch_bytes(L), dtype=torch.uint8, device=dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+        def timed(fn):
+            ms = []
+            for _ in range(6):
+                cache.reset()
+                e0.record()
+                fn()
+                e1.record()
+                e1.synchronize()
+                ms.append(e0.elapsed_time(e1))
+            return ms
+
+        call_ms = timed(lambda: cache.prefill(0, k, v, q, W.softmax_scale(), out=out, scratch=scratch))
+        append_ms = timed(lambda: cache.quantize_append(0, k, v, q))
+        call = sorted(call_ms[2:])[2]
+        app = sorted(append_ms[2:])[2]
+        flops = 4.0 * 128 * w.n_q_heads * L * (L + 1) / 2
+        attn = call - app
+        entries.append({
+            "workload": "prefill: qwen2.5-7b shape, one layer, one sequence", "shape": f"B=1 Hq={w.n_q_heads} Hkv={w.n_kv_heads} L={L}",
+            "call_ms": call, "append_ms": app, "attention_ms": attn, "flops": flops,
+            "roofline": {"bound": "tensor", "kernel": "prefill_pack_kernel + prefill_attention_kernel",
+                         "achieved": flops / (attn * 1e-3) / 1e12, "peak": sustained, "unit": "TFLOP/s",
+                         "frac": flops / (attn * 1e-3) / 1e12 / sustained,
+                         "frac_of_burst_peak": flops / (attn * 1e-3) / 1e12 / burst, "peak_source": src,
+                         "note": "attention_ms = the call minus the bulk append timed alone; causal flops only "
+                                 "(the masked half of the diagonal tiles is computed and not counted)"},
+            "whole_call_tflops": flops / (call * 1e-3) / 1e12, "device_status": cache.status()})
+        cache.close()
+        del cache, k, v, q, out, scratch
+        torch.cuda.empty_cache()
+    return entries
+
+
 def run_gpu(args, w):
     rank, world, local = dist_env()
     torch.cuda.set_device(local)
@@ -518,6 +573,7 @@ def run_gpu(args, w):
         cfgs += other_config(binding, dev, args, "longcot", W.small(W.CONFIGS["longcot"], n_layers=4),
                              "config 5: long-CoT stream", contexts=[8192, 32768, 65536, 131072])
         line["configs"] = cfgs
+        line["prefill_attention"] = prefill_attention_entries(binding, dev, args)
     if world == 1 and not args.no_cpu_baseline:
         sec, desc = oracle_sample(w, n_streams=8, reps=5)
         n_streams = w.n_layers * w.batch * w.n_kv_heads

@@ -104,7 +104,7 @@ typedef struct mixkvq_layout_desc {
   uint64_t extras_off, extras_stride;     /* per stream: extras arena                                */
   uint64_t base_bytes;                    /* size of one block's fixed part                          */
   uint32_t max_blocks, n_streams;
-  uint32_t n_blocks, residual_tokens;     /* current fill of this layer (same for all streams)       */
+  uint32_t n_blocks, residual_tokens;     /* current fill of sequence 0 (mixkvq_sequence_fill: any)  */
   uint64_t sink_off, sink_stride;         /* per stream: [sink_len][128] bf16 keys, then the same for values */
   uint32_t sink_tokens, sink_len;         /* sink rows filled so far, and their capacity              */
 } mixkvq_layout_desc;
@@ -170,6 +170,27 @@ int mixkvq_decode_attention(mixkvq_cache* cache, int layer, const void* q_dev, f
  * (Appendix D.1, D.2), which saves a kernel launch per layer. */
 int mixkvq_decode_step(mixkvq_cache* cache, int layer, const void* k_dev, const void* v_dev, const void* q_dev,
                        float* out_dev, float softmax_scale, void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/* (2) for a batch whose sequences differ in length (the serving setting of the efficiency experiment: requests of
+ * unequal length share a batch).  Sequence b takes the first n_tokens_host[b] tokens (0 <= n_tokens_host[b] <=
+ * n_tokens_max; 0 = the sequence takes no token in this call) of its rows of the tensors:
+ *   k_dev, v_dev [B, Hkv, n_tokens_max, 128], q_dev [B, Hq, n_tokens_max, 128] bf16; n_tokens_host: HOST array [B].
+ * Every sequence keeps its own number of packed blocks, residual tokens and sink rows; each is flushed when ITS window
+ * is full, exactly as if it were alone in the batch (the bytes of its streams equal those of a batch-1 cache fed the
+ * same tokens).  Neighbouring sequences with the same fill and the same count go through the kernels together, so a
+ * batch of equal lengths costs what mixkvq_quantize_append costs (which is this call with equal counts).
+ * The capacity check covers every sequence before anything is enqueued.
+ * After sequences have diverged, mixkvq_decode_attention, mixkvq_decode_step and mixkvq_select_channels work per
+ * sequence: the attention kernel reads every sequence's fill from a table in device memory (written on the stream as
+ * kernel arguments, no copy) and splits the positions of all streams evenly over its CTAs; a sequence without tokens
+ * gets an all-zero output.  Restrictions of a diverged batch: fragment layout, the default or the split-only
+ * attention kernel, B <= 128 (MIXKVQ_E_UNSUPPORTED otherwise). */
+int mixkvq_quantize_append_ragged(mixkvq_cache* cache, int layer, const void* k_dev, const void* v_dev, const void* q_dev,
+                                  int n_tokens_max, const int32_t* n_tokens_host, void* stream);
+
+/* Fill of sequence b of a layer (any pointer may be NULL). */
+int mixkvq_sequence_fill(const mixkvq_cache* cache, int layer, int b, uint32_t* n_blocks, uint32_t* residual_tokens,
+                         uint32_t* sink_tokens);
 
 /* The prefill phase of Section 4.2 for one layer: causal attention of the prompt over itself in full precision (Eq. 1,
  * position i sees positions 0..i), then the prompt's keys and values go into the cache exactly as

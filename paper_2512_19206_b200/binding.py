@@ -19,7 +19,7 @@ EXPORTS = [
     "mixkvq_select_channels", "mixkvq_select_channels_raw", "mixkvq_quantize_append",
     "mixkvq_decode_attention", "mixkvq_decode_attention_noalloc", "mixkvq_decode_step", "mixkvq_set_attention_kernel", "mixkvq_query_status",
     "mixkvq_cache_describe", "mixkvq_launch_count", "mixkvq_status_string",
-    "mixkvq_cache_written_externally", "mixkvq_test_arm_copy_timeout", "mixkvq_rope_append", "mixkvq_rope_decode_step", "mixkvq_prefill", "mixkvq_prefill_scratch_bytes",
+    "mixkvq_cache_written_externally", "mixkvq_test_arm_copy_timeout", "mixkvq_rope_append", "mixkvq_rope_decode_step", "mixkvq_prefill", "mixkvq_prefill_scratch_bytes", "mixkvq_quantize_append_ragged", "mixkvq_sequence_fill",
 ]
 
 DEV_EXTRAS_FULL, DEV_COPY_TIMEOUT = 1, 2
@@ -72,6 +72,8 @@ def lib():
         L.mixkvq_decode_attention_noalloc.argtypes = [vp, i32, vp, vp, f32, vp]
         L.mixkvq_decode_step.argtypes = [vp, i32, vp, vp, vp, vp, f32, vp, C.c_size_t, vp]
         L.mixkvq_set_attention_kernel.argtypes = [vp, i32]
+        L.mixkvq_quantize_append_ragged.argtypes = [vp, i32, vp, vp, vp, i32, C.POINTER(C.c_int32), vp]
+        L.mixkvq_sequence_fill.argtypes = [vp, i32, i32, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)]
         L.mixkvq_prefill.argtypes = [vp, i32, vp, vp, vp, i32, vp, f32, vp, C.c_size_t, vp]
         L.mixkvq_prefill_scratch_bytes.argtypes = [C.POINTER(Config), i32]
         L.mixkvq_prefill_scratch_bytes.restype = C.c_size_t
@@ -187,6 +189,19 @@ class Cache:
                                         _ptr(self.workspace), self.workspace.numel(), _stream()), "mixkvq_decode_step")
         return out
 
+    def quantize_append_ragged(self, layer, k, v, q, counts):
+        """k, v [B,Hkv,n_max,128], q [B,Hq,n_max,128] bf16; counts: per-sequence token counts (host ints)."""
+        arr = (C.c_int32 * len(counts))(*[int(c) for c in counts])
+        _check(lib().mixkvq_quantize_append_ragged(self.handle, layer, _ptr(k), _ptr(v), _ptr(q), k.shape[2], arr,
+                                                   _stream()), "mixkvq_quantize_append_ragged")
+
+    def sequence_fill(self, layer, b):
+        """(n_blocks, residual_tokens, sink_tokens) of sequence b."""
+        x = [C.c_uint32(0) for _ in range(3)]
+        _check(lib().mixkvq_sequence_fill(self.handle, layer, b, C.byref(x[0]), C.byref(x[1]), C.byref(x[2])),
+               "mixkvq_sequence_fill")
+        return tuple(int(v.value) for v in x)
+
     def prefill(self, layer, k, v, q, scale, out=None, scratch=None):
         """Causal attention of the prompt over itself (k, v [B,Hkv,n,128], q [B,Hq,n,128] bf16 -> [B,Hq,n,128] float32),
         then the prompt goes into the (empty) layer as quantize_append would put it.  `scratch`: a uint8 device
@@ -270,7 +285,7 @@ class Cache:
             return m[start:start + n].cpu().numpy().tobytes()
 
         R = self.cfg.residual_len
-        nb, r = d.n_blocks, d.residual_tokens
+        nb, r, n_sink = self.sequence_fill(layer, stream // self.cfg.n_kv_heads)
         state = cut(d.state_off, d.state_stride, 1152)
         used16 = int.from_bytes(state[1028:1032], "little")
         resk = cut(d.resk_off, d.resk_stride, R * 256)
@@ -282,6 +297,6 @@ class Cache:
             "state": state,
             "resK": resk[: r * 256],
             "resV": resv[: r * 256],
-            "sinkK": cut(d.sink_off, d.sink_stride, d.sink_tokens * 256),
-            "sinkV": cut(d.sink_off + d.sink_len * 256, d.sink_stride, d.sink_tokens * 256),
+            "sinkK": cut(d.sink_off, d.sink_stride, n_sink * 256),
+            "sinkV": cut(d.sink_off + d.sink_len * 256, d.sink_stride, n_sink * 256),
         }

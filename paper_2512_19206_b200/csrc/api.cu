@@ -1,5 +1,6 @@
 // Host side of the C ABI: argument checking, the cache memory map, per-layer length tracking and the
 // scheduling of the kernels.  No device allocation happens here.
+#include <algorithm>
 #include <new>
 #include <vector>
 
@@ -15,8 +16,9 @@ struct mixkvq_cache {
   uint32_t base_bytes, unit_bytes;
   uint64_t extras_budget;
   // byte offsets inside one layer and per-stream strides
-  uint64_t state_off, table_off, resk_off, resv_off, base_off, extras_off, sink_off, layer_stride;
+  uint64_t state_off, table_off, resk_off, resv_off, base_off, extras_off, sink_off, seq_off, layer_stride;
   uint64_t state_stride, table_stride, resk_stride, resv_stride, base_stride, extras_stride, sink_stride;
+  // fill of every sequence of every layer, index layer * batch + b: packed blocks, tokens in the residual window, sink rows
   std::vector<int> n_blocks, r, n_sink;
   int n_sms;
   int attn_kind;
@@ -88,18 +90,49 @@ uint64_t plan(const mixkvq_config* c, mixkvq_cache* h) {
   h->base_off = off;   off = align_up(off + h->base_stride * h->S, 256);
   h->extras_off = off; off = align_up(off + h->extras_stride * h->S, 256);
   h->sink_off = off;   off = align_up(off + h->sink_stride * h->S, 256);
+  h->seq_off = off;    off = align_up(off + (uint64_t)c->batch * 16 + (uint64_t)(c->batch + 1) * 4, 256);
   h->layer_stride = off;
   return kHeaderBytes + h->layer_stride * (uint64_t)c->n_layers;
 }
 
 size_t workspace_bytes(int S) { return (size_t)(kMaxCtas + 2 * S) * kPartialFloats * sizeof(float); }
 
-LayerView view(const mixkvq_cache* h, int layer) {
+inline int fi(const mixkvq_cache* h, int layer, int b) { return layer * h->cfg.batch + b; }
+
+bool same_fill(const mixkvq_cache* h, int layer, int b1, int b2) {
+  const int i = fi(h, layer, b1), j = fi(h, layer, b2);
+  return h->n_blocks[i] == h->n_blocks[j] && h->r[i] == h->r[j] && h->n_sink[i] == h->n_sink[j];
+}
+// every sequence of the layer holds the same number of blocks, residual tokens and sink rows
+bool uniform(const mixkvq_cache* h, int layer) {
+  for (int b = 1; b < h->cfg.batch; ++b)
+    if (!same_fill(h, layer, 0, b)) return false;
+  return true;
+}
+bool all_empty(const mixkvq_cache* h, int layer) {
+  for (int b = 0; b < h->cfg.batch; ++b) {
+    const int i = fi(h, layer, b);
+    if (h->n_blocks[i] || h->r[i] || h->n_sink[i]) return false;
+  }
+  return true;
+}
+long long tokens_held(const mixkvq_cache* h, int layer, int b) {
+  const int i = fi(h, layer, b);
+  return (long long)h->n_sink[i] + (long long)h->n_blocks[i] * h->R + h->r[i];
+}
+long long max_tokens_held(const mixkvq_cache* h, int layer) {
+  long long m = 0;
+  for (int b = 0; b < h->cfg.batch; ++b) m = std::max(m, tokens_held(h, layer, b));
+  return m;
+}
+
+// The layer's arrays for sequences b0 .. b0 + nb - 1 (all of them when nb < 0), which share the fill of sequence b0.
+LayerView view(const mixkvq_cache* h, int layer, int b0 = 0, int nb = -1) {
   LayerView v{};
-  v.B = h->cfg.batch; v.Hq = h->cfg.n_q_heads; v.Hkv = h->cfg.n_kv_heads; v.g = h->g;
+  v.B = nb < 0 ? h->cfg.batch : nb; v.Hq = h->cfg.n_q_heads; v.Hkv = h->cfg.n_kv_heads; v.g = h->g;
   v.R = h->R; v.G = h->G; v.U = h->U; v.NG = h->NG; v.VG = h->VG;
   v.max_blocks = h->max_blocks;
-  v.n_blocks = h->n_blocks[layer]; v.r = h->r[layer];
+  v.n_blocks = h->n_blocks[fi(h, layer, b0)]; v.r = h->r[fi(h, layer, b0)];
   v.tile = h->tile;
   v.budget_bf16 = h->cfg.budget_bf16; v.budget_u4 = h->cfg.budget_u4;
   v.v_bits = h->cfg.v_bits;
@@ -109,14 +142,15 @@ LayerView view(const mixkvq_cache* h, int layer) {
   v.score_bits = h->cfg.score_bits; v.importance_mode = h->cfg.importance_mode;
   v.tau_bf16 = h->cfg.tau_bf16; v.tau_u4 = h->cfg.tau_u4;
   char* L = h->mem + kHeaderBytes + h->layer_stride * (uint64_t)layer;
-  v.state = L + h->state_off;   v.state_stride = h->state_stride;
-  v.table = L + h->table_off;   v.table_stride = h->table_stride;
-  v.resk = L + h->resk_off;     v.resk_stride = h->resk_stride;
-  v.resv = L + h->resv_off;     v.resv_stride = h->resv_stride;
-  v.base = L + h->base_off;     v.base_stride = h->base_stride;
-  v.extras = L + h->extras_off; v.extras_stride = h->extras_stride;
-  v.sink = L + h->sink_off;     v.sink_stride = h->sink_stride;
-  v.sink_len = h->cfg.sink_len; v.n_sink = h->n_sink[layer];
+  const uint64_t s0 = (uint64_t)b0 * h->cfg.n_kv_heads;      // first stream of the view
+  v.state = L + h->state_off + s0 * h->state_stride;    v.state_stride = h->state_stride;
+  v.table = L + h->table_off + s0 * h->table_stride;    v.table_stride = h->table_stride;
+  v.resk = L + h->resk_off + s0 * h->resk_stride;       v.resk_stride = h->resk_stride;
+  v.resv = L + h->resv_off + s0 * h->resv_stride;       v.resv_stride = h->resv_stride;
+  v.base = L + h->base_off + s0 * h->base_stride;       v.base_stride = h->base_stride;
+  v.extras = L + h->extras_off + s0 * h->extras_stride; v.extras_stride = h->extras_stride;
+  v.sink = L + h->sink_off + s0 * h->sink_stride;       v.sink_stride = h->sink_stride;
+  v.sink_len = h->cfg.sink_len; v.n_sink = h->n_sink[fi(h, layer, b0)];
   v.status = reinterpret_cast<uint32_t*>(h->mem);
   v.debug_extra_tx = h->test_extra_tx;
   v.wait_polls = h->test_wait_polls;
@@ -128,9 +162,7 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 int zero_layer_state(mixkvq_cache* h, int layer, cudaStream_t st) {
   char* L = h->mem + kHeaderBytes + h->layer_stride * (uint64_t)layer;
   if (cudaMemsetAsync(L + h->state_off, 0, h->state_stride * h->S, st) != cudaSuccess) return MIXKVQ_E_CUDA;
-  h->n_blocks[layer] = 0;
-  h->r[layer] = 0;
-  h->n_sink[layer] = 0;
+  for (int b = 0; b < h->cfg.batch; ++b) h->n_blocks[fi(h, layer, b)] = h->r[fi(h, layer, b)] = h->n_sink[fi(h, layer, b)] = 0;
   h->last_packed_writer = kAllPacked;
   return MIXKVQ_OK;
 }
@@ -144,6 +176,34 @@ int run_attention(mixkvq_cache* h, int layer, const void* q, float* out, float s
   lv.stage_early = (h->last_packed_writer == kNoPackedWrite ||
                     (h->last_packed_writer >= 0 && h->last_packed_writer != layer)) ? 1 : 0;
   h->last_packed_writer = kNoPackedWrite;
+  if (!uniform(h, layer)) {
+    // ragged batch: the fills go to the layer's table in device memory (as kernel arguments), and the split kernel
+    // and the merge walk every stream's own positions
+    const int B = h->cfg.batch;
+    if (h->tile || h->attn_kind == 1 || B > kMaxRaggedBatch) return MIXKVQ_E_UNSUPPORTED;
+    SeqTableArgs a{};
+    a.n = B;
+    a.Hkv = h->cfg.n_kv_heads;
+    long long total = 0;
+    for (int b = 0; b < B; ++b) {
+      const int i = fi(h, layer, b);
+      a.fill[3 * b] = h->n_blocks[i];
+      a.fill[3 * b + 1] = h->r[i];
+      a.fill[3 * b + 2] = h->n_sink[i];
+      a.w[b] = attention_ws_positions_of(h->n_blocks[i], h->r[i], h->n_sink[i], h->U);
+      total += (long long)a.Hkv * a.w[b];
+    }
+    if (total >= (1ll << 31)) return MIXKVQ_E_UNSUPPORTED;
+    char* L = h->mem + kHeaderBytes + h->layer_stride * (uint64_t)layer + h->seq_off;
+    int4* seq = reinterpret_cast<int4*>(L);
+    int* prefix = reinterpret_cast<int*>(L + (size_t)B * 16);
+    if (launch_seq_table(a, seq, prefix, st) != cudaSuccess) return MIXKVQ_E_CUDA;
+    h->launches += 1;
+    lv.seq = seq;
+    lv.seq_prefix = prefix;
+    lv.seq_total = total;
+    lv.stage_early = 0;
+  }
   int launches = 0;
   cudaError_t e;
   if (h->attn_kind == 1)
@@ -154,6 +214,74 @@ int run_attention(mixkvq_cache* h, int layer, const void* q, float* out, float s
     e = launch_attention_ws(lv, q, h->attn_kind == 2 ? nullptr : out, scale, ws, h->n_sms, st, &launches);
   h->launches += launches;
   return e == cudaSuccess ? MIXKVQ_OK : MIXKVQ_E_CUDA;
+}
+
+// Appends tokens 0 .. n_tokens - 1 of the tensors (whose token dimension is n_stride long) to sequences b0 .. b0 + nb - 1,
+// which share one fill: sink rows first, then flush / bulk blocks / residual rows as the fill demands.
+int append_run_first(mixkvq_cache* cache, int layer, int b0, int nb, const void* k_dev, const void* v_dev, const void* q_dev,
+                     int n_stride, int n_tokens, cudaStream_t st) {
+  const char* k = static_cast<const char*>(k_dev) + (size_t)b0 * cache->cfg.n_kv_heads * n_stride * kD * 2;
+  const char* v = static_cast<const char*>(v_dev) + (size_t)b0 * cache->cfg.n_kv_heads * n_stride * kD * 2;
+  const char* q = static_cast<const char*>(q_dev) + (size_t)b0 * cache->cfg.n_q_heads * n_stride * kD * 2;
+  // the run's fill is kept in the first sequence's slots here; append_run copies it to the others
+  int& sink0 = cache->n_sink[fi(cache, layer, b0)];
+  int& r0 = cache->r[fi(cache, layer, b0)];
+  int& nb0 = cache->n_blocks[fi(cache, layer, b0)];
+  int t = 0;
+  while (t < n_tokens) {
+    if (sink0 < cache->cfg.sink_len) {
+      // the first tokens of the sequence are sink tokens: stored as they are, outside everything else
+      const int room = cache->cfg.sink_len - sink0;
+      const int m = n_tokens - t < room ? n_tokens - t : room;
+      LayerView lv = view(cache, layer, b0, nb);
+      if (launch_sink_append(lv, k, v, n_stride, t, m, st) != cudaSuccess) return MIXKVQ_E_CUDA;
+      cache->launches += 1;
+      cache->last_packed_writer = kNoPackedWrite;
+      sink0 += m;
+      t += m;
+      continue;
+    }
+    if (r0 == cache->R) {
+      LayerView lv = view(cache, layer, b0, nb);
+      if (launch_flush(lv, st) != cudaSuccess) return MIXKVQ_E_CUDA;
+      cache->launches += 1;
+      cache->last_packed_writer = layer;
+      nb0 += 1;
+      r0 = 0;
+    }
+    // prefill: complete windows go straight from the tensors to packed blocks; the last 1..R tokens stay in the
+    // residual window
+    if (r0 == 0 && n_tokens - t > cache->R) {
+      int nblk = (n_tokens - t - 1) / cache->R;
+      if (nblk > 32768) nblk = 32768;                  // grid.y limit
+      LayerView lv = view(cache, layer, b0, nb);
+      if (launch_flush_bulk(lv, k, v, q, n_stride, t, nblk, st) != cudaSuccess) return MIXKVQ_E_CUDA;
+      cache->launches += cache->cfg.importance_mode == 1 ? 4 : 3;
+      cache->last_packed_writer = layer;
+      nb0 += nblk;
+      t += nblk * cache->R;
+      continue;
+    }
+    const int m = (n_tokens - t < cache->R - r0) ? n_tokens - t : cache->R - r0;
+    LayerView lv = view(cache, layer, b0, nb);
+    if (launch_append(lv, k, v, q, n_stride, t, m, st) != cudaSuccess) return MIXKVQ_E_CUDA;
+    cache->launches += 1;
+    cache->last_packed_writer = kNoPackedWrite;
+    r0 += m;
+    t += m;
+  }
+  return MIXKVQ_OK;
+}
+
+int append_run(mixkvq_cache* cache, int layer, int b0, int nb, const void* k_dev, const void* v_dev, const void* q_dev,
+               int n_stride, int n_tokens, cudaStream_t st) {
+  const int rc = append_run_first(cache, layer, b0, nb, k_dev, v_dev, q_dev, n_stride, n_tokens, st);
+  for (int b = b0 + 1; b < b0 + nb; ++b) {
+    cache->n_sink[fi(cache, layer, b)] = cache->n_sink[fi(cache, layer, b0)];
+    cache->r[fi(cache, layer, b)] = cache->r[fi(cache, layer, b0)];
+    cache->n_blocks[fi(cache, layer, b)] = cache->n_blocks[fi(cache, layer, b0)];
+  }
+  return rc;
 }
 
 }  // namespace
@@ -181,9 +309,9 @@ int mixkvq_cache_init(const mixkvq_config* cfg, void* cache_dev, size_t bytes, v
   if (bytes < total) { delete h; return MIXKVQ_E_BUFFER_TOO_SMALL; }
   h->mem = static_cast<char*>(cache_dev);
   h->bytes = bytes;
-  h->n_blocks.assign(cfg->n_layers, 0);
-  h->r.assign(cfg->n_layers, 0);
-  h->n_sink.assign(cfg->n_layers, 0);
+  h->n_blocks.assign((size_t)cfg->n_layers * cfg->batch, 0);
+  h->r.assign((size_t)cfg->n_layers * cfg->batch, 0);
+  h->n_sink.assign((size_t)cfg->n_layers * cfg->batch, 0);
   h->attn_kind = 0;
   h->launches = 0;
   h->last_packed_writer = kAllPacked;
@@ -221,12 +349,26 @@ int mixkvq_cache_reset(mixkvq_cache* cache, int layer, void* stream) {
 
 int mixkvq_select_channels(mixkvq_cache* cache, int layer, uint8_t* tiers_dev, double* salience_dev, void* stream) {
   if (!cache || !tiers_dev || layer < 0 || layer >= cache->cfg.n_layers) return MIXKVQ_E_INVALID_ARG;
-  if (cache->r[layer] == 0) return MIXKVQ_E_EMPTY;
-  LayerView lv = view(cache, layer);
-  cache->launches += 1;
+  bool any = false;
+  for (int b = 0; b < cache->cfg.batch; ++b) any = any || cache->r[fi(cache, layer, b)] > 0;
+  if (!any) return MIXKVQ_E_EMPTY;
   cache->last_packed_writer = kNoPackedWrite;
-  return launch_select_window(lv, tiers_dev, salience_dev, static_cast<cudaStream_t>(stream)) == cudaSuccess
-             ? MIXKVQ_OK : MIXKVQ_E_CUDA;
+  // one launch per run of sequences with the same fill (one launch for a batch of equal lengths); a sequence whose
+  // window is empty has no scores: its rows of the outputs are left as they are
+  const int B = cache->cfg.batch, Hkv = cache->cfg.n_kv_heads;
+  for (int b0 = 0; b0 < B;) {
+    int b1 = b0 + 1;
+    while (b1 < B && same_fill(cache, layer, b0, b1)) ++b1;
+    if (cache->r[fi(cache, layer, b0)] > 0) {
+      LayerView lv = view(cache, layer, b0, b1 - b0);
+      if (launch_select_window(lv, tiers_dev + (size_t)b0 * Hkv * kD, salience_dev ? salience_dev + (size_t)b0 * Hkv * kD : nullptr,
+                               static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return MIXKVQ_E_CUDA;
+      cache->launches += 1;
+    }
+    b0 = b1;
+  }
+  return MIXKVQ_OK;
 }
 
 int mixkvq_select_channels_raw(const void* q_dev, const void* k_dev, int batch, int n_q_heads, int n_kv_heads,
@@ -243,54 +385,32 @@ int mixkvq_select_channels_raw(const void* q_dev, const void* k_dev, int batch, 
 
 int mixkvq_quantize_append(mixkvq_cache* cache, int layer, const void* k_dev, const void* v_dev, const void* q_dev,
                            int n_tokens, void* stream) {
-  if (!cache || !k_dev || !v_dev || !q_dev || layer < 0 || layer >= cache->cfg.n_layers || n_tokens < 1)
+  if (!cache || n_tokens < 1) return MIXKVQ_E_INVALID_ARG;
+  std::vector<int32_t> counts((size_t)cache->cfg.batch, n_tokens);
+  return mixkvq_quantize_append_ragged(cache, layer, k_dev, v_dev, q_dev, n_tokens, counts.data(), stream);
+}
+
+int mixkvq_quantize_append_ragged(mixkvq_cache* cache, int layer, const void* k_dev, const void* v_dev, const void* q_dev,
+                                  int n_tokens_max, const int32_t* n_tokens_host, void* stream) {
+  if (!cache || !k_dev || !v_dev || !q_dev || !n_tokens_host || layer < 0 || layer >= cache->cfg.n_layers || n_tokens_max < 1)
     return MIXKVQ_E_INVALID_ARG;
   if (!aligned16(k_dev) || !aligned16(v_dev) || !aligned16(q_dev)) return MIXKVQ_E_ALIGNMENT;
-  const long long have = (long long)cache->n_sink[layer] + (long long)cache->n_blocks[layer] * cache->R + cache->r[layer];
-  if (have + n_tokens > cache->cfg.max_tokens) return MIXKVQ_E_CAPACITY;
+  const int B = cache->cfg.batch;
+  for (int b = 0; b < B; ++b) {
+    if (n_tokens_host[b] < 0 || n_tokens_host[b] > n_tokens_max) return MIXKVQ_E_INVALID_ARG;
+    if (tokens_held(cache, layer, b) + n_tokens_host[b] > cache->cfg.max_tokens) return MIXKVQ_E_CAPACITY;
+  }
+  // runs of neighbouring sequences with the same fill and the same number of new tokens go through the kernels together
+  // (a batch of equal lengths is one run)
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  int t = 0;
-  while (t < n_tokens) {
-    if (cache->n_sink[layer] < cache->cfg.sink_len) {
-      // the first tokens of the sequence are sink tokens: stored as they are, outside everything else
-      const int room = cache->cfg.sink_len - cache->n_sink[layer];
-      const int m = n_tokens - t < room ? n_tokens - t : room;
-      LayerView lv = view(cache, layer);
-      if (launch_sink_append(lv, k_dev, v_dev, n_tokens, t, m, st) != cudaSuccess) return MIXKVQ_E_CUDA;
-      cache->launches += 1;
-      cache->last_packed_writer = kNoPackedWrite;
-      cache->n_sink[layer] += m;
-      t += m;
-      continue;
+  for (int b0 = 0; b0 < B;) {
+    int b1 = b0 + 1;
+    while (b1 < B && n_tokens_host[b1] == n_tokens_host[b0] && same_fill(cache, layer, b0, b1)) ++b1;
+    if (n_tokens_host[b0] > 0) {
+      const int rc = append_run(cache, layer, b0, b1 - b0, k_dev, v_dev, q_dev, n_tokens_max, n_tokens_host[b0], st);
+      if (rc != MIXKVQ_OK) return rc;
     }
-    if (cache->r[layer] == cache->R) {
-      LayerView lv = view(cache, layer);
-      if (launch_flush(lv, st) != cudaSuccess) return MIXKVQ_E_CUDA;
-      cache->launches += 1;
-      cache->last_packed_writer = layer;
-      cache->n_blocks[layer] += 1;
-      cache->r[layer] = 0;
-    }
-    // prefill: complete windows go straight from the tensors to packed blocks; the last 1..R tokens stay in the
-    // residual window
-    if (cache->r[layer] == 0 && n_tokens - t > cache->R) {
-      int nb = (n_tokens - t - 1) / cache->R;
-      if (nb > 32768) nb = 32768;                  // grid.y limit
-      LayerView lv = view(cache, layer);
-      if (launch_flush_bulk(lv, k_dev, v_dev, q_dev, n_tokens, t, nb, st) != cudaSuccess) return MIXKVQ_E_CUDA;
-      cache->launches += cache->cfg.importance_mode == 1 ? 4 : 3;
-      cache->last_packed_writer = layer;
-      cache->n_blocks[layer] += nb;
-      t += nb * cache->R;
-      continue;
-    }
-    const int m = (n_tokens - t < cache->R - cache->r[layer]) ? n_tokens - t : cache->R - cache->r[layer];
-    LayerView lv = view(cache, layer);
-    if (launch_append(lv, k_dev, v_dev, q_dev, n_tokens, t, m, st) != cudaSuccess) return MIXKVQ_E_CUDA;
-    cache->launches += 1;
-    cache->last_packed_writer = kNoPackedWrite;
-    cache->r[layer] += m;
-    t += m;
+    b0 = b1;
   }
   return MIXKVQ_OK;
 }
@@ -301,7 +421,7 @@ int mixkvq_decode_attention(mixkvq_cache* cache, int layer, const void* q_dev, f
     return MIXKVQ_E_INVALID_ARG;
   if (!aligned16(q_dev) || !aligned16(out_dev) || !aligned16(workspace_dev)) return MIXKVQ_E_ALIGNMENT;
   if (workspace_bytes_given < workspace_bytes(cache->S)) return MIXKVQ_E_BUFFER_TOO_SMALL;
-  if (cache->n_blocks[layer] == 0 && cache->r[layer] == 0 && cache->n_sink[layer] == 0) return MIXKVQ_E_EMPTY;
+  if (all_empty(cache, layer)) return MIXKVQ_E_EMPTY;
   return run_attention(cache, layer, q_dev, out_dev, softmax_scale, static_cast<float*>(workspace_dev),
                        static_cast<cudaStream_t>(stream));
 }
@@ -314,27 +434,38 @@ int mixkvq_decode_step(mixkvq_cache* cache, int layer, const void* k_dev, const 
   if (!aligned16(k_dev) || !aligned16(v_dev) || !aligned16(q_dev) || !aligned16(out_dev) || !aligned16(workspace_dev))
     return MIXKVQ_E_ALIGNMENT;
   if (workspace_bytes_given < workspace_bytes(cache->S)) return MIXKVQ_E_BUFFER_TOO_SMALL;
-  const long long have = (long long)cache->n_sink[layer] + (long long)cache->n_blocks[layer] * cache->R + cache->r[layer];
-  if (have + 1 > cache->cfg.max_tokens) return MIXKVQ_E_CAPACITY;
+  if (max_tokens_held(cache, layer) + 1 > cache->cfg.max_tokens) return MIXKVQ_E_CAPACITY;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (cache->attn_kind != 0 || cache->n_sink[layer] < cache->cfg.sink_len) {
+  const int B = cache->cfg.batch;
+  bool sink_room = false;
+  for (int b = 0; b < B; ++b) sink_room = sink_room || cache->n_sink[fi(cache, layer, b)] < cache->cfg.sink_len;
+  if (cache->attn_kind != 0 || sink_room) {
     // the comparison kernels do not take the new token themselves, and a sink token is not a residual token:
     // plain append, then attention
     int rc = mixkvq_quantize_append(cache, layer, k_dev, v_dev, q_dev, 1, stream);
     if (rc != MIXKVQ_OK) return rc;
     return run_attention(cache, layer, q_dev, out_dev, softmax_scale, static_cast<float*>(workspace_dev), st);
   }
-  if (cache->r[layer] == cache->R) {
-    LayerView lv = view(cache, layer);
-    if (launch_flush(lv, st) != cudaSuccess) return MIXKVQ_E_CUDA;
-    cache->launches += 1;
-    cache->last_packed_writer = layer;
-    cache->n_blocks[layer] += 1;
-    cache->r[layer] = 0;
+  // full windows are flushed first, one launch per run of neighbouring sequences with the same fill
+  for (int b0 = 0; b0 < B;) {
+    int b1 = b0 + 1;
+    while (b1 < B && same_fill(cache, layer, b0, b1)) ++b1;
+    if (cache->r[fi(cache, layer, b0)] == cache->R) {
+      LayerView lv = view(cache, layer, b0, b1 - b0);
+      if (launch_flush(lv, st) != cudaSuccess) return MIXKVQ_E_CUDA;
+      cache->launches += 1;
+      cache->last_packed_writer = layer;
+      for (int b = b0; b < b1; ++b) {
+        cache->n_blocks[fi(cache, layer, b)] += 1;
+        cache->r[fi(cache, layer, b)] = 0;
+      }
+    }
+    b0 = b1;
   }
-  cache->r[layer] += 1;        // the attention kernel stores the token at slot r - 1 and accumulates |q|
+  for (int b = 0; b < B; ++b) cache->r[fi(cache, layer, b)] += 1;   // the attention kernel stores the token at slot r - 1 and accumulates |q|
   const int rc = run_attention(cache, layer, q_dev, out_dev, softmax_scale, static_cast<float*>(workspace_dev), st, k_dev, v_dev);
-  if (rc != MIXKVQ_OK) cache->r[layer] -= 1;      // nothing was enqueued: the token is not part of the layer
+  if (rc != MIXKVQ_OK)
+    for (int b = 0; b < B; ++b) cache->r[fi(cache, layer, b)] -= 1;   // nothing was enqueued: the token is not part of the layer
   return rc;
 }
 
@@ -351,7 +482,7 @@ int mixkvq_prefill(mixkvq_cache* cache, int layer, const void* k_dev, const void
   if (!aligned16(k_dev) || !aligned16(v_dev) || !aligned16(q_dev) || !aligned16(out_dev) || !aligned16(scratch_dev))
     return MIXKVQ_E_ALIGNMENT;
   // the prompt attends to itself only: the layer must be empty
-  if (cache->n_blocks[layer] != 0 || cache->r[layer] != 0 || cache->n_sink[layer] != 0) return MIXKVQ_E_UNSUPPORTED;
+  if (!all_empty(cache, layer)) return MIXKVQ_E_UNSUPPORTED;
   if (n_tokens > cache->cfg.max_tokens ||
       scratch_bytes < prefill_scratch_bytes(cache->cfg.batch, cache->cfg.n_kv_heads, n_tokens))
     return MIXKVQ_E_CAPACITY;
@@ -371,8 +502,7 @@ int mixkvq_rope_append(mixkvq_cache* cache, int layer, void* k_dev, const void* 
     return MIXKVQ_E_INVALID_ARG;
   if (!aligned16(k_dev) || !aligned16(v_dev) || !aligned16(q_dev) || !aligned16(cos_dev) || !aligned16(sin_dev))
     return MIXKVQ_E_ALIGNMENT;
-  const long long have = (long long)cache->n_sink[layer] + (long long)cache->n_blocks[layer] * cache->R + cache->r[layer];
-  if (have + n_tokens > cache->cfg.max_tokens) return MIXKVQ_E_CAPACITY;      // nothing is rotated either
+  if (max_tokens_held(cache, layer) + n_tokens > cache->cfg.max_tokens) return MIXKVQ_E_CAPACITY;      // nothing is rotated either
   if (launch_rope(k_dev, q_dev, cos_dev, sin_dev, cache->cfg.batch, cache->cfg.n_kv_heads, cache->cfg.n_q_heads, n_tokens,
                   pos0, static_cast<cudaStream_t>(stream)) != cudaSuccess)
     return MIXKVQ_E_CUDA;
@@ -391,8 +521,7 @@ int mixkvq_rope_decode_step(mixkvq_cache* cache, int layer, void* k_dev, const v
       !aligned16(out_dev) || !aligned16(workspace_dev))
     return MIXKVQ_E_ALIGNMENT;
   if (workspace_bytes_given < workspace_bytes(cache->S)) return MIXKVQ_E_BUFFER_TOO_SMALL;
-  const long long have = (long long)cache->n_sink[layer] + (long long)cache->n_blocks[layer] * cache->R + cache->r[layer];
-  if (have + 1 > cache->cfg.max_tokens) return MIXKVQ_E_CAPACITY;
+  if (max_tokens_held(cache, layer) + 1 > cache->cfg.max_tokens) return MIXKVQ_E_CAPACITY;
   if (launch_rope(k_dev, q_dev, cos_dev, sin_dev, cache->cfg.batch, cache->cfg.n_kv_heads, cache->cfg.n_q_heads, 1, pos,
                   static_cast<cudaStream_t>(stream)) != cudaSuccess)
     return MIXKVQ_E_CUDA;
@@ -417,7 +546,7 @@ int mixkvq_decode_attention_noalloc(mixkvq_cache* cache, int layer, const void* 
   if (!cache || !q_dev || !out_dev || layer < 0 || layer >= cache->cfg.n_layers) return MIXKVQ_E_INVALID_ARG;
   if (!aligned16(q_dev) || !aligned16(out_dev)) return MIXKVQ_E_ALIGNMENT;
   if (cache->S > MIXKVQ_NOALLOC_MAX_STREAMS) return MIXKVQ_E_BUILTIN_SCRATCH;
-  if (cache->n_blocks[layer] == 0 && cache->r[layer] == 0 && cache->n_sink[layer] == 0) return MIXKVQ_E_EMPTY;
+  if (all_empty(cache, layer)) return MIXKVQ_E_EMPTY;
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MIXKVQ_E_CUDA;
   // the scratch array of the CURRENT device is used: it must be the device that holds the cache memory
@@ -475,11 +604,20 @@ int mixkvq_cache_describe(const mixkvq_cache* cache, int layer, mixkvq_layout_de
   out->base_bytes = cache->base_bytes;
   out->max_blocks = (uint32_t)cache->max_blocks;
   out->n_streams = (uint32_t)cache->S;
-  out->n_blocks = (uint32_t)cache->n_blocks[layer];
-  out->residual_tokens = (uint32_t)cache->r[layer];
+  out->n_blocks = (uint32_t)cache->n_blocks[fi(cache, layer, 0)];
+  out->residual_tokens = (uint32_t)cache->r[fi(cache, layer, 0)];
   out->sink_off = L + cache->sink_off;     out->sink_stride = cache->sink_stride;
-  out->sink_tokens = (uint32_t)cache->n_sink[layer];
+  out->sink_tokens = (uint32_t)cache->n_sink[fi(cache, layer, 0)];
   out->sink_len = (uint32_t)cache->cfg.sink_len;
+  return MIXKVQ_OK;
+}
+
+int mixkvq_sequence_fill(const mixkvq_cache* cache, int layer, int b, uint32_t* n_blocks, uint32_t* residual_tokens,
+                         uint32_t* sink_tokens) {
+  if (!cache || layer < 0 || layer >= cache->cfg.n_layers || b < 0 || b >= cache->cfg.batch) return MIXKVQ_E_INVALID_ARG;
+  if (n_blocks) *n_blocks = (uint32_t)cache->n_blocks[fi(cache, layer, b)];
+  if (residual_tokens) *residual_tokens = (uint32_t)cache->r[fi(cache, layer, b)];
+  if (sink_tokens) *sink_tokens = (uint32_t)cache->n_sink[fi(cache, layer, b)];
   return MIXKVQ_OK;
 }
 

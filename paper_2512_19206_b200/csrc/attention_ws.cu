@@ -25,7 +25,8 @@
 namespace mixkvq {
 
 cudaError_t launch_combine(const float* ws, float* out, int g, int Hkv, int Hq, int mode, int n,
-                           long long units_per_stream, int S, cudaStream_t stream);
+                           long long units_per_stream, int S, cudaStream_t stream, const int4* seq = nullptr,
+                           const int* seq_prefix = nullptr);
 
 namespace {
 
@@ -281,12 +282,13 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
   constexpr int UPG = G / 32;                                 // units per key group
 
   const int S = lv.B * lv.Hkv, U = lv.U, g = lv.g;
-  const int packed_units = lv.n_blocks * U;
+  // Fill of the stream at hand: the same for every stream, or (ragged batch) taken per sequence from the table in
+  // device memory at the start of every segment.
+  int f_nb = lv.n_blocks, f_r = lv.r, f_ns = lv.n_sink;
+  int packed_units = f_nb * U;
   // unquantized 32-token units: those of the residual window, then those of the sink
-  const int res_units = (lv.r + 31) / 32, bf16_units = res_units + (lv.n_sink + 31) / 32;
-  const int Us = packed_units + kResidualWeight * bf16_units;             // split positions; an unquantized unit spans several
-  const long long total = (long long)Us * S;
-  const long long cb = split_begin(total, gridDim.x, blockIdx.x), ce = split_begin(total, gridDim.x, blockIdx.x + 1);
+  int res_units = (f_r + 31) / 32, bf16_units = res_units + (f_ns + 31) / 32;
+  int Us = packed_units + kResidualWeight * bf16_units;             // split positions; an unquantized unit spans several
 
   // Programmatic dependent launch: the grid may have been started while the kernel before it in the stream was still
   // running.  Nothing above touches global memory.  dep_wait() waits for that kernel's results and lets the kernel after
@@ -302,7 +304,9 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
       dep_waited = true;
     }
   };
-  if (!lv.stage_early) dep_wait();
+  if (!lv.stage_early || lv.seq != nullptr) dep_wait();     // the table of a ragged batch is read right below
+  const long long total = lv.seq != nullptr ? (long long)lv.seq_prefix[lv.B] : (long long)Us * S;
+  const long long cb = split_begin(total, gridDim.x, blockIdx.x), ce = split_begin(total, gridDim.x, blockIdx.x + 1);
 
   uint32_t ring_stage = 0;        // ring stage of the next packed unit this pair consumes
   uint32_t ring_parity = 0;       // phase parity of that stage's barriers
@@ -320,9 +324,26 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
   };
 
   for (long long seg = cb; seg < ce;) {
-    const int s = (int)(seg / Us);
-    const int ub = (int)(seg - (long long)s * Us);
-    const int ue = (int)min((long long)Us, ce - (long long)s * Us);
+    int s, ub, ue;
+    if (lv.seq != nullptr) {
+      // ragged batch: the sequence whose positions hold seg (sequences without positions are stepped over)
+      int b = 0;
+      while (b + 1 < lv.B && (long long)lv.seq_prefix[b + 1] <= seg) ++b;
+      const int4 f = lv.seq[b];
+      f_nb = f.x; f_r = f.y; f_ns = f.z; Us = f.w;
+      packed_units = f_nb * U;
+      res_units = (f_r + 31) / 32;
+      bf16_units = res_units + (f_ns + 31) / 32;
+      const long long rel = seg - (long long)lv.seq_prefix[b];
+      const int hk = (int)(rel / Us);
+      s = b * lv.Hkv + hk;
+      ub = (int)(rel - (long long)hk * Us);
+      ue = (int)min((long long)Us, ce - (long long)lv.seq_prefix[b] - (long long)hk * Us);
+    } else {
+      s = (int)(seg / Us);
+      ub = (int)(seg - (long long)s * Us);
+      ue = (int)min((long long)Us, ce - (long long)s * Us);
+    }
     seg += ue - ub;
     // ---- this pair's share of the segment.  The unquantized units of the segment go to different pairs (unit i to
     // pair kPairs - 1 - i % kPairs); the packed units are split in order so that every pair carries about the same weight.
@@ -413,7 +434,7 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
     const int first_res = kPairs - 1 - pair;
     // fused decode step: the newest token (slot r - 1) is not in the residual store yet; the pair whose unit holds it
     // takes its rows from the step's tensors, stores them and updates the importance accumulator
-    const int jn = lv.r - 1;
+    const int jn = f_r - 1;
 
     if (logits_role) {
       // =====================================================================================================
@@ -427,7 +448,7 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
         const int bu = res_b + ri;                        // unquantized unit: residual window first, then the sink
         const bool in_sink = bu >= res_units;
         const int wu = in_sink ? bu - res_units : bu;     // unit inside its window
-        const int rt = in_sink ? lv.n_sink : lv.r;        // tokens in that window
+        const int rt = in_sink ? f_ns : f_r;        // tokens in that window
         const int j0 = wu * 32;
         const char* resk = in_sink ? lv.sink + (size_t)s * lv.sink_stride : lv.resk + (size_t)s * lv.resk_stride;
         const bool holds_new = !in_sink && lv.new_k != nullptr && jn >= j0 && jn < j0 + 32;
@@ -519,7 +540,7 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
         // ---- a block: its table entry, its promoted channels' query entries
         const uint2 entry = pf_entry;
         const uint4 head = pf_head;              // the first 16 bytes of the block's extras: up to 8 pairs of promoted channels
-        if (bi + 1 < lv.n_blocks) pf_entry = table[bi + 1];
+        if (bi + 1 < f_nb) pf_entry = table[bi + 1];
         const int n16 = entry.y & 0xFF, n4 = (entry.y >> 8) & 0xFF, n16p = (n16 + 1) >> 1;
         const char* ex = extras + (size_t)entry.x * 16;                       // the block's extras
         const uint32_t ex_unit = extras_unit_bytes(n16, n4, kU4 == 2);
@@ -768,7 +789,7 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
         u = 0;
         ++bi;
         // the next block's channel lists (its table entry has arrived by now)
-        if (bi < lv.n_blocks && (pf_entry.y & 0xFFFFu)) pf_head = *reinterpret_cast<const uint4*>(extras + (size_t)pf_entry.x * 16);
+        if (bi < f_nb && (pf_entry.y & 0xFFFFu)) pf_head = *reinterpret_cast<const uint4*>(extras + (size_t)pf_entry.x * 16);
       }
       if (gave_up && lane == 0) atomicOr(lv.status, (uint32_t)MIXKVQ_DEV_COPY_TIMEOUT);
     } else {
@@ -805,7 +826,7 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
         const int bu = res_b + ri;
         const bool in_sink = bu >= res_units;
         const int wu = in_sink ? bu - res_units : bu;
-        const int rt = in_sink ? lv.n_sink : lv.r;
+        const int rt = in_sink ? f_ns : f_r;
         const int j0 = wu * 32;
         const char* resv = in_sink ? lv.sink + (size_t)s * lv.sink_stride + (size_t)lv.sink_len * 256
                                    : lv.resv + (size_t)s * lv.resv_stride;
@@ -1158,14 +1179,20 @@ long long attention_ws_positions(const LayerView& lv) {
   return (long long)lv.n_blocks * lv.U + (long long)kResidualWeight * ((lv.r + 31) / 32 + (lv.n_sink + 31) / 32);
 }
 
+// Split positions of one stream with the given fill (the entry w of a ragged batch's table)
+int attention_ws_positions_of(int n_blocks, int r, int n_sink, int U) {
+  return n_blocks * U + kResidualWeight * ((r + 31) / 32 + (n_sink + 31) / 32);
+}
+
 // Number of CTAs the split kernel runs for this layer state (also the number of partial-slot owners).  When there are
 // fewer streams than CTA slots the grid is a multiple of the stream count, so that no CTA straddles two streams
-// (a second segment costs a pipeline drain, a query load and a second partial).
+// (a second segment costs a pipeline drain, a query load and a second partial).  Ragged batch: the positions of all
+// streams are split evenly, wherever the boundaries fall.
 int attention_ws_grid(const LayerView& lv, int n_sms) {
   const int S = lv.B * lv.Hkv;
-  const long long total = attention_ws_positions(lv) * S;
+  const long long total = lv.seq != nullptr ? lv.seq_total : attention_ws_positions(lv) * S;
   int grid = (int)min((long long)min(n_sms * kCtasPerSm, kMaxCtas / 2), total);
-  if (grid > S) grid = grid / S * S;
+  if (grid > S && lv.seq == nullptr) grid = grid / S * S;
   return grid < 1 ? 1 : grid;
 }
 
@@ -1180,7 +1207,7 @@ cudaError_t launch_attention_ws(const LayerView& lv, const void* q, float* out, 
   else e = launch_g<128>(lv, q, scale, ws, grid, stream);
   *launches = 1;
   if (e != cudaSuccess || out == nullptr) return e;     // out == nullptr: split kernel only (timing)
-  e = launch_combine(ws, out, lv.g, lv.Hkv, lv.Hq, 1, grid, Us, S, stream);
+  e = launch_combine(ws, out, lv.g, lv.Hkv, lv.Hq, 1, grid, Us, S, stream, lv.seq, lv.seq_prefix);
   *launches = 2;
   return e;
 }

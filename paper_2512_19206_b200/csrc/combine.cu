@@ -8,12 +8,23 @@ namespace mixkvq {
 // S*units_per_stream work units evenly; CTA c wrote its part of stream s to slot c + s.
 __global__ void __launch_bounds__(128)
 combine_kernel(const float* __restrict__ ws, float* __restrict__ out, int g, int Hkv, int Hq, int mode, int n,
-               long long units_per_stream, int S) {
+               long long units_per_stream, int S, const int4* __restrict__ seq, const int* __restrict__ seq_prefix) {
   const int s = blockIdx.x / g, h = blockIdx.x % g, c = threadIdx.x;
   int first, count;
+  // started early (programmatic dependent launch): wait here for the kernel that wrote the partials
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (mode == 0) {
     first = s * n;
     count = n;
+  } else if (seq != nullptr) {
+    // ragged batch: sequence b's streams own positions [prefix[b] + hk * w, + w), w = seq[b].w (none when w == 0)
+    const int bq = s / Hkv, w = seq[bq].w;
+    const long long total = seq_prefix[S / Hkv];
+    const long long x0 = (long long)seq_prefix[bq] + (long long)(s % Hkv) * w, x1 = x0 + w - 1;
+    const int c0 = w ? (int)(((x0 + 1) * n - 1) / total) : 0, c1 = w ? (int)(((x1 + 1) * n - 1) / total) : -1;
+    first = c0 + s;
+    count = c1 - c0 + 1;
   } else {
     const long long total = units_per_stream * S;
     const long long x0 = units_per_stream * s, x1 = units_per_stream * (s + 1) - 1;
@@ -23,9 +34,6 @@ combine_kernel(const float* __restrict__ ws, float* __restrict__ out, int g, int
   }
   const int b = s / Hkv, hk = s % Hkv;
   const float* base = ws + (size_t)first * kPartialFloats + h * 130;
-  // started early (programmatic dependent launch): wait here for the kernel that wrote the partials
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // one pass with a running maximum; the loads of a chunk of partials are independent of one another, so a stream with
   // up to kChunk partials costs one round trip to memory
   constexpr int kChunk = 12;
@@ -54,12 +62,13 @@ combine_kernel(const float* __restrict__ ws, float* __restrict__ out, int g, int
     }
     M = Mn;
   }
-  // l == 0 only when every split gave up (its partial is then m = -inf, l = 0, o = 0 and the status word says so)
+  // l == 0 only when every split gave up (its partial is then m = -inf, l = 0, o = 0 and the status word says so) or
+  // when the sequence of a ragged batch holds no token
   out[((size_t)b * Hq + hk * g + h) * kD + c] = l > 0.f ? o / l : 0.f;
 }
 
 cudaError_t launch_combine(const float* ws, float* out, int g, int Hkv, int Hq, int mode, int n,
-                           long long units_per_stream, int S, cudaStream_t stream) {
+                           long long units_per_stream, int S, cudaStream_t stream, const int4* seq, const int* seq_prefix) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(S * g));
   cfg.blockDim = dim3(128);
@@ -69,7 +78,26 @@ cudaError_t launch_combine(const float* ws, float* out, int g, int Hkv, int Hq, 
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, combine_kernel, ws, out, g, Hkv, Hq, mode, n, units_per_stream, S);
+  return cudaLaunchKernelEx(&cfg, combine_kernel, ws, out, g, Hkv, Hq, mode, n, units_per_stream, S, seq, seq_prefix);
+}
+
+// The table of a ragged batch, from the host's per-sequence fill (kernel arguments: no copy, ordered in the stream).
+__global__ void seq_table_kernel(SeqTableArgs a, int4* __restrict__ seq, int* __restrict__ seq_prefix) {
+  const int b = threadIdx.x;
+  if (b < a.n) seq[b] = make_int4(a.fill[3 * b], a.fill[3 * b + 1], a.fill[3 * b + 2], a.w[b]);
+  if (b == 0) {
+    int acc = 0;
+    for (int i = 0; i < a.n; ++i) {
+      seq_prefix[i] = acc;
+      acc += a.Hkv * a.w[i];
+    }
+    seq_prefix[a.n] = acc;
+  }
+}
+
+cudaError_t launch_seq_table(const SeqTableArgs& a, int4* seq, int* seq_prefix, cudaStream_t stream) {
+  seq_table_kernel<<<1, kMaxRaggedBatch, 0, stream>>>(a, seq, seq_prefix);
+  return cudaGetLastError();
 }
 
 // Two sets of partials per stream (packed blocks, residual window), each written by a grid that split its

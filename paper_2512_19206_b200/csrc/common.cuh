@@ -19,6 +19,8 @@ constexpr int kMaxCtas = 148 * 8;       // upper bound on the attention grid (si
 enum Tier : uint8_t { kU2 = 0, kU4 = 1, kBF16 = 2 };
 
 // Geometry + pointers of one layer, passed by value to every kernel.
+constexpr int kMaxRaggedBatch = 128;   // sequences of a batch whose fills may differ
+
 struct LayerView {
   // geometry
   int B, Hq, Hkv, g;          // batch, query heads, KV heads, GQA group size
@@ -56,6 +58,12 @@ struct LayerView {
   // test hook for the give-up path: the barrier of every warp pair's first staged copy is armed for this many bytes
   // more than are copied, so that it never completes (0 in normal use)
   uint32_t debug_extra_tx;
+  // Ragged batch (sequences of different fill): per sequence (n_blocks, r, n_sink, split positions of one of its
+  // streams) and the prefix sums over the sequences of Hkv * positions ([B + 1], the last one = seq_total), both in
+  // device memory; null when every sequence has the fill n_blocks, r, n_sink above.
+  const int4* seq;
+  const int* seq_prefix;
+  long long seq_total;
 };
 
 __host__ __device__ inline uint32_t extras_header_bytes(int n16, int n4) {
@@ -189,6 +197,10 @@ cudaError_t launch_prefill_attention(const void* q, const void* k, const void* v
                                      int Hkv, int L, float scale, uint32_t* status, uint32_t max_polls, cudaStream_t stream);
 size_t prefill_scratch_bytes(int B, int Hkv, int L);
 cudaError_t prefill_attention_setup();
+int attention_ws_positions_of(int n_blocks, int r, int n_sink, int U);
+// writes a ragged batch's table: fill[3 b + {0, 1, 2}] = (n_blocks, r, n_sink) of sequence b, positions w[b] per stream
+struct SeqTableArgs { int n, Hkv; int fill[3 * kMaxRaggedBatch]; int w[kMaxRaggedBatch]; };
+cudaError_t launch_seq_table(const SeqTableArgs& a, int4* seq, int* seq_prefix, cudaStream_t stream);
 cudaError_t launch_rope(void* k, void* q, const float* cos_t, const float* sin_t, int B, int Hkv, int Hq, int n_tokens,
                         int pos0, cudaStream_t stream);
 cudaError_t launch_flush(const LayerView& lv, cudaStream_t stream);

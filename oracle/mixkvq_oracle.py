@@ -21,6 +21,9 @@ What each function follows:
 * ``effective_bits`` / ``fp16_cache_bytes``  B_eff of Appendix C; the footprint example of Section 1.
 * ``causal_attention``                    Eq. 1 for the prompt (the prefill phase of Section 4.2): every position attends
                                           to itself and the positions before it, full precision, fp64.
+* ``OracleStream.attention_partial`` /    Eq. 1 over a sequence whose tokens are spread over several caches (a context
+  ``merge_partials``                      split over GPUs): each cache's output and log-denominator, merged by the
+                                          log-sum-exp identity; equal to Eq. 1 over all tokens by construction.
 * ``rope``                                the rotary embedding that Appendix D puts before the scores ("saliency
                                           evaluation is performed post-transformation"): keys and queries are
                                           rotated, then appended.
@@ -319,6 +322,34 @@ class OracleStream:
         if return_probs:
             return o.astype(np.float32), p
         return o.astype(np.float32)
+
+    def attention_partial(self, q, scale):
+        """Eq. 1 restricted to the tokens this stream holds, in the form a sequence split needs: (o, lse) with
+        o float64 [g, D] the softmax-weighted values over these tokens alone and lse float64 [g] the natural
+        logarithm of the softmax denominator sum_j exp(scale q.k_j).  A stream without tokens gives o = 0, lse = -inf."""
+        Kt, Vt = self.keys(), self.values()
+        g = np.asarray(q).shape[0]
+        if Kt.shape[0] == 0:
+            return np.zeros((g, D), np.float64), np.full(g, -np.inf)
+        logits = (np.asarray(q, np.float32).astype(np.float64) @ Kt.T) * float(scale)
+        m = logits.max(axis=1, keepdims=True)
+        p = np.exp(logits - m)
+        den = p.sum(axis=1, keepdims=True)
+        return (p @ Vt) / den, (m + np.log(den))[:, 0]
+
+
+def merge_partials(os, lses):
+    """Softmax attention over the union of disjoint token sets from the per-set results (the log-sum-exp identity):
+    with w_r = exp(lse_r),  o = sum_r w_r o_r / sum_r w_r.  os [n, ..., D], lses [n, ...] (fp64); parts with
+    lse = -inf (no tokens) carry weight 0; if every part is empty the result is 0."""
+    os = np.asarray(os, np.float64)
+    lses = np.asarray(lses, np.float64)
+    top = lses.max(axis=0)
+    safe = np.where(np.isfinite(top), top, 0.0)
+    w = np.exp(lses - safe)                       # exp(-inf) = 0 for the empty parts
+    den = w.sum(axis=0)
+    num = (w[..., None] * os).sum(axis=0)
+    return np.where(den[..., None] > 0, num / np.where(den > 0, den, 1.0)[..., None], 0.0)
 
 
 def rope(x, cos, sin):

@@ -192,6 +192,23 @@ int mixkvq_quantize_append_ragged(mixkvq_cache* cache, int layer, const void* k_
 int mixkvq_sequence_fill(const mixkvq_cache* cache, int layer, int b, uint32_t* n_blocks, uint32_t* residual_tokens,
                          uint32_t* sink_tokens);
 
+/* Decode attention for a context whose tokens are spread over several caches (one per GPU: a sequence split for
+ * contexts beyond one GPU's memory).  Eq. 1 over this cache's tokens alone, in the form the merge needs:
+ *   out_dev [B, Hq, 128] float: softmax-weighted values over this cache's tokens (normalised by this cache's own
+ *   denominator);  lse_dev [B, Hq] float: natural logarithm of that denominator sum_j exp(scale q.k_j).
+ * A sequence (or a whole cache) without tokens gives zeros and lse = -inf.  Same kernels, workspace and queue
+ * behaviour as mixkvq_decode_attention; fragment layout and the default kernel only (MIXKVQ_E_UNSUPPORTED otherwise). */
+int mixkvq_decode_attention_partial(mixkvq_cache* cache, int layer, const void* q_dev, float* out_dev, float* lse_dev,
+                                    float softmax_scale, void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/* Eq. 1 over the union of disjoint token sets from the per-set results of mixkvq_decode_attention_partial (the
+ * log-sum-exp identity): out = sum_r w_r o_r / sum_r w_r, w_r = exp(lse_r - max_r lse_r).  Stateless.
+ *   o_parts_dev [n_parts, rows, 128] float, lse_parts_dev [n_parts, rows] float (rows = B * Hq; the layout an
+ *   all-gather of the ranks' results produces)  ->  out_dev [rows, 128] float.  Parts with lse = -inf weigh 0;
+ *   rows whose parts are all empty come out as zeros.  1 <= n_parts <= 1024. */
+int mixkvq_merge_partials(const float* o_parts_dev, const float* lse_parts_dev, int n_parts, int rows, float* out_dev,
+                          void* stream);
+
 /* The prefill phase of Section 4.2 for one layer: causal attention of the prompt over itself in full precision (Eq. 1,
  * position i sees positions 0..i), then the prompt's keys and values go into the cache exactly as
  * mixkvq_quantize_append(n_tokens) would put them (complete windows quantized, the last 1..R tokens in the residual

@@ -19,7 +19,7 @@ EXPORTS = [
     "mixkvq_select_channels", "mixkvq_select_channels_raw", "mixkvq_quantize_append",
     "mixkvq_decode_attention", "mixkvq_decode_attention_noalloc", "mixkvq_decode_step", "mixkvq_set_attention_kernel", "mixkvq_query_status",
     "mixkvq_cache_describe", "mixkvq_launch_count", "mixkvq_status_string",
-    "mixkvq_cache_written_externally", "mixkvq_test_arm_copy_timeout", "mixkvq_rope_append", "mixkvq_rope_decode_step", "mixkvq_prefill", "mixkvq_prefill_scratch_bytes", "mixkvq_quantize_append_ragged", "mixkvq_sequence_fill",
+    "mixkvq_cache_written_externally", "mixkvq_test_arm_copy_timeout", "mixkvq_rope_append", "mixkvq_rope_decode_step", "mixkvq_prefill", "mixkvq_prefill_scratch_bytes", "mixkvq_quantize_append_ragged", "mixkvq_sequence_fill", "mixkvq_decode_attention_partial", "mixkvq_merge_partials",
 ]
 
 DEV_EXTRAS_FULL, DEV_COPY_TIMEOUT = 1, 2
@@ -74,6 +74,8 @@ def lib():
         L.mixkvq_set_attention_kernel.argtypes = [vp, i32]
         L.mixkvq_quantize_append_ragged.argtypes = [vp, i32, vp, vp, vp, i32, C.POINTER(C.c_int32), vp]
         L.mixkvq_sequence_fill.argtypes = [vp, i32, i32, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)]
+        L.mixkvq_decode_attention_partial.argtypes = [vp, i32, vp, vp, vp, f32, vp, C.c_size_t, vp]
+        L.mixkvq_merge_partials.argtypes = [vp, vp, i32, i32, vp, vp]
         L.mixkvq_prefill.argtypes = [vp, i32, vp, vp, vp, i32, vp, f32, vp, C.c_size_t, vp]
         L.mixkvq_prefill_scratch_bytes.argtypes = [C.POINTER(Config), i32]
         L.mixkvq_prefill_scratch_bytes.restype = C.c_size_t
@@ -126,6 +128,19 @@ def cache_bytes(cfg: Config):
     a, b = C.c_size_t(), C.c_size_t()
     _check(lib().mixkvq_cache_bytes(C.byref(cfg), C.byref(a), C.byref(b)), "mixkvq_cache_bytes")
     return a.value, b.value
+
+
+def merge_partials(o_parts: torch.Tensor, lse_parts: torch.Tensor, out=None):
+    """o_parts [n, ..., 128], lse_parts [n, ...] float32 (device) -> [..., 128]: attention over the union of the parts."""
+    n = o_parts.shape[0]
+    rows = lse_parts[0].numel()
+    if out is None:
+        out = torch.empty(o_parts.shape[1:], dtype=torch.float32, device=o_parts.device)
+    if not (o_parts.is_cuda and o_parts.is_contiguous() and lse_parts.is_contiguous()):
+        raise ValueError("merge_partials needs contiguous CUDA tensors")
+    _check(lib().mixkvq_merge_partials(_ptr(o_parts), _ptr(lse_parts), n, rows, _ptr(out), _stream()),
+           "mixkvq_merge_partials")
+    return out
 
 
 def select_channels_raw(q: torch.Tensor, k: torch.Tensor, score_bits, tau_bf16, tau_u4, want_salience=True):
@@ -188,6 +203,18 @@ class Cache:
         _check(lib().mixkvq_decode_step(self.handle, layer, _ptr(k), _ptr(v), _ptr(q), _ptr(out), float(scale),
                                         _ptr(self.workspace), self.workspace.numel(), _stream()), "mixkvq_decode_step")
         return out
+
+    def decode_attention_partial(self, layer, q, scale, out=None, lse=None):
+        """q [B,Hq,128] bf16 -> (out [B,Hq,128], lse [B,Hq]) float32: attention over this cache's tokens alone and the
+        natural log of its softmax denominator (the inputs of merge_partials)."""
+        if out is None:
+            out = torch.empty(q.shape, dtype=torch.float32, device=q.device)
+        if lse is None:
+            lse = torch.empty(q.shape[:2], dtype=torch.float32, device=q.device)
+        _check(lib().mixkvq_decode_attention_partial(self.handle, layer, _ptr(q), _ptr(out), _ptr(lse), float(scale),
+                                                     _ptr(self.workspace), self.workspace.numel(), _stream()),
+               "mixkvq_decode_attention_partial")
+        return out, lse
 
     def quantize_append_ragged(self, layer, k, v, q, counts):
         """k, v [B,Hkv,n_max,128], q [B,Hq,n_max,128] bf16; counts: per-sequence token counts (host ints)."""

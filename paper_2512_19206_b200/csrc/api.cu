@@ -169,7 +169,7 @@ int zero_layer_state(mixkvq_cache* h, int layer, cudaStream_t st) {
 
 // Picks the decode-attention kernel for the layer's layout and the selected kind, enqueues it and counts its launches.
 int run_attention(mixkvq_cache* h, int layer, const void* q, float* out, float scale, float* ws, cudaStream_t st,
-                  const void* new_k = nullptr, const void* new_v = nullptr) {
+                  const void* new_k = nullptr, const void* new_v = nullptr, float* lse = nullptr) {
   LayerView lv = view(h, layer);
   lv.new_k = static_cast<const uint16_t*>(new_k);
   lv.new_v = static_cast<const uint16_t*>(new_v);
@@ -211,7 +211,7 @@ int run_attention(mixkvq_cache* h, int layer, const void* q, float* out, float s
   else if (h->tile)
     e = launch_attention_tc(lv, q, h->attn_kind == 2 ? nullptr : out, scale, ws, h->n_sms, st, &launches);
   else
-    e = launch_attention_ws(lv, q, h->attn_kind == 2 ? nullptr : out, scale, ws, h->n_sms, st, &launches);
+    e = launch_attention_ws(lv, q, h->attn_kind == 2 ? nullptr : out, scale, ws, h->n_sms, st, &launches, lse);
   h->launches += launches;
   return e == cudaSuccess ? MIXKVQ_OK : MIXKVQ_E_CUDA;
 }
@@ -424,6 +424,32 @@ int mixkvq_decode_attention(mixkvq_cache* cache, int layer, const void* q_dev, f
   if (all_empty(cache, layer)) return MIXKVQ_E_EMPTY;
   return run_attention(cache, layer, q_dev, out_dev, softmax_scale, static_cast<float*>(workspace_dev),
                        static_cast<cudaStream_t>(stream));
+}
+
+int mixkvq_decode_attention_partial(mixkvq_cache* cache, int layer, const void* q_dev, float* out_dev, float* lse_dev,
+                                    float softmax_scale, void* workspace_dev, size_t workspace_bytes_given, void* stream) {
+  if (!cache || !q_dev || !out_dev || !lse_dev || !workspace_dev || layer < 0 || layer >= cache->cfg.n_layers)
+    return MIXKVQ_E_INVALID_ARG;
+  if (!aligned16(q_dev) || !aligned16(out_dev) || !aligned16(workspace_dev)) return MIXKVQ_E_ALIGNMENT;
+  if (workspace_bytes_given < workspace_bytes(cache->S)) return MIXKVQ_E_BUFFER_TOO_SMALL;
+  if (cache->tile || cache->attn_kind != 0) return MIXKVQ_E_UNSUPPORTED;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (all_empty(cache, layer)) {
+    // this cache holds no token of the context: weight 0 in the merge
+    cache->launches += 1;
+    return launch_empty_partial(out_dev, lse_dev, cache->cfg.batch * cache->cfg.n_q_heads, st) == cudaSuccess
+               ? MIXKVQ_OK : MIXKVQ_E_CUDA;
+  }
+  return run_attention(cache, layer, q_dev, out_dev, softmax_scale, static_cast<float*>(workspace_dev), st, nullptr, nullptr,
+                       lse_dev);
+}
+
+int mixkvq_merge_partials(const float* o_parts_dev, const float* lse_parts_dev, int n_parts, int rows, float* out_dev,
+                          void* stream) {
+  if (!o_parts_dev || !lse_parts_dev || !out_dev || n_parts < 1 || n_parts > 1024 || rows < 1) return MIXKVQ_E_INVALID_ARG;
+  if (!aligned16(o_parts_dev) || !aligned16(out_dev)) return MIXKVQ_E_ALIGNMENT;
+  return launch_merge_partials(o_parts_dev, lse_parts_dev, n_parts, rows, out_dev, static_cast<cudaStream_t>(stream)) ==
+                 cudaSuccess ? MIXKVQ_OK : MIXKVQ_E_CUDA;
 }
 
 int mixkvq_decode_step(mixkvq_cache* cache, int layer, const void* k_dev, const void* v_dev, const void* q_dev,

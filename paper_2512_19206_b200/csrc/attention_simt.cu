@@ -7,7 +7,7 @@ namespace mixkvq {
 
 cudaError_t launch_combine(const float* ws, float* out, int g, int Hkv, int Hq, int mode, int n,
                            long long units_per_stream, int S, cudaStream_t stream, const int4* seq = nullptr,
-                           const int* seq_prefix = nullptr);
+                           const int* seq_prefix = nullptr, float* lse_out = nullptr);
 
 __global__ void __launch_bounds__(128)
 attention_simt_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float scale_log2e, float* __restrict__ ws,

@@ -26,7 +26,7 @@ namespace mixkvq {
 
 cudaError_t launch_combine(const float* ws, float* out, int g, int Hkv, int Hq, int mode, int n,
                            long long units_per_stream, int S, cudaStream_t stream, const int4* seq = nullptr,
-                           const int* seq_prefix = nullptr);
+                           const int* seq_prefix = nullptr, float* lse_out = nullptr);
 
 namespace {
 
@@ -1197,7 +1197,7 @@ int attention_ws_grid(const LayerView& lv, int n_sms) {
 }
 
 cudaError_t launch_attention_ws(const LayerView& lv, const void* q, float* out, float scale, float* ws, int n_sms,
-                                cudaStream_t stream, int* launches) {
+                                cudaStream_t stream, int* launches, float* lse_out) {
   const int S = lv.B * lv.Hkv;
   const long long Us = attention_ws_positions(lv);
   const int grid = attention_ws_grid(lv, n_sms);
@@ -1207,7 +1207,7 @@ cudaError_t launch_attention_ws(const LayerView& lv, const void* q, float* out, 
   else e = launch_g<128>(lv, q, scale, ws, grid, stream);
   *launches = 1;
   if (e != cudaSuccess || out == nullptr) return e;     // out == nullptr: split kernel only (timing)
-  e = launch_combine(ws, out, lv.g, lv.Hkv, lv.Hq, 1, grid, Us, S, stream, lv.seq, lv.seq_prefix);
+  e = launch_combine(ws, out, lv.g, lv.Hkv, lv.Hq, 1, grid, Us, S, stream, lv.seq, lv.seq_prefix, lse_out);
   *launches = 2;
   return e;
 }

@@ -8,7 +8,8 @@ namespace mixkvq {
 // S*units_per_stream work units evenly; CTA c wrote its part of stream s to slot c + s.
 __global__ void __launch_bounds__(128)
 combine_kernel(const float* __restrict__ ws, float* __restrict__ out, int g, int Hkv, int Hq, int mode, int n,
-               long long units_per_stream, int S, const int4* __restrict__ seq, const int* __restrict__ seq_prefix) {
+               long long units_per_stream, int S, const int4* __restrict__ seq, const int* __restrict__ seq_prefix,
+               float* __restrict__ lse_out) {
   const int s = blockIdx.x / g, h = blockIdx.x % g, c = threadIdx.x;
   int first, count;
   // started early (programmatic dependent launch): wait here for the kernel that wrote the partials
@@ -65,10 +66,13 @@ combine_kernel(const float* __restrict__ ws, float* __restrict__ out, int g, int
   // l == 0 only when every split gave up (its partial is then m = -inf, l = 0, o = 0 and the status word says so) or
   // when the sequence of a ragged batch holds no token
   out[((size_t)b * Hq + hk * g + h) * kD + c] = l > 0.f ? o / l : 0.f;
+  // natural logarithm of the softmax denominator (the maximum M is kept in the base-2 domain)
+  if (lse_out != nullptr && c == 0) lse_out[(size_t)b * Hq + hk * g + h] = l > 0.f ? (M + log2f(l)) * 0.6931471805599453f : -INFINITY;
 }
 
 cudaError_t launch_combine(const float* ws, float* out, int g, int Hkv, int Hq, int mode, int n,
-                           long long units_per_stream, int S, cudaStream_t stream, const int4* seq, const int* seq_prefix) {
+                           long long units_per_stream, int S, cudaStream_t stream, const int4* seq, const int* seq_prefix,
+                           float* lse_out) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(S * g));
   cfg.blockDim = dim3(128);
@@ -78,7 +82,7 @@ cudaError_t launch_combine(const float* ws, float* out, int g, int Hkv, int Hq, 
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, combine_kernel, ws, out, g, Hkv, Hq, mode, n, units_per_stream, S, seq, seq_prefix);
+  return cudaLaunchKernelEx(&cfg, combine_kernel, ws, out, g, Hkv, Hq, mode, n, units_per_stream, S, seq, seq_prefix, lse_out);
 }
 
 // The table of a ragged batch, from the host's per-sequence fill (kernel arguments: no copy, ordered in the stream).
@@ -97,6 +101,43 @@ __global__ void seq_table_kernel(SeqTableArgs a, int4* __restrict__ seq, int* __
 
 cudaError_t launch_seq_table(const SeqTableArgs& a, int4* seq, int* seq_prefix, cudaStream_t stream) {
   seq_table_kernel<<<1, kMaxRaggedBatch, 0, stream>>>(a, seq, seq_prefix);
+  return cudaGetLastError();
+}
+
+// Softmax attention over the union of disjoint token sets from the per-set results: o = sum_r w_r o_r / sum_r w_r with
+// w_r = exp(lse_r - max_r lse_r).  o_parts [n_parts][rows][128], lse_parts [n_parts][rows]; a part with lse = -inf
+// (no tokens) has weight 0; all parts empty: zeros.
+__global__ void __launch_bounds__(128)
+merge_partials_kernel(const float* __restrict__ o_parts, const float* __restrict__ lse_parts, int n_parts, int rows,
+                      float* __restrict__ out) {
+  const int row = blockIdx.x, c = threadIdx.x;
+  float top = -INFINITY;
+  for (int r = 0; r < n_parts; ++r) top = fmaxf(top, lse_parts[(size_t)r * rows + row]);
+  float den = 0.f, num = 0.f;
+  if (top != -INFINITY) {
+    for (int r = 0; r < n_parts; ++r) {
+      const float w = expf(lse_parts[(size_t)r * rows + row] - top);
+      den += w;
+      num += w * o_parts[((size_t)r * rows + row) * kD + c];
+    }
+  }
+  out[(size_t)row * kD + c] = den > 0.f ? num / den : 0.f;
+}
+
+// The partial of a cache that holds no token: zeros and lse = -inf.
+__global__ void __launch_bounds__(128) empty_partial_kernel(float* __restrict__ out, float* __restrict__ lse) {
+  out[(size_t)blockIdx.x * kD + threadIdx.x] = 0.f;
+  if (threadIdx.x == 0) lse[blockIdx.x] = -INFINITY;
+}
+
+cudaError_t launch_empty_partial(float* out, float* lse, int rows, cudaStream_t stream) {
+  empty_partial_kernel<<<rows, 128, 0, stream>>>(out, lse);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_merge_partials(const float* o_parts, const float* lse_parts, int n_parts, int rows, float* out,
+                                  cudaStream_t stream) {
+  merge_partials_kernel<<<rows, 128, 0, stream>>>(o_parts, lse_parts, n_parts, rows, out);
   return cudaGetLastError();
 }
 

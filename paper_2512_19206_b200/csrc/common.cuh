@@ -201,6 +201,9 @@ int attention_ws_positions_of(int n_blocks, int r, int n_sink, int U);
 // writes a ragged batch's table: fill[3 b + {0, 1, 2}] = (n_blocks, r, n_sink) of sequence b, positions w[b] per stream
 struct SeqTableArgs { int n, Hkv; int fill[3 * kMaxRaggedBatch]; int w[kMaxRaggedBatch]; };
 cudaError_t launch_seq_table(const SeqTableArgs& a, int4* seq, int* seq_prefix, cudaStream_t stream);
+cudaError_t launch_empty_partial(float* out, float* lse, int rows, cudaStream_t stream);
+cudaError_t launch_merge_partials(const float* o_parts, const float* lse_parts, int n_parts, int rows, float* out,
+                                  cudaStream_t stream);
 cudaError_t launch_rope(void* k, void* q, const float* cos_t, const float* sin_t, int B, int Hkv, int Hq, int n_tokens,
                         int pos0, cudaStream_t stream);
 cudaError_t launch_flush(const LayerView& lv, cudaStream_t stream);
@@ -213,7 +216,7 @@ cudaError_t launch_select_raw(const void* q, const void* k, int B, int Hq, int H
 cudaError_t launch_attention_simt(const LayerView& lv, const void* q, float* out, float scale, float* ws,
                                   int n_sms, cudaStream_t stream, int* launches);
 cudaError_t launch_attention_ws(const LayerView& lv, const void* q, float* out, float scale, float* ws,
-                                int n_sms, cudaStream_t stream, int* launches);
+                                int n_sms, cudaStream_t stream, int* launches, float* lse_out = nullptr);
 cudaError_t attention_ws_setup();
 // tile layout (R == 128): tcgen05 kernel
 cudaError_t launch_attention_tc(const LayerView& lv, const void* q, float* out, float scale, float* ws,

@@ -605,6 +605,8 @@ def main():
     ap.add_argument("--layers", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--prefill-tokens", type=int, default=0,
+                    help="run only the prefill call on a prompt of this many tokens (one layer, one sequence)")
     ap.add_argument("--no-configs", action="store_true", help="skip the other workload shapes")
     ap.add_argument("--preset", default=None, choices=["P24", "P27", "P4BASE"],
                     help="threshold preset: two tiers (default), three tiers, or 4-bit base precision")
@@ -633,6 +635,14 @@ def main():
         w = W.small(w, **over)
     if args.impl == "reference":
         run_reference(args, w)
+    elif args.prefill_tokens:
+        # the prefill call alone on one GPU (for profiling it on a small case): one JSON line with its entries
+        from paper_2512_19206_b200 import binding
+        binding.lib()
+        dev = torch.device("cuda", 0)
+        torch.cuda.set_device(dev)
+        print(json.dumps({"prefill_attention": prefill_attention_entries(binding, dev, args, (args.prefill_tokens,))}),
+              flush=True)
     else:
         run_gpu(args, w)
 

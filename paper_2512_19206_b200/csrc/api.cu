@@ -167,6 +167,35 @@ int zero_layer_state(mixkvq_cache* h, int layer, cudaStream_t st) {
   return MIXKVQ_OK;
 }
 
+// Ragged batch: writes the fills of the layer's sequences to its table in device memory (as kernel arguments: ordered
+// in the stream, no copy) and points the view at it.
+int upload_seq_table(mixkvq_cache* h, int layer, cudaStream_t st, LayerView* lv) {
+  const int B = h->cfg.batch;
+  if (B > kMaxRaggedBatch) return MIXKVQ_E_UNSUPPORTED;
+  SeqTableArgs a{};
+  a.n = B;
+  a.Hkv = h->cfg.n_kv_heads;
+  long long total = 0;
+  for (int b = 0; b < B; ++b) {
+    const int i = fi(h, layer, b);
+    a.fill[3 * b] = h->n_blocks[i];
+    a.fill[3 * b + 1] = h->r[i];
+    a.fill[3 * b + 2] = h->n_sink[i];
+    a.w[b] = attention_ws_positions_of(h->n_blocks[i], h->r[i], h->n_sink[i], h->U);
+    total += (long long)a.Hkv * a.w[b];
+  }
+  if (total >= (1ll << 31)) return MIXKVQ_E_UNSUPPORTED;
+  char* L = h->mem + kHeaderBytes + h->layer_stride * (uint64_t)layer + h->seq_off;
+  int4* seq = reinterpret_cast<int4*>(L);
+  int* prefix = reinterpret_cast<int*>(L + (size_t)B * 16);
+  if (launch_seq_table(a, seq, prefix, st) != cudaSuccess) return MIXKVQ_E_CUDA;
+  h->launches += 1;
+  lv->seq = seq;
+  lv->seq_prefix = prefix;
+  lv->seq_total = total;
+  return MIXKVQ_OK;
+}
+
 // Picks the decode-attention kernel for the layer's layout and the selected kind, enqueues it and counts its launches.
 int run_attention(mixkvq_cache* h, int layer, const void* q, float* out, float scale, float* ws, cudaStream_t st,
                   const void* new_k = nullptr, const void* new_v = nullptr, float* lse = nullptr) {
@@ -177,31 +206,10 @@ int run_attention(mixkvq_cache* h, int layer, const void* q, float* out, float s
                     (h->last_packed_writer >= 0 && h->last_packed_writer != layer)) ? 1 : 0;
   h->last_packed_writer = kNoPackedWrite;
   if (!uniform(h, layer)) {
-    // ragged batch: the fills go to the layer's table in device memory (as kernel arguments), and the split kernel
-    // and the merge walk every stream's own positions
-    const int B = h->cfg.batch;
-    if (h->tile || h->attn_kind == 1 || B > kMaxRaggedBatch) return MIXKVQ_E_UNSUPPORTED;
-    SeqTableArgs a{};
-    a.n = B;
-    a.Hkv = h->cfg.n_kv_heads;
-    long long total = 0;
-    for (int b = 0; b < B; ++b) {
-      const int i = fi(h, layer, b);
-      a.fill[3 * b] = h->n_blocks[i];
-      a.fill[3 * b + 1] = h->r[i];
-      a.fill[3 * b + 2] = h->n_sink[i];
-      a.w[b] = attention_ws_positions_of(h->n_blocks[i], h->r[i], h->n_sink[i], h->U);
-      total += (long long)a.Hkv * a.w[b];
-    }
-    if (total >= (1ll << 31)) return MIXKVQ_E_UNSUPPORTED;
-    char* L = h->mem + kHeaderBytes + h->layer_stride * (uint64_t)layer + h->seq_off;
-    int4* seq = reinterpret_cast<int4*>(L);
-    int* prefix = reinterpret_cast<int*>(L + (size_t)B * 16);
-    if (launch_seq_table(a, seq, prefix, st) != cudaSuccess) return MIXKVQ_E_CUDA;
-    h->launches += 1;
-    lv.seq = seq;
-    lv.seq_prefix = prefix;
-    lv.seq_total = total;
+    // ragged batch: the split kernel and the merge walk every stream's own positions
+    if (h->tile || h->attn_kind == 1) return MIXKVQ_E_UNSUPPORTED;
+    const int rc = upload_seq_table(h, layer, st, &lv);
+    if (rc != MIXKVQ_OK) return rc;
     lv.stage_early = 0;
   }
   int launches = 0;
@@ -472,21 +480,25 @@ int mixkvq_decode_step(mixkvq_cache* cache, int layer, const void* k_dev, const 
     if (rc != MIXKVQ_OK) return rc;
     return run_attention(cache, layer, q_dev, out_dev, softmax_scale, static_cast<float*>(workspace_dev), st);
   }
-  // full windows are flushed first, one launch per run of neighbouring sequences with the same fill
-  for (int b0 = 0; b0 < B;) {
-    int b1 = b0 + 1;
-    while (b1 < B && same_fill(cache, layer, b0, b1)) ++b1;
-    if (cache->r[fi(cache, layer, b0)] == cache->R) {
-      LayerView lv = view(cache, layer, b0, b1 - b0);
-      if (launch_flush(lv, st) != cudaSuccess) return MIXKVQ_E_CUDA;
-      cache->launches += 1;
-      cache->last_packed_writer = layer;
-      for (int b = b0; b < b1; ++b) {
+  // full windows are flushed first: one launch; in a ragged batch the kernel reads the fills from the layer's table and
+  // only the sequences whose window is full take part
+  bool any_full = false;
+  for (int b = 0; b < B; ++b) any_full = any_full || cache->r[fi(cache, layer, b)] == cache->R;
+  if (any_full) {
+    LayerView lv = view(cache, layer);
+    if (!uniform(cache, layer)) {
+      if (cache->tile) return MIXKVQ_E_UNSUPPORTED;
+      const int rc = upload_seq_table(cache, layer, st, &lv);
+      if (rc != MIXKVQ_OK) return rc;
+    }
+    if (launch_flush(lv, st) != cudaSuccess) return MIXKVQ_E_CUDA;
+    cache->launches += 1;
+    cache->last_packed_writer = layer;
+    for (int b = 0; b < B; ++b)
+      if (cache->r[fi(cache, layer, b)] == cache->R) {
         cache->n_blocks[fi(cache, layer, b)] += 1;
         cache->r[fi(cache, layer, b)] = 0;
       }
-    }
-    b0 = b1;
   }
   for (int b = 0; b < B; ++b) cache->r[fi(cache, layer, b)] += 1;   // the attention kernel stores the token at slot r - 1 and accumulates |q|
   const int rc = run_attention(cache, layer, q_dev, out_dev, softmax_scale, static_cast<float*>(workspace_dev), st, k_dev, v_dev);

@@ -117,7 +117,14 @@ flush_kernel(LayerView lv, BulkSrc src) {
 
   const int s = blockIdx.x, tid = threadIdx.x;
   const bool bulk = src.phase != 0;
-  const int block_index = lv.n_blocks + (bulk ? (int)blockIdx.y : 0);
+  int first_block = lv.n_blocks;
+  if (lv.seq != nullptr) {
+    // ragged batch (single flush only): the sequences whose window is full take part, each with its own block count
+    const int4 f = lv.seq[s / lv.Hkv];
+    if (f.y != R) return;
+    first_block = f.x;
+  }
+  const int block_index = first_block + (bulk ? (int)blockIdx.y : 0);
   const size_t tok0 = (size_t)s * src.n_tokens + src.t0 + (size_t)blockIdx.y * R;     // bulk: first token of the window
   char* state = lv.state + (size_t)s * lv.state_stride;
   char* blk = lv.base + (size_t)s * lv.base_stride + (size_t)block_index * lv.base_bytes;

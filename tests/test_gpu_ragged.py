@@ -84,6 +84,37 @@ def test_ragged_appends_and_attention(binding, preset, kwargs):
         assert np.array_equal(sal[b, hk].cpu().numpy(), a_ref)
 
 
+def test_ragged_decode_steps_flush_each_sequence_at_its_own_step(binding):
+    """140 fused decode steps on a batch whose windows fill up at different steps: every step is one attention launch,
+    a step in which some windows are full adds ONE flush launch for those sequences only."""
+    w = W.small(W.CONFIGS["llama8b"], n_layers=1, batch=4, tokens=1024, **W.P27)
+    R = w.residual_len
+    cache = U.make_cache(binding, w, max_tokens=1024)
+    oracle = {(b, hk): U.oracle_stream(w) for b in range(w.batch) for hk in (0, w.n_kv_heads - 1)}
+    k, v, q = W.tokens(w, 0, 0, 300)
+    feed(cache, oracle, w, 0, k, v, q, [300, 120, 7, 0])
+    flush_steps = 0
+    for step in range(140):
+        k, v, q = W.tokens(w, 0, 2000 + step, 1)
+        n0 = cache.launch_count()
+        due = any(cache.sequence_fill(0, b)[1] == R for b in range(w.batch))
+        out = cache.decode_step(0, k.cuda(), v.cuda(), q.cuda(), W.softmax_scale())
+        # table + split + merge, and table + flush before them when a window is full
+        assert cache.launch_count() - n0 == (5 if due else 3)
+        flush_steps += due
+        kf, vf, qf = U.f32(k), U.f32(v), U.f32(q)
+        for (b, hk), st in oracle.items():
+            st.append(kf[b, hk, 0], vf[b, hk, 0], qf[b, hk * w.g:(hk + 1) * w.g, 0])
+        if step % 35 == 34 or due:
+            o = out.cpu().numpy()
+            for (b, hk), st in oracle.items():
+                ref = st.attention(qf[b, hk * w.g:(hk + 1) * w.g, 0], W.softmax_scale())
+                assert float(np.abs(o[b, hk * w.g:(hk + 1) * w.g] - ref).max()) <= ATTN_TOL, (step, b, hk)
+    assert flush_steps >= 4                       # the four sequences reach a full window at four different steps
+    U.compare_regions(cache, 0, w, oracle)
+    assert cache.status() == 0
+
+
 def test_equal_counts_are_one_run(binding):
     """A ragged call with equal counts on a uniform batch launches what the plain append launches."""
     w = W.small(W.CONFIGS["qwen7b"], n_layers=1, batch=3, tokens=400, **W.P27)

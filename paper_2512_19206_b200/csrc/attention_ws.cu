@@ -596,23 +596,34 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
             }
         }
 
+        // The UINT4 high-plane words of a unit's first two tiles (three tiers) are requested one unit ahead inside a block.
+        uint32_t u4n[2][2] = {{0u, 0u}, {0u, 0u}};
+        auto request_plane = [&](const char* e) {
+          if constexpr (kU4 == 1) {
+            if (n4 > 0) {
+              const int n4pairs = (n4 + 1) >> 1;
+              const uint32_t* hw = reinterpret_cast<const uint32_t*>(e + 128 * n16p);
+#pragma unroll
+              for (int kk = 0; kk < 2; ++kk)
+#pragma unroll
+                for (int hp = 0; hp < 2; ++hp) {
+                  const int pp = 8 * kk + 4 * hp + t;
+                  u4n[kk][hp] = pp < n4pairs ? hw[pp * 4 + (r & 3)] : 0u;
+                }
+            }
+          }
+        };
+        if constexpr (kU4 == 1) request_plane(exu);
+
 #pragma unroll 1
         for (int iu = 0; iu < nu; ++iu) {
           wait_or_give_up(bar_u32 + ring_stage * 8u, ring_parity);
           const uint32_t stg = lane16 + ring_stage * kStageBytes;         // this lane's 16 bytes of the stage's first section
           const bool has_meta = (UPG == 1) || (done + iu == 0) || (((u + iu) & (UPG - 1)) == 0);
-          // the UINT4 high-plane words of the first two tiles of this unit are requested early
-          uint32_t u4w[2][2] = {{0u, 0u}, {0u, 0u}};
-          if (kU4 == 1 && n4 > 0) {
-            const int n4pairs = (n4 + 1) >> 1;
-            const uint32_t* hw = reinterpret_cast<const uint32_t*>(exu + 128 * n16p);
-#pragma unroll
-            for (int kk = 0; kk < 2; ++kk)
-#pragma unroll
-              for (int hp = 0; hp < 2; ++hp) {
-                const int p = 8 * kk + 4 * hp + t;
-                if (p < n4pairs) u4w[kk][hp] = hw[p * 4 + (r & 3)];
-              }
+          // this unit's UINT4 high-plane words (requested a unit ago); the next unit's are requested right away
+          const uint32_t u4w[2][2] = {{u4n[0][0], u4n[0][1]}, {u4n[1][0], u4n[1][1]}};
+          if constexpr (kU4 == 1) {
+            if (iu + 1 < nu) request_plane(exu + ex_unit);
           }
           // the key codes: two 16-byte loads per lane are the A fragments of all sixteen key tiles (with a 4-bit base the
           // first plane to run is the high plane, which lies with the block's extras in global memory)

@@ -79,8 +79,10 @@ __device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t a_desc, uint
       "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&r)[32]) {
-  uint32_t u[32];
+// A load of 32 columns of the thread's tensor-memory lane.  The registers are valid only after tmem_wait_ld32 / tmem_wait_ld16 on them (the wait
+// names the registers as operands, so that no use of them is scheduled before it).  tcgen05.wait::ld covers every load
+// the thread has issued, so a load issued before a block of arithmetic and waited for after it runs under that arithmetic.
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&u)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
@@ -90,9 +92,35 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&r)[32]) {
         "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
       : "r"(taddr)
       : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) r[i] = __uint_as_float(u[i]);
+}
+__device__ __forceinline__ void tmem_wait_ld32(uint32_t (&u)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(u[0]), "+r"(u[1]), "+r"(u[2]), "+r"(u[3]), "+r"(u[4]), "+r"(u[5]), "+r"(u[6]), "+r"(u[7]), "+r"(u[8]),
+                 "+r"(u[9]), "+r"(u[10]), "+r"(u[11]), "+r"(u[12]), "+r"(u[13]), "+r"(u[14]), "+r"(u[15]), "+r"(u[16]),
+                 "+r"(u[17]), "+r"(u[18]), "+r"(u[19]), "+r"(u[20]), "+r"(u[21]), "+r"(u[22]), "+r"(u[23]), "+r"(u[24]),
+                 "+r"(u[25]), "+r"(u[26]), "+r"(u[27]), "+r"(u[28]), "+r"(u[29]), "+r"(u[30]), "+r"(u[31])
+               :
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&u)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]), "=r"(u[8]),
+        "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld16(uint32_t (&u)[16]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(u[0]), "+r"(u[1]), "+r"(u[2]), "+r"(u[3]), "+r"(u[4]), "+r"(u[5]), "+r"(u[6]), "+r"(u[7]), "+r"(u[8]),
+                 "+r"(u[9]), "+r"(u[10]), "+r"(u[11]), "+r"(u[12]), "+r"(u[13]), "+r"(u[14]), "+r"(u[15])
+               :
+               : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&w)[8]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"r"(taddr), "r"(w[0]), "r"(w[1]),
+               "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+               : "memory");
 }
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -128,14 +156,6 @@ __device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint
       "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&w)[16]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
-      "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]), "r"(w[8]), "r"(w[9]),
-      "r"(w[10]), "r"(w[11]), "r"(w[12]), "r"(w[13]), "r"(w[14]), "r"(w[15])
-      : "memory");
-}
-
 // K, V [B * Hkv][L][128] bf16 -> tile images [B * Hkv][n_tiles][32 KB]: K as the K-major B operand of Q K^T (bf16),
 // V as the MN-major B operand of P V (fp16); rows past L are zero.  Consecutive threads write consecutive 16 bytes.
 __global__ void __launch_bounds__(256)
@@ -169,35 +189,68 @@ prefill_pack_kernel(const __nv_bfloat16* __restrict__ k, const __nv_bfloat16* __
 template <bool kMask>
 __device__ __forceinline__ void softmax_tile(uint32_t s_addr, int n_valid, float scale_log2e, float& m_run, float& l_run,
                                              float& alpha) {
-  float mx = -INFINITY;
-#pragma unroll 1
-  for (int cc = 0; cc < 4; ++cc) {
-    float s[32];
-    tmem_ld32(s_addr + 32 * cc, s);
+  // ---- pass 1: the row maximum; chunk c + 1 is in flight while chunk c is reduced
+  float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};      // four independent chains
+  {
+    uint32_t a[32], b[32];
+    auto reduce = [&](const uint32_t (&u)[32], int cc) {
 #pragma unroll
-    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, (!kMask || 32 * cc + i < n_valid) ? s[i] : -INFINITY);
+      for (int i = 0; i < 32; ++i)
+        mx4[i & 3] = fmaxf(mx4[i & 3], (!kMask || 32 * cc + i < n_valid) ? __uint_as_float(u[i]) : -INFINITY);
+    };
+    tmem_ld32_issue(s_addr, a);
+    tmem_wait_ld32(a);
+    tmem_ld32_issue(s_addr + 32, b);
+    reduce(a, 0);
+    tmem_wait_ld32(b);
+    tmem_ld32_issue(s_addr + 64, a);
+    reduce(b, 1);
+    tmem_wait_ld32(a);
+    tmem_ld32_issue(s_addr + 96, b);
+    reduce(a, 2);
+    tmem_wait_ld32(b);
+    reduce(b, 3);
   }
+  const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
   const float m_new = fmaxf(m_run, mx * scale_log2e);
   alpha = ex2(m_run - m_new);                       // 0 on the first tile
-  float sum0 = 0.f, sum1 = 0.f;
-#pragma unroll 1
-  for (int cc = 0; cc < 4; ++cc) {
-    float s[32];
-    tmem_ld32(s_addr + 32 * cc, s);
-    uint32_t w[16];
+  // ---- pass 2: probabilities in chunks of 16 columns, the next chunk in flight; P chunk c (8 columns of fp16 pairs)
+  // lies inside the S columns of chunks <= c, which are already in registers
+  float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+  {
+    uint32_t a[16], b[16];
+    auto probs = [&](const uint32_t (&u)[16], int cc) {
+      uint32_t w[8];
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      const int c0 = 32 * cc + 2 * i;
-      const float p0 = (!kMask || c0 < n_valid) ? ex2(fmaf(s[2 * i], scale_log2e, -m_new)) : 0.f;
-      const float p1 = (!kMask || c0 + 1 < n_valid) ? ex2(fmaf(s[2 * i + 1], scale_log2e, -m_new)) : 0.f;
-      sum0 += p0;
-      sum1 += p1;
-      w[i] = pack_half2(p0, p1);
+      for (int i = 0; i < 8; ++i) {
+        const int c0 = 16 * cc + 2 * i;
+        const float p0 = (!kMask || c0 < n_valid) ? ex2(fmaf(__uint_as_float(u[2 * i]), scale_log2e, -m_new)) : 0.f;
+        const float p1 = (!kMask || c0 + 1 < n_valid) ? ex2(fmaf(__uint_as_float(u[2 * i + 1]), scale_log2e, -m_new)) : 0.f;
+        if (i & 1) {
+          sum2 += p0;
+          sum3 += p1;
+        } else {
+          sum0 += p0;
+          sum1 += p1;
+        }
+        w[i] = pack_half2(p0, p1);
+      }
+      tmem_st8(s_addr + 8 * cc, w);
+    };
+    tmem_ld16_issue(s_addr, a);
+    tmem_wait_ld16(a);
+#pragma unroll
+    for (int cc = 0; cc < 8; cc += 2) {
+      tmem_ld16_issue(s_addr + 16 * (cc + 1), b);
+      probs(a, cc);                                // writes columns [8 cc, 8 cc + 8): all inside chunks <= cc
+      tmem_wait_ld16(b);
+      if (cc + 2 < 8) tmem_ld16_issue(s_addr + 16 * (cc + 2), a);
+      probs(b, cc + 1);
+      if (cc + 2 < 8) tmem_wait_ld16(a);
     }
-    tmem_st16(s_addr + 16 * cc, w);               // columns already read: chunk cc of P lies inside chunks <= cc of S
   }
   asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-  l_run = l_run * alpha + (sum0 + sum1);
+  l_run = l_run * alpha + ((sum0 + sum1) + (sum2 + sum3));
   m_run = m_new;
 }
 
@@ -358,15 +411,28 @@ prefill_attention_kernel(const __nv_bfloat16* __restrict__ q, const unsigned cha
       mbar_arrive(bar(kPReady + g));
       if (!wait(kTFull + g, (uint32_t)j & 1u)) break;
       tc_fence_after();
+      {
+        uint32_t xa[32], xb[32];
+        tmem_ld32_issue(t_addr, xa);
+        tmem_wait_ld32(xa);
+        tmem_ld32_issue(t_addr + 32, xb);
 #pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
-        float x[32];
-        tmem_ld32(t_addr + 32 * cc, x);
+        for (int i = 0; i < 32; ++i) o[i] = fmaf(o[i], alpha, __uint_as_float(xa[i]));
+        tmem_wait_ld32(xb);
+        tmem_ld32_issue(t_addr + 64, xa);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) o[32 * cc + i] = fmaf(o[32 * cc + i], alpha, x[i]);
+        for (int i = 0; i < 32; ++i) o[32 + i] = fmaf(o[32 + i], alpha, __uint_as_float(xb[i]));
+        tmem_wait_ld32(xa);
+        tmem_ld32_issue(t_addr + 96, xb);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o[64 + i] = fmaf(o[64 + i], alpha, __uint_as_float(xa[i]));
+        tmem_wait_ld32(xb);
+        // T is in registers: the tensor core may overwrite it while the last chunk is folded in
+        tc_fence_before();
+        mbar_arrive(bar(kTFree + g));
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o[96 + i] = fmaf(o[96 + i], alpha, __uint_as_float(xb[i]));
       }
-      tc_fence_before();
-      mbar_arrive(bar(kTFree + g));
     }
     if (pos < L && !dead) {
       const float inv = 1.f / l_run;

@@ -404,14 +404,32 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
     // chain of two dependent loads; they go out here, with the first copies
     const char* extras = lv.extras + (size_t)s * lv.extras_stride;
     const uint2* table = reinterpret_cast<const uint2*>(lv.table + (size_t)s * lv.table_stride);
-    uint2 pf_entry = make_uint2(0u, 0u);
+    uint2 pf_entry = make_uint2(0u, 0u), pf_entry_next = make_uint2(0u, 0u);
     uint4 pf_head = make_uint4(~0u, ~0u, ~0u, ~0u);
+    uint32_t pf_ids[4] = {0xFFFFu, 0xFFFFu, 0xFFFFu, 0xFFFFu};   // three tiers: the lane's four pairs of UINT4 channel numbers
+    // the channel lists of the block with table entry e: the head of its extras and (three tiers) the UINT4 channel
+    // numbers of the lane's pairs t, t + 4, t + 8, t + 12
+    auto request_lists = [&](const uint2& e) {
+      if (e.y & 0xFFFFu) {
+        const char* ex = extras + (size_t)e.x * 16;
+        pf_head = *reinterpret_cast<const uint4*>(ex);
+        if constexpr (kU4 == 1) {
+          const int n16p = ((e.y & 0xFF) + 1) >> 1, n4pairs = (((e.y >> 8) & 0xFF) + 1) >> 1;
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int p = 4 * i + (lane & 3);
+            pf_ids[i] = p < n4pairs ? (uint32_t)*reinterpret_cast<const uint16_t*>(ex + 2 * n16p + 2 * p) : 0xFFFFu;
+          }
+        }
+      }
+    };
     if (!logits_role) {
 #pragma unroll 1
       for (int i = 0; i < kStages; ++i) issue((ring_stage + i) & (kStages - 1), i == 0);
     } else if (n_pack > 0 && lv.stage_early) {
       pf_entry = table[wb / U];
-      if (pf_entry.y & 0xFFFFu) pf_head = *reinterpret_cast<const uint4*>(extras + (size_t)pf_entry.x * 16);
+      if (wb / U + 1 < f_nb) pf_entry_next = table[wb / U + 1];
+      request_lists(pf_entry);
     }
     dep_wait();
 
@@ -505,7 +523,8 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
         u = wb - bi * U;
         if (!lv.stage_early) {
           pf_entry = table[bi];
-          if (pf_entry.y & 0xFFFFu) pf_head = *reinterpret_cast<const uint4*>(extras + (size_t)pf_entry.x * 16);
+          if (bi + 1 < f_nb) pf_entry_next = table[bi + 1];
+          request_lists(pf_entry);
         }
       }
       // B fragments of q for the base key tiles: head r, channels 16kt + {2t, 2t+1} and {2t+8, 2t+9}, times mult(kt)
@@ -540,7 +559,12 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
         // ---- a block: its table entry, its promoted channels' query entries
         const uint2 entry = pf_entry;
         const uint4 head = pf_head;              // the first 16 bytes of the block's extras: up to 8 pairs of promoted channels
-        if (bi + 1 < f_nb) pf_entry = table[bi + 1];
+        const uint32_t ids[4] = {pf_ids[0], pf_ids[1], pf_ids[2], pf_ids[3]};
+        // Everything a block needs from global memory before its first unit was requested a whole block earlier: here
+        // go out the lists of block bi + 1 (its table entry arrived during the block before) and the entry of bi + 2.
+        pf_entry = pf_entry_next;
+        if (bi + 1 < f_nb) request_lists(pf_entry);
+        if (bi + 2 < f_nb) pf_entry_next = table[bi + 2];
         const int n16 = entry.y & 0xFF, n4 = (entry.y >> 8) & 0xFF, n16p = (n16 + 1) >> 1;
         const char* ex = extras + (size_t)entry.x * 16;                       // the block's extras
         const uint32_t ex_unit = extras_unit_bytes(n16, n4, kU4 == 2);
@@ -577,18 +601,12 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
         // pair, where the two channels' scales sit in the scale table (byte offset of the half, 0xFFFF: no channel)
         uint32_t u4q[2][2] = {{0u, 0u}, {0u, 0u}}, u4s[2][2] = {{~0u, ~0u}, {~0u, ~0u}};
         if (kU4 == 1 && n4 > 0) {
-          const int n4pairs = (n4 + 1) >> 1;
-          const unsigned char* ids4 = reinterpret_cast<const unsigned char*>(ex) + 2 * n16p;
 #pragma unroll
           for (int kk = 0; kk < 2; ++kk)
 #pragma unroll
             for (int hp = 0; hp < 2; ++hp) {
-              const int p = 8 * kk + 4 * hp + t;
-              uint32_t c0 = 255u, c1 = 255u;
-              if (p < n4pairs) {
-                c0 = ids4[2 * p];
-                c1 = ids4[2 * p + 1];
-              }
+              // pair 8 kk + 4 hp + t: its channel numbers were requested a block ahead (0xFF: no channel)
+              const uint32_t c0 = ids[2 * kk + hp] & 0xFFu, c1 = ids[2 * kk + hp] >> 8;
               const uint32_t q0 = c0 < 128 ? lds16(qfrow_u32 + 2 * c0) : 0u;
               const uint32_t q1 = c1 < 128 ? lds16(qfrow_u32 + 2 * c1) : 0u;
               u4q[kk][hp] = q0 | (q1 << 16);
@@ -799,8 +817,6 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
         done += nu;
         u = 0;
         ++bi;
-        // the next block's channel lists (its table entry has arrived by now)
-        if (bi < f_nb && (pf_entry.y & 0xFFFFu)) pf_head = *reinterpret_cast<const uint4*>(extras + (size_t)pf_entry.x * 16);
       }
       if (gave_up && lane == 0) atomicOr(lv.status, (uint32_t)MIXKVQ_DEV_COPY_TIMEOUT);
     } else {

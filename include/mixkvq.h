@@ -40,7 +40,10 @@ enum {
   MIXKVQ_E_ALIGNMENT = -3,            /* a device pointer is not 16-byte aligned                     */
   MIXKVQ_E_BUFFER_TOO_SMALL = -4,     /* cache memory or attention workspace smaller than required   */
   MIXKVQ_E_CAPACITY = -5,             /* append would exceed max_tokens                              */
-  MIXKVQ_E_CUDA = -6,                 /* a CUDA runtime call or kernel launch reported an error      */
+  MIXKVQ_E_CUDA = -6,                 /* a CUDA runtime call or kernel launch reported an error: an
+                                         append may then have advanced part of the way (the handle
+                                         counts what was enqueued before the failing launch), so the
+                                         layer's contents are undefined until mixkvq_cache_reset      */
   MIXKVQ_E_EMPTY = -7,                /* attention or selection requested on a layer with no tokens  */
   MIXKVQ_E_BUILTIN_SCRATCH = -8       /* mixkvq_decode_attention_noalloc: batch * n_kv_heads exceeds
                                          MIXKVQ_NOALLOC_MAX_STREAMS                                  */

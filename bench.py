@@ -221,7 +221,8 @@ def tier_mix(cache, w):
         d = cache.describe(layer)
         for s in range(d.n_streams):
             start = d.table_off + d.table_stride * s
-            t = cache.mem[start:start + d.n_blocks * 8].cpu().numpy().reshape(-1, 8)
+            blocks = cache.sequence_fill(layer, s // w.n_kv_heads)[0]
+            t = cache.mem[start:start + blocks * 8].cpu().numpy().reshape(-1, 8)
             n16 += int(t[:, 4].sum()); n4 += int(t[:, 5].sum()); nb += t.shape[0]
     nb = max(nb, 1)
     return n16 / nb, n4 / nb
@@ -325,6 +326,43 @@ def other_config(binding, dev, args, name, w, label, contexts=None):
     del cache
     torch.cuda.empty_cache()
     return entries
+
+
+def ragged_config(binding, dev, args):
+    """The decode-attention kernel on a batch of unequal lengths (the serving case): the headline model shape, four
+    layers, eight sequences between 640 and 32768 tokens, appended with per-sequence counts."""
+    w = W.small(W.CONFIGS["qwen7b"], n_layers=4)
+    lengths = [32768, 29000, 23500, 17000, 12345, 9000, 4097, 640]
+    cache = make_cache(binding, w, args, dev, 2 * w.residual_len + 8)
+    for layer in range(w.n_layers):
+        for t in range(0, max(lengths), PREFILL_CHUNK):
+            n = min(PREFILL_CHUNK, max(lengths) - t)
+            k, v, q = W.tokens(w, layer, t, n, device=dev)
+            cache.quantize_append_ragged(layer, k, v, q, [min(max(L - t, 0), n) for L in lengths])
+    torch.cuda.synchronize()
+    scale = W.softmax_scale()
+    out = torch.empty((w.n_layers, w.batch, w.n_q_heads, 128), dtype=torch.float32, device=dev)
+    qs = [W.decode_query(w, layer, 0, device=dev) for layer in range(w.n_layers)]
+    kern_ms, attn_us = attention_timings(cache, w, qs, out, scale)
+    n16, n4 = tier_mix(cache, w)             # of sequence 0, the longest
+    one = W.small(w, batch=1)
+    alg, units = 0.0, 0
+    for b in range(w.batch):
+        nb, r, _ = cache.sequence_fill(0, b)
+        alg += algorithmic_bytes_per_layer(one, n16, n4, r, nb * w.residual_len, 0, args.v_bits)
+        units += (nb * w.residual_len // 32 + (r + 31) // 32) * w.n_kv_heads
+    n_sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    alg += 2 * (min(2 * n_sms, units) + w.batch * w.n_kv_heads) * w.g * 130 * 4
+    peak, _ = measured_peaks()
+    entry = {"workload": "ragged batch: qwen2.5-7b shape, sequences of " + ", ".join(str(L) for L in lengths) + " tokens",
+             "shape": f"B={w.batch} Hq={w.n_q_heads} Hkv={w.n_kv_heads} G={w.group_size}", "layers_measured": w.n_layers,
+             "kernel_us": kern_ms * 1e3, "kernel_us_note": "the split kernel and the 2 us launch that writes the fill table",
+             "algorithmic_bytes": alg, "achieved_gbs": alg / (kern_ms * 1e-3) / 1e9, "frac": alg / (kern_ms * 1e-3) / 1e9 / peak,
+             "attention_us_per_layer": attn_us, "device_status": cache.status()}
+    cache.close()
+    del cache
+    torch.cuda.empty_cache()
+    return [entry]
 
 
 def tensor_peaks():
@@ -572,6 +610,9 @@ def run_gpu(args, w):
                              "config 4: qwen2.5-32b (3 distinct layers of 64)")
         cfgs += other_config(binding, dev, args, "longcot", W.small(W.CONFIGS["longcot"], n_layers=4),
                              "config 5: long-CoT stream", contexts=[8192, 32768, 65536, 131072])
+        cfgs += other_config(binding, dev, args, "qwen7b", W.small(W.CONFIGS["qwen7b"], n_layers=4, **W.P27),
+                             "config 2 with three tiers (the 2.7-bit mix), 4 layers")
+        cfgs += ragged_config(binding, dev, args)
         line["configs"] = cfgs
         line["prefill_attention"] = prefill_attention_entries(binding, dev, args)
     if world == 1 and not args.no_cpu_baseline:

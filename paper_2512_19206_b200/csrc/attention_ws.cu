@@ -54,7 +54,8 @@ __host__ __device__ constexpr int pair_bytes(bool v4) {
 constexpr int kBarsPerPair = 2 * kStages + 2;
 constexpr int kQS = 136;                     // halves per row of the query tables (272 bytes: rows fall on different banks)
 constexpr int kBarBytes = ((kPairs * kBarsPerPair * 8 + 127) / 128) * 128;
-constexpr int kSharedTail = kBarBytes + 2 * 8 * kQS * 2 + 2 * kPairs * 32;
+constexpr int kPrefixBytes = ((kMaxRaggedBatch + 1) * 4 + 15) / 16 * 16;     // a ragged batch's prefix sums
+constexpr int kSharedTail = kBarBytes + 2 * 8 * kQS * 2 + 2 * kPairs * 32 + kPrefixBytes;
 __host__ __device__ constexpr int smem_bytes(bool v4) { return kPairs * pair_bytes(v4) + kSharedTail; }
 constexpr int kResidualWeight = 3;           // an unquantized 32-token unit counts as this many packed units in the split
 constexpr int kMergeStride = 132;            // floats per head row of a pair's output in the merge
@@ -262,6 +263,7 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
   const uint32_t qf16_u32 = qb16_u32 + 8 * kQS * 2;                         // [8][kQS] q, fp16
   float* mS = reinterpret_cast<float*>(smem + kPairs * kPairBytes + kBarBytes + 2 * 8 * kQS * 2);    // [kPairs][8]
   float* lS = mS + kPairs * 8;                                                                       // [kPairs][8]
+  int* prefS = reinterpret_cast<int*>(lS + kPairs * 8);                     // ragged batch: seq_prefix[0 .. B]
 
   if (threadIdx.x < kPairs * kBarsPerPair) {
     mbar_init(tail_u32 + 8 * threadIdx.x, 1);
@@ -305,7 +307,12 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
     }
   };
   if (!lv.stage_early || lv.seq != nullptr) dep_wait();     // the table of a ragged batch is read right below
-  const long long total = lv.seq != nullptr ? (long long)lv.seq_prefix[lv.B] : (long long)Us * S;
+  if (lv.seq != nullptr) {
+    // the prefix sums go to shared memory in one round trip: the segments below search them
+    for (int i = threadIdx.x; i <= lv.B; i += kThreads) prefS[i] = lv.seq_prefix[i];
+    __syncthreads();
+  }
+  const long long total = lv.seq != nullptr ? (long long)prefS[lv.B] : (long long)Us * S;
   const long long cb = split_begin(total, gridDim.x, blockIdx.x), ce = split_begin(total, gridDim.x, blockIdx.x + 1);
 
   uint32_t ring_stage = 0;        // ring stage of the next packed unit this pair consumes
@@ -328,17 +335,17 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
     if (lv.seq != nullptr) {
       // ragged batch: the sequence whose positions hold seg (sequences without positions are stepped over)
       int b = 0;
-      while (b + 1 < lv.B && (long long)lv.seq_prefix[b + 1] <= seg) ++b;
+      while (b + 1 < lv.B && (long long)prefS[b + 1] <= seg) ++b;
       const int4 f = lv.seq[b];
       f_nb = f.x; f_r = f.y; f_ns = f.z; Us = f.w;
       packed_units = f_nb * U;
       res_units = (f_r + 31) / 32;
       bf16_units = res_units + (f_ns + 31) / 32;
-      const long long rel = seg - (long long)lv.seq_prefix[b];
+      const long long rel = seg - (long long)prefS[b];
       const int hk = (int)(rel / Us);
       s = b * lv.Hkv + hk;
       ub = (int)(rel - (long long)hk * Us);
-      ue = (int)min((long long)Us, ce - (long long)lv.seq_prefix[b] - (long long)hk * Us);
+      ue = (int)min((long long)Us, ce - (long long)prefS[b] - (long long)hk * Us);
     } else {
       s = (int)(seg / Us);
       ub = (int)(seg - (long long)s * Us);

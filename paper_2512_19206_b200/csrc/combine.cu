@@ -87,6 +87,10 @@ cudaError_t launch_combine(const float* ws, float* out, int g, int Hkv, int Hq, 
 
 // The table of a ragged batch, from the host's per-sequence fill (kernel arguments: no copy, ordered in the stream).
 __global__ void seq_table_kernel(SeqTableArgs a, int4* __restrict__ seq, int* __restrict__ seq_prefix) {
+  // a link of the chain of dependent launches: started early, waits for everything before it (a kernel that still
+  // reads the table's previous contents included), and only then lets the attention kernel behind it start
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int b = threadIdx.x;
   if (b < a.n) seq[b] = make_int4(a.fill[3 * b], a.fill[3 * b + 1], a.fill[3 * b + 2], a.w[b]);
   if (b == 0) {
@@ -100,8 +104,16 @@ __global__ void seq_table_kernel(SeqTableArgs a, int4* __restrict__ seq, int* __
 }
 
 cudaError_t launch_seq_table(const SeqTableArgs& a, int4* seq, int* seq_prefix, cudaStream_t stream) {
-  seq_table_kernel<<<1, kMaxRaggedBatch, 0, stream>>>(a, seq, seq_prefix);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(1);
+  cfg.blockDim = dim3(kMaxRaggedBatch);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, seq_table_kernel, a, seq, seq_prefix);
 }
 
 // Softmax attention over the union of disjoint token sets from the per-set results: o = sum_r w_r o_r / sum_r w_r with

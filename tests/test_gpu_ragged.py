@@ -115,6 +115,29 @@ def test_ragged_decode_steps_flush_each_sequence_at_its_own_step(binding):
     assert cache.status() == 0
 
 
+@pytest.mark.parametrize("R,G,v_bits", [(256, 128, 2), (64, 64, 4), (128, 32, 4)])
+def test_ragged_other_geometries(binding, R, G, v_bits):
+    """Ragged appends, decode steps and attention with other window and group sizes and with 4-bit values."""
+    w = W.small(W.CONFIGS["llama8b"], n_layers=1, batch=3, tokens=1024, residual_len=R, group_size=G, **W.P24)
+    cache = U.make_cache(binding, w, max_tokens=1100, v_bits=v_bits)
+    oracle = {(b, hk): U.oracle_stream(w, v_bits=v_bits) for b in range(w.batch) for hk in (0, w.n_kv_heads - 1)}
+    k, v, q = W.tokens(w, 0, 0, 900)
+    feed(cache, oracle, w, 0, k, v, q, [900, 2 * R, 33])
+    lengths = [900, 2 * R, 33]
+    U.compare_regions(cache, 0, w, oracle)
+    check_attention(cache, oracle, w, 0, 3, lengths)
+    for step in range(3):
+        k, v, q = W.tokens(w, 0, 3000 + step, 1)
+        out = cache.decode_step(0, k.cuda(), v.cuda(), q.cuda(), W.softmax_scale()).cpu().numpy()
+        kf, vf, qf = U.f32(k), U.f32(v), U.f32(q)
+        for (b, hk), st in oracle.items():
+            st.append(kf[b, hk, 0], vf[b, hk, 0], qf[b, hk * w.g:(hk + 1) * w.g, 0])
+            ref = st.attention(qf[b, hk * w.g:(hk + 1) * w.g, 0], W.softmax_scale())
+            assert float(np.abs(out[b, hk * w.g:(hk + 1) * w.g] - ref).max()) <= ATTN_TOL, (step, b, hk)
+    U.compare_regions(cache, 0, w, oracle)
+    assert cache.status() == 0
+
+
 def test_equal_counts_are_one_run(binding):
     """A ragged call with equal counts on a uniform batch launches what the plain append launches."""
     w = W.small(W.CONFIGS["qwen7b"], n_layers=1, batch=3, tokens=400, **W.P27)

@@ -274,11 +274,12 @@ int mixkvq_decode_attention_noalloc(mixkvq_cache* cache, int layer, const void* 
  * handle: the next decode attention of every layer then waits for all earlier work of the stream before its first read. */
 int mixkvq_cache_written_externally(mixkvq_cache* cache);
 
-/* Test hook for the give-up path of the decode-attention kernel (fragment layout).  While extra_bytes > 0 (a multiple
- * of 16), the barrier of the first staged copy of every warp pair is armed for extra_bytes more than the copy delivers,
- * so it never completes, and every wait gives up after max_polls polls (0: the default): the call returns, the device
- * status word carries MIXKVQ_DEV_COPY_TIMEOUT and the output rows are zero.  Nothing faults or hangs: the copies
- * themselves are the normal ones.  (0, 0) restores normal operation. */
+/* Test hook for the give-up path of the decode-attention kernel (fragment layout) and of the prefill attention.  While
+ * extra_bytes > 0 (a multiple of 16), the barrier of the first staged copy of every warp pair (decode) or of every
+ * CTA's first key tile (prefill) is armed for extra_bytes more than the copy delivers, so it never completes, and every
+ * wait gives up after max_polls polls (0: the default): the call returns, the device status word carries
+ * MIXKVQ_DEV_COPY_TIMEOUT, the decode output rows are zero and the prefill output is left unwritten.  Nothing faults or
+ * hangs: the copies themselves are the normal ones.  (0, 0) restores normal operation. */
 int mixkvq_test_arm_copy_timeout(mixkvq_cache* cache, uint32_t extra_bytes, uint32_t max_polls);
 
 /* Selects the decode-attention kernel: 0 = tensor-core kernel (default), 1 = plain-ALU kernel

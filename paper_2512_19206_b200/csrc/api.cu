@@ -526,7 +526,7 @@ int mixkvq_prefill(mixkvq_cache* cache, int layer, const void* k_dev, const void
     return MIXKVQ_E_CAPACITY;
   if (launch_prefill_attention(q_dev, k_dev, v_dev, out_dev, scratch_dev, cache->cfg.batch, cache->cfg.n_q_heads,
                                cache->cfg.n_kv_heads, n_tokens, softmax_scale, reinterpret_cast<uint32_t*>(cache->mem),
-                               cache->test_wait_polls, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+                               cache->test_wait_polls, cache->test_extra_tx, static_cast<cudaStream_t>(stream)) != cudaSuccess)
     return MIXKVQ_E_CUDA;
   cache->launches += 2;
   cache->last_packed_writer = kNoPackedWrite;

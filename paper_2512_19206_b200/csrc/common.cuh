@@ -194,7 +194,8 @@ cudaError_t launch_sink_append(const LayerView& lv, const void* k, const void* v
                                cudaStream_t stream);
 // causal full-precision attention over a prompt (tcgen05)
 cudaError_t launch_prefill_attention(const void* q, const void* k, const void* v, float* out, void* scratch, int B, int Hq,
-                                     int Hkv, int L, float scale, uint32_t* status, uint32_t max_polls, cudaStream_t stream);
+                                     int Hkv, int L, float scale, uint32_t* status, uint32_t max_polls, uint32_t debug_extra_tx,
+                                     cudaStream_t stream);
 size_t prefill_scratch_bytes(int B, int Hkv, int L);
 cudaError_t prefill_attention_setup();
 int attention_ws_positions_of(int n_blocks, int r, int n_sink, int U);

@@ -260,7 +260,7 @@ __device__ __forceinline__ void softmax_tile(uint32_t s_addr, int n_valid, float
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_attention_kernel(const __nv_bfloat16* __restrict__ q, const unsigned char* __restrict__ kt,
                          const unsigned char* __restrict__ vt, float* __restrict__ out, int BH, int Hq, int Hkv, int L,
-                         int n_tiles, int n_qtiles, float scale_log2e, uint32_t* status, uint32_t max_polls) {
+                         int n_tiles, int n_qtiles, float scale_log2e, uint32_t* status, uint32_t max_polls, uint32_t debug_extra_tx) {
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char* Qs = smem;                              // two tiles
   unsigned char* Ks = smem + 2 * kTileBytes;             // two stages
@@ -369,7 +369,8 @@ prefill_attention_kernel(const __nv_bfloat16* __restrict__ q, const unsigned cha
         const int st = j & 1;
         const uint32_t ph_prev = (uint32_t)((j >> 1) - 1) & 1u;
         if (j >= 2 && !wait(kKEmpty + st, ph_prev)) break;
-        mbar_expect_tx(bar(kKFull + st), kTileBytes);
+        // (test hook: the first copy's barrier can be armed for more bytes than arrive, so that it never completes)
+        mbar_expect_tx(bar(kKFull + st), kTileBytes + (j == 0 ? debug_extra_tx : 0u));
         bulk_copy(smem_u32(Ks + st * kTileBytes), ktg + (size_t)j * kTileBytes, kTileBytes, bar(kKFull + st));
         if (j >= 2 && !wait(kVEmpty + st, ph_prev)) {   // the K copy above is awaited below like the others
           issued = j + 1;
@@ -381,9 +382,10 @@ prefill_attention_kernel(const __nv_bfloat16* __restrict__ q, const unsigned cha
         issued = j + 1;
       }
       // no copy may be in flight when the CTA ends: the last copy into each stage has landed once its barrier's phase is over
-      dead = false;
       for (int j = max(0, issued - 2); j < issued; ++j) {
+        dead = false;                                    // every one of these waits is made, whatever the others did
         wait(kKFull + (j & 1), (uint32_t)(j >> 1) & 1u);
+        dead = false;
         wait(kVFull + (j & 1), (uint32_t)(j >> 1) & 1u);
       }
     }
@@ -457,7 +459,8 @@ size_t prefill_scratch_bytes(int B, int Hkv, int L) {
 }
 
 cudaError_t launch_prefill_attention(const void* q, const void* k, const void* v, float* out, void* scratch, int B, int Hq,
-                                     int Hkv, int L, float scale, uint32_t* status, uint32_t max_polls, cudaStream_t stream) {
+                                     int Hkv, int L, float scale, uint32_t* status, uint32_t max_polls, uint32_t debug_extra_tx,
+                                     cudaStream_t stream) {
   const int n_tiles = (L + kTile - 1) / kTile, n_qtiles = (L + kQRows - 1) / kQRows;
   unsigned char* kt = static_cast<unsigned char*>(scratch);
   unsigned char* vt = kt + (size_t)B * Hkv * n_tiles * kTileBytes;
@@ -465,7 +468,7 @@ cudaError_t launch_prefill_attention(const void* q, const void* k, const void* v
       static_cast<const __nv_bfloat16*>(k), static_cast<const __nv_bfloat16*>(v), kt, vt, L, n_tiles);
   prefill_attention_kernel<<<(unsigned)(n_qtiles * B * Hq), kThreads, kSmem, stream>>>(
       static_cast<const __nv_bfloat16*>(q), kt, vt, out, B * Hq, Hq, Hkv, L, n_tiles, n_qtiles,
-      scale * 1.4426950408889634f, status, max_polls ? max_polls : kPolls);
+      scale * 1.4426950408889634f, status, max_polls ? max_polls : kPolls, debug_extra_tx);
   return cudaGetLastError();
 }
 

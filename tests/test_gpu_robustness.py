@@ -52,6 +52,29 @@ def test_a_wait_that_runs_out_returns_with_the_status_bit(binding):
     assert torch.equal(again, want)
 
 
+def test_a_prefill_wait_that_runs_out_returns_with_the_status_bit(binding):
+    """The same for the prefill attention: the barrier of every CTA's first key tile never completes, every role of the
+    CTA gives up after 64 polls, the call returns with the status bit and writes no output; after a reset the call works."""
+    w = W.small(W.CONFIGS["qwen7b"], n_layers=1, batch=1, tokens=600, **W.P24)
+    k, v, q = [t.cuda() for t in W.tokens(w, 0, 0, 600)]
+    cache = U.make_cache(binding, w)
+    want = cache.prefill(0, k, v, q, W.softmax_scale())
+    assert cache.status() == 0
+    cache.reset()
+    cache.test_arm_copy_timeout(16, 64)
+    out = torch.full_like(want, 7.0)
+    cache.prefill(0, k, v, q, W.softmax_scale(), out=out)
+    torch.cuda.synchronize()                                   # the call came back
+    assert cache.status() & binding.DEV_COPY_TIMEOUT
+    assert bool((out == 7.0).all())                            # no row was written
+    cache.test_arm_copy_timeout(0, 0)
+    cache.reset()
+    assert cache.status() == 0
+    again = cache.prefill(0, k, v, q, W.softmax_scale())
+    assert cache.status() == 0
+    assert torch.equal(again, want)
+
+
 def test_attention_right_after_a_flush_and_after_an_external_write(binding):
     """Packed blocks are requested ahead of the stream-order wait except right after a flush of the same layer (or
     when the caller says it wrote cache memory itself); the results do not depend on which path was taken."""

@@ -27,6 +27,23 @@ def test_library_exports_every_declared_symbol(binding):
     assert sorted(binding.EXPORTS) == declared
 
 
+def test_header_is_plain_c_and_cpp(tmp_path):
+    """include/mixkvq.h compiles by itself as C99 and as C++ (no CUDA or torch type in any signature), and the struct
+    sizes the binding assumes are the compiler's."""
+    import subprocess
+    inc = os.path.join(ROOT, "include")
+    src = ('#include "mixkvq.h"\n#include <stdio.h>\n'
+           'int main(void) { printf("%zu %zu\\n", sizeof(mixkvq_config), sizeof(mixkvq_layout_desc)); return 0; }\n')
+    for compiler, name, std in (("gcc", "t.c", "-std=c99"), ("g++", "t.cpp", "-std=c++14")):
+        f = tmp_path / name
+        f.write_text(src)
+        exe = tmp_path / (name + ".out")
+        subprocess.run([compiler, std, "-Wall", "-Werror", "-pedantic", "-I", inc, str(f), "-o", str(exe)], check=True)
+        sizes = subprocess.run([str(exe)], capture_output=True, text=True, check=True).stdout.split()
+        from paper_2512_19206_b200 import binding as b
+        assert [int(x) for x in sizes] == [C.sizeof(b.Config), C.sizeof(b.LayoutDesc)]
+
+
 def test_config_struct_matches_header(binding):
     assert C.sizeof(binding.Config) == 80          # 14 int32/float fields, one uint64, two budgets, sink length, pad
     assert C.sizeof(binding.LayoutDesc) == 13 * 8 + 4 * 4 + 2 * 8 + 2 * 4

@@ -59,6 +59,10 @@ constexpr int kSharedTail = kBarBytes + 2 * 8 * kQS * 2 + 2 * kPairs * 32 + kPre
 __host__ __device__ constexpr int smem_bytes(bool v4) { return kPairs * pair_bytes(v4) + kSharedTail; }
 constexpr int kResidualWeight = 3;           // an unquantized 32-token unit counts as this many packed units in the split
 constexpr int kMergeStride = 132;            // floats per head row of a pair's output in the merge
+// With a 4-bit base the logits warp runs two key passes per unit and is by far the longer role: the promoted channels'
+// tile is then the values warp's work (with the other mixes it stays with the logits warp: a stall of the values warp on
+// global loads delays the ring's refill, which costs more than the tile does).
+__host__ __device__ constexpr bool promoted_in_values(int u4) { return u4 == 2; }
 constexpr float kMaxSlack = 3.0f;            // a packed unit's probabilities are at most 2^kMaxSlack (log2 domain)
 // A wait on a barrier polls at most this many times; a poll suspends the thread for up to about a microsecond, so
 // the wait gives up after about two seconds at the latest (a few milliseconds if the polls return at once).
@@ -433,10 +437,11 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
     if (!logits_role) {
 #pragma unroll 1
       for (int i = 0; i < kStages; ++i) issue((ring_stage + i) & (kStages - 1), i == 0);
-    } else if (n_pack > 0 && lv.stage_early) {
+    }
+    if (n_pack > 0 && lv.stage_early && (logits_role || promoted_in_values(kU4))) {
       pf_entry = table[wb / U];
       if (wb / U + 1 < f_nb) pf_entry_next = table[wb / U + 1];
-      request_lists(pf_entry);
+      if (logits_role != promoted_in_values(kU4)) request_lists(pf_entry);
     }
     dep_wait();
 
@@ -531,7 +536,7 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
         if (!lv.stage_early) {
           pf_entry = table[bi];
           if (bi + 1 < f_nb) pf_entry_next = table[bi + 1];
-          request_lists(pf_entry);
+          if constexpr (!promoted_in_values(kU4)) request_lists(pf_entry);
         }
       }
       // B fragments of q for the base key tiles: head r, channels 16kt + {2t, 2t+1} and {2t+8, 2t+9}, times mult(kt)
@@ -570,7 +575,9 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
         // Everything a block needs from global memory before its first unit was requested a whole block earlier: here
         // go out the lists of block bi + 1 (its table entry arrived during the block before) and the entry of bi + 2.
         pf_entry = pf_entry_next;
-        if (bi + 1 < f_nb) request_lists(pf_entry);
+        if constexpr (!promoted_in_values(kU4)) {
+          if (bi + 1 < f_nb) request_lists(pf_entry);
+        }
         if (bi + 2 < f_nb) pf_entry_next = table[bi + 2];
         const int n16 = entry.y & 0xFF, n4 = (entry.y >> 8) & 0xFF, n16p = (n16 + 1) >> 1;
         const char* ex = extras + (size_t)entry.x * 16;                       // the block's extras
@@ -592,7 +599,7 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
             xa[mt][3] = *reinterpret_cast<const uint32_t*>(e + xa_hi + mt * 64 + 32);
           }
         };
-        if (n16 > 0) {
+        if (!promoted_in_values(kU4) && n16 > 0) {
           load_xa(exu);
           auto gather_q = [&](int p, uint32_t word) -> uint32_t {       // pair p < 8: its two channel numbers are in `word`
             if (p >= n16p) return 0u;
@@ -719,7 +726,7 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
             key_pass(hw0, hw1, true, false);
           }
           // ---- promoted channels (raw bf16 keys) with a gathered q
-          if (n16 > 0) {
+          if (!promoted_in_values(kU4) && n16 > 0) {
 #pragma unroll
             for (int mt = 0; mt < 2; ++mt) mma_bf16(Sx[mt], xa[mt][0], xa[mt][1], xa[mt][2], xa[mt][3], xb0, xb1);
             // the registers are free again: request the next unit's pairs now, most of an iteration ahead of their use
@@ -966,8 +973,69 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
       const uint32_t lane16 = ring_u32 + lane * 16, lane32 = ring_u32 + kLBufBase + lane * 32;
       const uint32_t lane8 = ring_u32 + kLBufBase + kLBufZeroOff + lane * 8;
       const uint32_t vm_rd = ring_u32 + kUnitOff + 2048 + lane * (4 * VG);
+      // ---- 4-bit base: the promoted channels' tile (raw bf16 keys from the blocks' extras, a gathered q) is added here
+      // to the logits the partner hands over.  Requested ahead like everything from global memory: table entries two
+      // blocks, channel lists one block, a unit's rows one unit.
+      const uint32_t qrow_v = qb16_u32 + r * (kQS * 2);
+      int vbi = 0, vcur = 0, vleft = 0;           // block, unit inside it, units of the block left for this warp
+      int n16 = 0, n16p = 0;
+      const char* ex = extras;                    // the block's extras, and those of the current unit
+      const char* exu = extras;
+      uint32_t ex_unit = 0;
+      uint32_t xb0 = 0u, xb1 = 0u, xa[2][4] = {{0u, 0u, 0u, 0u}, {0u, 0u, 0u, 0u}};     // as in the logits warp
+      auto load_xa = [&](const char* e) {
+        const int xa_lo = (min(t, n16p - 1) * 32 + r) * 4, xa_hi = (min(t + 4, n16p - 1) * 32 + r) * 4;
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+          xa[mt][0] = *reinterpret_cast<const uint32_t*>(e + xa_lo + mt * 64);
+          xa[mt][1] = *reinterpret_cast<const uint32_t*>(e + xa_lo + mt * 64 + 32);
+          xa[mt][2] = *reinterpret_cast<const uint32_t*>(e + xa_hi + mt * 64);
+          xa[mt][3] = *reinterpret_cast<const uint32_t*>(e + xa_hi + mt * 64 + 32);
+        }
+      };
+      if constexpr (promoted_in_values(kU4)) {
+        if (n_pack > 0) {
+          vbi = wb / U;
+          vcur = wb - vbi * U;
+          if (!lv.stage_early) {
+            pf_entry = table[vbi];
+            if (vbi + 1 < f_nb) pf_entry_next = table[vbi + 1];
+            request_lists(pf_entry);
+          }
+        }
+      }
 #pragma unroll 1
       for (int done = 0; done < n_pack; ++done) {
+        if constexpr (promoted_in_values(kU4)) {
+          if (vleft == 0) {
+            // a block: its table entry and lists arrived a block ago; the next block's lists and the entry after that go out now
+            const uint2 entry = pf_entry;
+            const uint4 head = pf_head;          // the first 16 bytes of the block's extras: up to 8 pairs of promoted channels
+            pf_entry = pf_entry_next;
+            if (vbi + 1 < f_nb) request_lists(pf_entry);
+            if (vbi + 2 < f_nb) pf_entry_next = table[vbi + 2];
+            n16 = entry.y & 0xFF;
+            n16p = (n16 + 1) >> 1;
+            const int n4 = (entry.y >> 8) & 0xFF;
+            ex = extras + (size_t)entry.x * 16;
+            ex_unit = extras_unit_bytes(n16, n4, true);
+            exu = ex + extras_header_bytes(n16, n4) + (size_t)vcur * ex_unit;
+            vleft = min(U - vcur, n_pack - done);
+            xb0 = xb1 = 0u;
+            if (n16 > 0) {
+              load_xa(exu);
+              auto gather_q = [&](int p, uint32_t word) -> uint32_t {     // pair p < 8: its two channel numbers are in `word`
+                if (p >= n16p) return 0u;
+                const uint32_t cc = word >> (16 * (p & 1));
+                const uint32_t c0 = cc & 0xFF, c1 = (cc >> 8) & 0xFF;
+                const uint32_t lo = (c0 < 128) ? lds16(qrow_v + 2 * c0) : 0u, hi = (c1 < 128) ? lds16(qrow_v + 2 * c1) : 0u;
+                return lo | (hi << 16);
+              };
+              xb0 = gather_q(t, (t & 2) ? head.y : head.x);
+              xb1 = gather_q(t + 4, (t & 2) ? head.w : head.z);
+            }
+          }
+        }
         wait_or_give_up(bar_u32 + ring_stage * 8u, ring_parity);
         const uint32_t st = lane16 + ring_stage * kStageBytes + kUnitOff;      // this lane's 16 bytes of the unit's first section
         // ---- value-group preparation (lane = token).  The tables of the previous unit were last read before the
@@ -997,8 +1065,48 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
         const uint32_t lb = lane32 + ring_stage * kLBufBytes;
         const uint4 s0 = lds128(lb), s1 = lds128(lb + 16);
         const uint2 zq = lds64(lane8 + ring_stage * kLBufBytes);
-        const float sx[2][4] = {{__uint_as_float(s0.x), __uint_as_float(s0.y), __uint_as_float(s0.z), __uint_as_float(s0.w)},
-                                {__uint_as_float(s1.x), __uint_as_float(s1.y), __uint_as_float(s1.z), __uint_as_float(s1.w)}};
+        float sx[2][4] = {{__uint_as_float(s0.x), __uint_as_float(s0.y), __uint_as_float(s0.z), __uint_as_float(s0.w)},
+                          {__uint_as_float(s1.x), __uint_as_float(s1.y), __uint_as_float(s1.z), __uint_as_float(s1.w)}};
+        if constexpr (promoted_in_values(kU4)) {
+          // ---- promoted channels (raw bf16 keys) with a gathered q
+          if (n16 > 0) {
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt) mma_bf16(sx[mt], xa[mt][0], xa[mt][1], xa[mt][2], xa[mt][3], xb0, xb1);
+            // the registers are free again: request the next unit's pairs now, a whole iteration ahead of their use
+            if (vleft > 1) load_xa(exu + ex_unit);
+            for (int kk = 1; kk * 8 < n16p; ++kk) {       // more than 16 promoted channels
+              uint32_t a[2][4], id0 = 0xFFFFFFFFu, id1 = 0xFFFFFFFFu;
+              const uint32_t* xw = reinterpret_cast<const uint32_t*>(exu);
+              const int p0 = 8 * kk + t, p1 = p0 + 4;
+#pragma unroll
+              for (int mt = 0; mt < 2; ++mt) a[mt][0] = a[mt][1] = a[mt][2] = a[mt][3] = 0;
+              if (p0 < n16p) {
+                id0 = *reinterpret_cast<const uint16_t*>(ex + 2 * p0);
+#pragma unroll
+                for (int mt = 0; mt < 2; ++mt) {
+                  a[mt][0] = xw[p0 * 32 + mt * 16 + r];
+                  a[mt][1] = xw[p0 * 32 + mt * 16 + 8 + r];
+                }
+              }
+              if (p1 < n16p) {
+                id1 = *reinterpret_cast<const uint16_t*>(ex + 2 * p1);
+#pragma unroll
+                for (int mt = 0; mt < 2; ++mt) {
+                  a[mt][2] = xw[p1 * 32 + mt * 16 + r];
+                  a[mt][3] = xw[p1 * 32 + mt * 16 + 8 + r];
+                }
+              }
+              auto gather_bf16 = [&](uint32_t cc) -> uint32_t {
+                const uint32_t c0 = cc & 0xFF, c1 = (cc >> 8) & 0xFF;
+                const uint32_t lo = (c0 < 128) ? lds16(qrow_v + 2 * c0) : 0u, hi = (c1 < 128) ? lds16(qrow_v + 2 * c1) : 0u;
+                return lo | (hi << 16);
+              };
+              const uint32_t b0 = gather_bf16(id0), b1 = gather_bf16(id1);
+#pragma unroll
+              for (int mt = 0; mt < 2; ++mt) mma_bf16(sx[mt], a[mt][0], a[mt][1], a[mt][2], a[mt][3], b0, b1);
+            }
+          }
+        }
         // logit = (sx + q . z) * scale: the zero-point term of the key group is the same for every token of the unit
         const float zl0 = __uint_as_float(zq.x) * scale_log2e, zl1 = __uint_as_float(zq.y) * scale_log2e;
         // ---- online softmax (log2 domain); heads 2t, 2t+1; tokens r, r+8 of each m-tile.
@@ -1069,6 +1177,14 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
         __syncwarp();
         issue(ring_stage, false);
         advance_stage();
+        if constexpr (promoted_in_values(kU4)) {
+          exu += ex_unit;
+          ++vcur;
+          if (--vleft == 0) {
+            ++vbi;
+            vcur = 0;
+          }
+        }
       }
       if (gave_up) {
         if (lane == 0) atomicOr(lv.status, (uint32_t)MIXKVQ_DEV_COPY_TIMEOUT);

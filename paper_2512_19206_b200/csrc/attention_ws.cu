@@ -59,10 +59,12 @@ constexpr int kSharedTail = kBarBytes + 2 * 8 * kQS * 2 + 2 * kPairs * 32 + kPre
 __host__ __device__ constexpr int smem_bytes(bool v4) { return kPairs * pair_bytes(v4) + kSharedTail; }
 constexpr int kResidualWeight = 3;           // an unquantized 32-token unit counts as this many packed units in the split
 constexpr int kMergeStride = 132;            // floats per head row of a pair's output in the merge
-// With a 4-bit base the logits warp runs two key passes per unit and is by far the longer role: the promoted channels'
-// tile is then the values warp's work (with the other mixes it stays with the logits warp: a stall of the values warp on
-// global loads delays the ring's refill, which costs more than the tile does).
-__host__ __device__ constexpr bool promoted_in_values(int u4) { return u4 == 2; }
+// With three tiers and with a 4-bit base the logits warp is by far the longer role (further tiles for the UINT4 high
+// plane, or a second key pass): the promoted channels' tile is then the values warp's work.  With two tiers it stays with
+// the logits warp: a stall of the values warp on global loads delays the ring's refill, which costs more there than the
+// tile does.  (The gathered UINT4 tiles stay with the logits warp in every case: moved, they made the values warp the
+// longer role and the kernel slower.)
+__host__ __device__ constexpr bool promoted_in_values(int u4) { return u4 != 0; }
 constexpr float kMaxSlack = 3.0f;            // a packed unit's probabilities are at most 2^kMaxSlack (log2 domain)
 // A wait on a barrier polls at most this many times; a poll suspends the thread for up to about a microsecond, so
 // the wait gives up after about two seconds at the latest (a few milliseconds if the polls return at once).
@@ -441,7 +443,7 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
     if (n_pack > 0 && lv.stage_early && (logits_role || promoted_in_values(kU4))) {
       pf_entry = table[wb / U];
       if (wb / U + 1 < f_nb) pf_entry_next = table[wb / U + 1];
-      if (logits_role != promoted_in_values(kU4)) request_lists(pf_entry);
+      if (logits_role ? kU4 != 2 : promoted_in_values(kU4)) request_lists(pf_entry);     // whoever needs the lists
     }
     dep_wait();
 
@@ -536,7 +538,7 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
         if (!lv.stage_early) {
           pf_entry = table[bi];
           if (bi + 1 < f_nb) pf_entry_next = table[bi + 1];
-          if constexpr (!promoted_in_values(kU4)) request_lists(pf_entry);
+          if constexpr (kU4 != 2) request_lists(pf_entry);
         }
       }
       // B fragments of q for the base key tiles: head r, channels 16kt + {2t, 2t+1} and {2t+8, 2t+9}, times mult(kt)
@@ -575,7 +577,7 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
         // Everything a block needs from global memory before its first unit was requested a whole block earlier: here
         // go out the lists of block bi + 1 (its table entry arrived during the block before) and the entry of bi + 2.
         pf_entry = pf_entry_next;
-        if constexpr (!promoted_in_values(kU4)) {
+        if constexpr (kU4 != 2) {          // the UINT4 channel numbers (three tiers) or the promoted channels' (two tiers)
           if (bi + 1 < f_nb) request_lists(pf_entry);
         }
         if (bi + 2 < f_nb) pf_entry_next = table[bi + 2];
@@ -973,7 +975,7 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
       const uint32_t lane16 = ring_u32 + lane * 16, lane32 = ring_u32 + kLBufBase + lane * 32;
       const uint32_t lane8 = ring_u32 + kLBufBase + kLBufZeroOff + lane * 8;
       const uint32_t vm_rd = ring_u32 + kUnitOff + 2048 + lane * (4 * VG);
-      // ---- 4-bit base: the promoted channels' tile (raw bf16 keys from the blocks' extras, a gathered q) is added here
+      // ---- three tiers, 4-bit base: the promoted channels' tile (raw bf16 keys from the blocks' extras, a gathered q) is added here
       // to the logits the partner hands over.  Requested ahead like everything from global memory: table entries two
       // blocks, channel lists one block, a unit's rows one unit.
       const uint32_t qrow_v = qb16_u32 + r * (kQS * 2);
@@ -1018,7 +1020,7 @@ attention_ws_kernel(LayerView lv, const __nv_bfloat16* __restrict__ q, float sca
             n16p = (n16 + 1) >> 1;
             const int n4 = (entry.y >> 8) & 0xFF;
             ex = extras + (size_t)entry.x * 16;
-            ex_unit = extras_unit_bytes(n16, n4, true);
+            ex_unit = extras_unit_bytes(n16, n4, kU4 == 2);
             exu = ex + extras_header_bytes(n16, n4) + (size_t)vcur * ex_unit;
             vleft = min(U - vcur, n_pack - done);
             xb0 = xb1 = 0u;
